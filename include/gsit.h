@@ -1,0 +1,146 @@
+/*
+ * gsit.h -- C ABI of the Interlaced-Mask (IM) attention library for NVIDIA B200 (sm_100a).
+ *
+ * The library computes the attention of GsiT (arXiv 2505.01068): one set of query/key/value weights
+ * is applied to the concatenation V_m = [V_0; V_1; V_2] of three modality sequences (Section
+ * "Multimodal Transformers as Graphs"), and a 3x3 pattern of modality blocks -- the Interlaced Mask
+ * of Section "All-Modal-In-One Fusion", Eq. IFM / IEM -- decides which query block may attend which
+ * key block.  Only the open blocks are ever computed and the softmax runs over just their keys
+ * (Section "Inner Decomposition for Efficiency"); a dense masked L x L product is never formed.
+ *
+ * General conventions
+ *   - Segments are positional: s = 0,1,2 in the order the caller concatenated them, lengths
+ *     seg_len[s], L = seg_len[0]+seg_len[1]+seg_len[2].
+ *   - valid_len (DEVICE pointer, int32 [batch][3], or NULL = no padding) gives, per sample and segment,
+ *     the number of real rows at the start of the segment; the rest of the segment is padding.
+ *     Values outside [0, seg_len[s]] are clamped on the device and GSIT_DEVFLAG_CLAMPED is raised.
+ *   - Padded rows of every output are exactly +0.0 (lse: -inf).  A real query whose open blocks hold no
+ *     real key also yields +0.0 / -inf.  Contents of padded input rows (NaN and Inf included) never
+ *     influence a real output row.
+ *   - All tensors are row-major and live in DEVICE memory unless stated otherwise; the caller owns every
+ *     buffer; the library allocates nothing, keeps no pointer after a call returns and launches all work
+ *     asynchronously on the given stream without synchronising the host.
+ *   - dtype GSIT_F32: activations and weights are float.  dtype GSIT_BF16: activations and weights are
+ *     bfloat16, accumulation is float.  Biases, LayerNorm parameters, lse and the residual stream
+ *     x / y of gsit_im_layer_fwd are float in both cases.
+ *   - Errors are reported by return code only; nothing aborts, throws or traps.  Problems visible on the
+ *     host (NULL pointers, bad sizes, unsupported shapes, misalignment, short workspace) are rejected
+ *     before any launch.  There is no CPU fallback.
+ *   - GSIT_BF16 needs: d_model % 16 == 0, head_dim in {8,16,32,64}, every row stride a multiple of 8
+ *     elements, pointers 16-byte aligned.  GSIT_F32 needs head_dim <= 256.
+ */
+#ifndef GSIT_H_
+#define GSIT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  GSIT_OK = 0,
+  GSIT_ERR_INVALID_ARG = 1,  /* NULL pointer, non-positive size, d_model % heads != 0, bad enum, misalignment */
+  GSIT_ERR_UNSUPPORTED = 2,  /* shape or dtype outside what the kernels cover */
+  GSIT_ERR_WORKSPACE = 3,    /* workspace NULL or smaller than gsit_workspace_bytes() */
+  GSIT_ERR_CUDA = 4,         /* a CUDA runtime / driver call failed */
+  GSIT_ERR_TIMEOUT = 5       /* a bounded device-side wait expired (see gsit_last_device_status) */
+} gsit_status;
+
+typedef enum { GSIT_F32 = 0, GSIT_BF16 = 1 } gsit_dtype;
+
+/* Which blocks are open.  Rows = query segment s, columns = key segment r.
+ *   INTER_FWD: s attends (s+1)%3   -- M_inter^forward of Eq. IFM  (J O J / J J O / O J J)
+ *   INTER_BWD: s attends (s+2)%3   -- M_inter^backward of Eq. IFM (J J O / O J J / J O J)
+ *   INTRA:     s attends s         -- M_intra, the IEM            (O J J / J O J / J J O)
+ *   CUSTOM:    bit (3*s + r) of custom_mask set = block open (ablation structures of Appendix
+ *              "Graph Structures", the unmasked naive graph 0x1FF, ...).  With several open blocks in a
+ *              block row the softmax runs over the union of their real keys. */
+typedef enum {
+  GSIT_PHASE_INTER_FWD = 0,
+  GSIT_PHASE_INTER_BWD = 1,
+  GSIT_PHASE_INTRA = 2,
+  GSIT_PHASE_CUSTOM = 3
+} gsit_phase;
+
+/* Problem description shared by all calls.  HOST struct, passed by pointer, read during the call only. */
+typedef struct gsit_shape {
+  int32_t batch;            /* B >= 1 */
+  int32_t seg_len[3];       /* each >= 0, sum >= 1 */
+  int32_t d_model;          /* d = heads * head_dim */
+  int32_t heads;            /* H */
+  const int32_t* valid_len; /* DEVICE int32 [B][3] or NULL */
+  int32_t dtype;            /* gsit_dtype */
+  int32_t phase;            /* gsit_phase */
+  uint32_t custom_mask;     /* used when phase == GSIT_PHASE_CUSTOM */
+  float scale;              /* score scale; <= 0 selects 1/sqrt(head_dim) */
+} gsit_shape;
+
+/* Weights of one IM encoder layer (HOST struct of DEVICE pointers).  Matrices are [out_features,
+ * in_features] row-major in shape->dtype; y = x W^T.  Biases and LayerNorm vectors are float and may be
+ * NULL (bias 0, gamma 1, beta 0). */
+typedef struct gsit_layer_weights {
+  const float* ln1_gamma; const float* ln1_beta;   /* [d] */
+  const void* w_qkv;  const float* b_qkv;          /* [3d, d] rows = (W_q; W_k; W_v), [3d] */
+  const void* w_o;    const float* b_o;            /* [d, d], [d] */
+  const float* ln2_gamma; const float* ln2_beta;   /* [d] */
+  const void* w_1;    const float* b_1;            /* [d_ff, d], [d_ff] */
+  const void* w_2;    const float* b_2;            /* [d, d_ff], [d] */
+  int32_t d_ff;                                    /* width of the MLP (the paper's d^p >= d^f) */
+  float ln_eps;                                    /* <= 0 selects 1e-5 */
+} gsit_layer_weights;
+
+typedef void* gsit_stream; /* a cudaStream_t; NULL = the legacy default stream */
+
+/* Shared QKV projection (Section "Multimodal Transformers as Graphs"; Appendix A, Eq. adjmat_all:
+ * A = (W_q V_m)(W_k V_m)^T, i.e. one W_q, W_k, W_v for the whole concatenated sequence).
+ *   x     [B, L, d]  row stride x_row_stride elements (>= d)
+ *   w_qkv [3d, d], b_qkv float [3d] or NULL
+ *   qkv   [B, L, 3, H, hd] contiguous: qkv[b,p,0] = q, [b,p,1] = k, [b,p,2] = v; padded rows = 0. */
+gsit_status gsit_im_qkv_proj(const gsit_shape* shape, const void* x, int64_t x_row_stride, const void* w_qkv,
+                             const float* b_qkv, void* qkv, gsit_stream stream);
+
+/* IM attention (Eq. "All-Modal-In-One fusion": G = softmax(MHSA_1(V_m) + M), aggregation MHSA_2; computed
+ * block-wise as Section "Inner Decomposition" and Appendix A "From Set to Set Aggregation" describe).
+ *   q, k, v  [B, L, H, hd] views with a common row stride (elements) between sequence positions:
+ *            d for three separate tensors, 3d for the fused buffer written by gsit_im_qkv_proj
+ *   out      [B, L, d] contiguous, heads concatenated along features
+ *   lse      float [B, H, L] or NULL: natural-log-sum-exp of the scaled scores of each row
+ *   workspace / workspace_bytes: gsit_workspace_bytes(shape, GSIT_CALL_ATTENTION, 0) bytes (may be 0/NULL). */
+gsit_status gsit_im_attention_fwd(const gsit_shape* shape, const void* q, const void* k, const void* v,
+                                  int64_t row_stride, void* out, float* lse, void* workspace,
+                                  size_t workspace_bytes, gsit_stream stream);
+
+/* One IM encoder layer, a = MLP o MHSA_2 (Eq. 1 / Eq. "All-Modal-In-One fusion"), in the pre-LayerNorm
+ * form with residuals:   h = LN1(x); O = IM-attention(h W_qkv^T + b_qkv);
+ *                        y1 = x + O W_o^T + b_o;   y = y1 + relu(LN2(y1) W_1^T + b_1) W_2^T + b_2.
+ *   x  float [B, L, d] with row stride x_row_stride;  y  float [B, L, d] with row stride y_row_stride
+ *      (strides let two encoders write the halves of one [B, L, 2d] buffer -- the feature concat of the
+ *      fusion encoder pair).  x and y must not overlap.
+ *   workspace: gsit_workspace_bytes(shape, GSIT_CALL_LAYER, d_ff) bytes, 256-byte aligned. */
+gsit_status gsit_im_layer_fwd(const gsit_shape* shape, const gsit_layer_weights* weights, const float* x,
+                              int64_t x_row_stride, float* y, int64_t y_row_stride, void* workspace,
+                              size_t workspace_bytes, gsit_stream stream);
+
+typedef enum { GSIT_CALL_QKV_PROJ = 0, GSIT_CALL_ATTENTION = 1, GSIT_CALL_LAYER = 2 } gsit_call;
+
+/* Scratch bytes the given call needs for this shape (d_ff is read for GSIT_CALL_LAYER only).
+ * Returns 0 for calls that need none and (size_t)-1 for an invalid shape. */
+size_t gsit_workspace_bytes(const gsit_shape* shape, int which_call, int32_t d_ff);
+
+/* Device status flags, accumulated by kernels of this library on the current device. */
+#define GSIT_DEVFLAG_CLAMPED 1u  /* a valid_len value was outside [0, seg_len] and was clamped */
+#define GSIT_DEVFLAG_TIMEOUT 2u  /* a bounded wait on an asynchronous copy expired; results are invalid */
+
+/* Synchronises `stream`, reads and clears the device status flags into *flags (HOST, may be NULL).
+ * Returns GSIT_ERR_TIMEOUT if GSIT_DEVFLAG_TIMEOUT was set, GSIT_ERR_CUDA on a CUDA error, else GSIT_OK. */
+gsit_status gsit_last_device_status(gsit_stream stream, uint32_t* flags);
+
+const char* gsit_status_string(gsit_status status);
+int gsit_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GSIT_H_ */

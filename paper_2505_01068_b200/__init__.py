@@ -1,0 +1,12 @@
+"""B200-native Interlaced-Mask attention of GsiT (arXiv 2505.01068): thin Python access to libgsit.so.
+
+The C ABI is declared in include/gsit.h; `binding` marshals torch tensors into it.  Nothing here computes:
+all arithmetic runs in the library's CUDA kernels, and a missing library raises.
+"""
+from .binding import (CALL_ATTENTION, CALL_LAYER, CALL_QKV_PROJ, DEVFLAG_CLAMPED, DEVFLAG_TIMEOUT, DTYPE_BF16,
+                      DTYPE_F32, EXPORTS, PHASE_CUSTOM, PHASE_INTER_BWD, PHASE_INTER_FWD, PHASE_INTRA, GsitError,
+                      im_attention_fwd, im_layer_fwd, im_qkv_proj, last_device_status, load, make_shape,
+                      status_string, version, workspace_bytes)
+from .stack import GsitStack
+
+__all__ = [n for n in dir() if not n.startswith("_")]

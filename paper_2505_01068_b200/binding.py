@@ -1,0 +1,182 @@
+"""ctypes binding of libgsit.so: argument marshalling only.
+
+Every step of the hot path runs in the CUDA kernels of the library; PyTorch is used here for device
+memory (output and workspace allocation) and for the current stream.  There is no CPU fallback: if the
+library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+import torch
+
+PHASE_INTER_FWD, PHASE_INTER_BWD, PHASE_INTRA, PHASE_CUSTOM = 0, 1, 2, 3
+DTYPE_F32, DTYPE_BF16 = 0, 1
+CALL_QKV_PROJ, CALL_ATTENTION, CALL_LAYER = 0, 1, 2
+DEVFLAG_CLAMPED, DEVFLAG_TIMEOUT = 1, 2
+
+_LIB_PATH = Path(__file__).resolve().parent / "libgsit.so"
+_lib = None
+
+
+class GsitError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: gsit status {code} ({status_string(code)})")
+        self.code = code
+
+
+class Shape(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("seg_len", ctypes.c_int32 * 3), ("d_model", ctypes.c_int32),
+                ("heads", ctypes.c_int32), ("valid_len", ctypes.c_void_p), ("dtype", ctypes.c_int32),
+                ("phase", ctypes.c_int32), ("custom_mask", ctypes.c_uint32), ("scale", ctypes.c_float)]
+
+
+class LayerWeights(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in
+                ("ln1_gamma", "ln1_beta", "w_qkv", "b_qkv", "w_o", "b_o", "ln2_gamma", "ln2_beta",
+                 "w_1", "b_1", "w_2", "b_2")] + [("d_ff", ctypes.c_int32), ("ln_eps", ctypes.c_float)]
+
+
+EXPORTS = ("gsit_im_qkv_proj", "gsit_im_attention_fwd", "gsit_im_layer_fwd", "gsit_workspace_bytes",
+           "gsit_last_device_status", "gsit_status_string", "gsit_version")
+
+
+def load():
+    """Loads libgsit.so (built in-tree by paper_2505_01068_b200.build); fails loudly when it is absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not _LIB_PATH.exists():
+        raise FileNotFoundError(f"{_LIB_PATH} is missing: run `python -m paper_2505_01068_b200.build` "
+                                "(there is no fallback path)")
+    lib = ctypes.CDLL(str(_LIB_PATH))
+    vp, i64, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_size_t
+    sp = ctypes.POINTER(Shape)
+    lib.gsit_im_qkv_proj.argtypes = [sp, vp, i64, vp, vp, vp, vp]
+    lib.gsit_im_qkv_proj.restype = ctypes.c_int
+    lib.gsit_im_attention_fwd.argtypes = [sp, vp, vp, vp, i64, vp, vp, vp, sz, vp]
+    lib.gsit_im_attention_fwd.restype = ctypes.c_int
+    lib.gsit_im_layer_fwd.argtypes = [sp, ctypes.POINTER(LayerWeights), vp, i64, vp, i64, vp, sz, vp]
+    lib.gsit_im_layer_fwd.restype = ctypes.c_int
+    lib.gsit_workspace_bytes.argtypes = [sp, ctypes.c_int, ctypes.c_int32]
+    lib.gsit_workspace_bytes.restype = sz
+    lib.gsit_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
+    lib.gsit_last_device_status.restype = ctypes.c_int
+    lib.gsit_status_string.argtypes = [ctypes.c_int]
+    lib.gsit_status_string.restype = ctypes.c_char_p
+    lib.gsit_version.restype = ctypes.c_int
+    _lib = lib
+    return lib
+
+
+def status_string(code: int) -> str:
+    return load().gsit_status_string(int(code)).decode()
+
+
+def version() -> int:
+    return int(load().gsit_version())
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr(t) -> int | None:
+    return None if t is None else t.data_ptr()
+
+
+def _dtype_code(t: torch.dtype) -> int:
+    if t == torch.float32:
+        return DTYPE_F32
+    if t == torch.bfloat16:
+        return DTYPE_BF16
+    raise TypeError(f"unsupported dtype {t}")
+
+
+def make_shape(batch, seg_len, d_model, heads, valid_len, dtype_code, phase, custom_mask=0, scale=0.0) -> Shape:
+    if valid_len is not None:
+        assert valid_len.is_cuda and valid_len.dtype == torch.int32 and valid_len.is_contiguous()
+        assert tuple(valid_len.shape) == (batch, 3)
+    return Shape(int(batch), (ctypes.c_int32 * 3)(*[int(s) for s in seg_len]), int(d_model), int(heads),
+                 _ptr(valid_len), int(dtype_code), int(phase), int(custom_mask), float(scale))
+
+
+def _check(code: int, what: str):
+    if code != 0:
+        raise GsitError(code, what)
+
+
+def workspace_bytes(shape: Shape, which_call: int, d_ff: int = 0) -> int:
+    n = load().gsit_workspace_bytes(ctypes.byref(shape), int(which_call), int(d_ff))
+    if n == ctypes.c_size_t(-1).value:
+        raise GsitError(1, "gsit_workspace_bytes")
+    return int(n)
+
+
+def last_device_status() -> tuple[int, int]:
+    """Synchronises the current stream; returns (status code, flags) and clears the device flags."""
+    flags = ctypes.c_uint32(0)
+    code = load().gsit_last_device_status(_stream(), ctypes.byref(flags))
+    return int(code), int(flags.value)
+
+
+def im_qkv_proj(x, w_qkv, b_qkv, seg_len, heads, valid_len=None, out=None):
+    """x [B, L, d] (last dim contiguous) -> qkv [B, L, 3, H, hd]."""
+    B, L, d = x.shape
+    assert x.is_cuda and x.stride(2) == 1 and x.stride(0) == L * x.stride(1) and w_qkv.is_contiguous()
+    shape = make_shape(B, seg_len, d, heads, valid_len, _dtype_code(x.dtype), PHASE_INTRA)
+    if out is None:
+        out = torch.empty((B, L, 3, heads, d // heads), dtype=x.dtype, device=x.device)
+    _check(load().gsit_im_qkv_proj(ctypes.byref(shape), _ptr(x), x.stride(1), _ptr(w_qkv), _ptr(b_qkv), _ptr(out),
+                                   _stream()), "gsit_im_qkv_proj")
+    return out
+
+
+def im_attention_fwd(q, k, v, seg_len, valid_len=None, phase=PHASE_INTER_FWD, custom_mask=0, scale=0.0,
+                     want_lse=False, out=None):
+    """q, k, v: [B, L, H, hd] views sharing strides (e.g. qkv[:, :, i] of the fused buffer).  Returns out [B, L, d]
+    (and lse [B, H, L] float when want_lse)."""
+    B, L, H, hd = q.shape
+    d = H * hd
+    for t in (q, k, v):
+        assert t.is_cuda and t.shape == q.shape and t.stride() == q.stride() and t.dtype == q.dtype
+    assert q.stride(3) == 1 and q.stride(2) == hd and q.stride(0) == L * q.stride(1)
+    shape = make_shape(B, seg_len, d, H, valid_len, _dtype_code(q.dtype), phase, custom_mask, scale)
+    if out is None:
+        out = torch.empty((B, L, d), dtype=q.dtype, device=q.device)
+    lse = torch.empty((B, H, L), dtype=torch.float32, device=q.device) if want_lse else None
+    _check(load().gsit_im_attention_fwd(ctypes.byref(shape), _ptr(q), _ptr(k), _ptr(v), q.stride(1), _ptr(out),
+                                        _ptr(lse), None, 0, _stream()), "gsit_im_attention_fwd")
+    return (out, lse) if want_lse else out
+
+
+_W_KEYS = ("ln1_g", "ln1_b", "w_qkv", "b_qkv", "w_o", "b_o", "ln2_g", "ln2_b", "w_1", "b_1", "w_2", "b_2")
+
+
+def make_layer_weights(w: dict, ln_eps: float = 1e-5) -> LayerWeights:
+    """w maps ln1_g, ln1_b, w_qkv, b_qkv, w_o, b_o, ln2_g, ln2_b, w_1, b_1, w_2, b_2 to device tensors or None."""
+    for kk in ("w_qkv", "w_o", "w_1", "w_2"):
+        assert w[kk].is_cuda and w[kk].is_contiguous()
+    for kk in ("ln1_g", "ln1_b", "b_qkv", "b_o", "ln2_g", "ln2_b", "b_1", "b_2"):
+        assert w.get(kk) is None or (w[kk].dtype == torch.float32 and w[kk].is_contiguous())
+    return LayerWeights(*[_ptr(w.get(kk)) for kk in _W_KEYS], int(w["w_1"].shape[0]), float(ln_eps))
+
+
+def im_layer_fwd(x, weights: dict, seg_len, heads, valid_len=None, phase=PHASE_INTER_FWD, custom_mask=0, scale=0.0,
+                 ln_eps=1e-5, out=None, workspace=None):
+    """x float32 [B, L, d] (row stride free) -> y float32 [B, L, d]; weights in bf16 or float32 select the path."""
+    B, L, d = x.shape
+    assert x.is_cuda and x.dtype == torch.float32 and x.stride(2) == 1 and x.stride(0) == L * x.stride(1)
+    code = _dtype_code(weights["w_qkv"].dtype)
+    shape = make_shape(B, seg_len, d, heads, valid_len, code, phase, custom_mask, scale)
+    lw = make_layer_weights(weights, ln_eps)
+    if out is None:
+        out = torch.empty((B, L, d), dtype=torch.float32, device=x.device)
+    assert out.stride(2) == 1 and out.stride(0) == L * out.stride(1)
+    need = workspace_bytes(shape, CALL_LAYER, lw.d_ff)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=x.device)
+    _check(load().gsit_im_layer_fwd(ctypes.byref(shape), ctypes.byref(lw), _ptr(x), x.stride(1), _ptr(out),
+                                    out.stride(1), _ptr(workspace), workspace.numel(), _stream()), "gsit_im_layer_fwd")
+    return out

@@ -1,0 +1,321 @@
+// Kernel body of the bf16 IM attention (included by attn_bf16.cu only).
+#pragma once
+
+namespace gsit {
+namespace {
+
+template <int HD, int CW>
+__global__ void __launch_bounds__(NTHREADS, 2)
+attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                 const __grid_constant__ CUtensorMap tmV, const Geometry g, __nv_bfloat16* __restrict__ out,
+                 float* __restrict__ lse, const float sl2 /* scale * log2(e) */) {
+  using C = Cfg<HD, CW>;
+  constexpr int G = C::G, R = C::R, QT = C::QT, PITCH = C::PITCH, SWZ = C::SWZ, KSTEP = C::KSTEP, NT = C::NT,
+                KSQ = C::KSQ, NTO = C::NTO, CPR = CW / 8 /* 16-byte chunks per tile row */;
+  constexpr bool HOIST = (R > 1);  // several query slabs per warp reuse the K/V fragments of a step
+
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t sQ = (raw + 1023u) & ~1023u;
+  const uint32_t sK = sQ + C::Q_BYTES;
+  const uint32_t sV = sK + STAGES * C::KV_BYTES;
+  const uint32_t bar_full = sV + STAGES * C::KV_BYTES;  // STAGES barriers, 8 bytes each
+  const uint32_t bar_q = bar_full + 8 * STAGES;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int head_in_slice = warp % G, sg = warp / G;
+  const int cb = head_in_slice * (HD / 8);  // first 16-byte chunk of this warp's head inside a tile row
+
+  // ---- which tile of which block row ----
+  int tile = blockIdx.x, s = 0;
+#pragma unroll
+  for (int ss = 0; ss < 2; ++ss) {
+    const int nts = (g.seg_len[s] + QT - 1) / QT;
+    if (tile >= nts) { tile -= nts; ++s; }
+  }
+  const int q0 = tile * QT;
+  const int rows_in_tile = min(QT, g.seg_len[s] - q0);
+  const int b = blockIdx.z, cs = blockIdx.y;
+  const int q_real_all = max(0, min(rows_in_tile, valid_rows(g, b, s) - q0));
+  const int kn0 = ((g.allowed >> (3 * s + 0)) & 1u) ? valid_rows(g, b, 0) : 0;
+  const int kn1 = ((g.allowed >> (3 * s + 1)) & 1u) ? valid_rows(g, b, 1) : 0;
+  const int kn2 = ((g.allowed >> (3 * s + 2)) & 1u) ? valid_rows(g, b, 2) : 0;
+  const int nk0 = (kn0 + KT - 1) / KT, nk1 = (kn1 + KT - 1) / KT, nk2 = (kn2 + KT - 1) / KT;
+  const int T = (q_real_all > 0) ? nk0 + nk1 + nk2 : 0;  // key tiles this CTA walks
+  const int q_real = (T > 0) ? q_real_all : 0;           // rows that receive a computed result
+  const int64_t grow0 = (int64_t)b * g.L + g.seg_off[s] + q0;  // first global row of the tile
+  const int xcol = cs * CW;
+
+  auto locate = [&](int i, int& r, int& krem, int& yrow) {
+    int t = i;
+    r = 0;
+    if (t >= nk0) { t -= nk0; r = 1; if (t >= nk1) { t -= nk1; r = 2; } }
+    const int kn = (r == 0) ? kn0 : (r == 1) ? kn1 : kn2;
+    krem = kn - t * KT;
+    yrow = b * g.L + g.seg_off[r] + t * KT;
+  };
+  auto issue = [&](int i) {  // one thread: TMA loads of key tile i into its stage
+    int r, krem, yrow;
+    locate(i, r, krem, yrow);
+    const int st = i % STAGES;
+    mbar_expect_tx(bar_full + 8 * st, 2 * C::KV_BYTES);
+    tma_load_2d(sK + st * C::KV_BYTES, &tmK, xcol, yrow, bar_full + 8 * st);
+    tma_load_2d(sV + st * C::KV_BYTES, &tmV, xcol, yrow, bar_full + 8 * st);
+  };
+
+  float O[R][NTO][4];
+  float m[R][2], l[R][2];
+#pragma unroll
+  for (int r_ = 0; r_ < R; ++r_) {
+    m[r_][0] = m[r_][1] = -INFINITY;
+    l[r_][0] = l[r_][1] = 0.f;
+#pragma unroll
+    for (int n = 0; n < NTO; ++n) O[r_][n][0] = O[r_][n][1] = O[r_][n][2] = O[r_][n][3] = 0.f;
+  }
+
+  if (T > 0) {
+    if (tid == 0) {
+#pragma unroll
+      for (int st = 0; st < STAGES; ++st) mbar_init(bar_full + 8 * st, 1);
+      mbar_init(bar_q, 1);
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+    if (tid == 0) {
+      mbar_expect_tx(bar_q, C::Q_BYTES);
+      tma_load_2d(sQ, &tmQ, xcol, (int)grow0, bar_q);
+      for (int i = 0; i < STAGES - 1 && i < T; ++i) issue(i);
+    }
+
+    // ---- query fragments, kept in registers for the whole key walk ----
+    uint32_t QF[R][KSQ][4];
+    mbar_wait(g, bar_q, 0);
+#pragma unroll
+    for (int r_ = 0; r_ < R; ++r_) {
+      const int row0 = (sg * R + r_) * 16;
+      if constexpr (HD == 8) {
+        const int row = row0 + (lane & 15);
+        ldsm_x2(sQ + swz<SWZ>(row * PITCH + cb * 16), QF[r_][0][0], QF[r_][0][1]);
+        QF[r_][0][2] = QF[r_][0][3] = 0;
+      } else {
+        const int mi = lane >> 3;
+        const int row = row0 + (mi & 1) * 8 + (lane & 7);
+#pragma unroll
+        for (int ks = 0; ks < KSQ; ++ks)
+          ldsm_x4(sQ + swz<SWZ>(row * PITCH + (cb + ks * 2 + (mi >> 1)) * 16), QF[r_][ks][0], QF[r_][ks][1],
+                  QF[r_][ks][2], QF[r_][ks][3]);
+      }
+    }
+
+    for (int i = 0; i < T; ++i) {
+      const int st = i % STAGES;
+      if (tid == 0 && i + STAGES - 1 < T) issue(i + STAGES - 1);
+      mbar_wait(g, bar_full + 8 * st, (i / STAGES) & 1);
+      int r, krem, yrow;
+      locate(i, r, krem, yrow);
+      const uint32_t sKs = sK + st * C::KV_BYTES, sVs = sV + st * C::KV_BYTES;
+      if (krem < KT) {
+        // Rows past the valid length hold whatever follows in memory: clear them in V so that a zero weight
+        // times a NaN/Inf value cannot poison the accumulator (their scores are replaced by -inf below).
+        for (int idx = tid; idx < (KT - krem) * CPR; idx += NTHREADS) {
+          const uint32_t a = sVs + (krem + idx / CPR) * PITCH + (idx % CPR) * 16;
+          asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0) : "memory");
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncthreads();
+      }
+
+#pragma unroll
+      for (int stp = 0; stp < KT / KSTEP; ++stp) {
+        const int kb = stp * KSTEP;
+        if (kb >= krem) break;
+        const bool ragged = (krem - kb) < KSTEP;
+        uint32_t KF[NT][KSQ][2];
+        uint32_t VF[KSTEP / 16][NTO][2];
+
+        auto load_k_pair = [&](int p) {  // K fragments of score n-tiles 2p, 2p+1 (HD >= 16)
+          const int mi = lane >> 3;
+          const int key = kb + p * 16 + (mi >> 1) * 8 + (lane & 7);
+#pragma unroll
+          for (int ks = 0; ks < KSQ; ++ks)
+            ldsm_x4(sKs + swz<SWZ>(key * PITCH + (cb + ks * 2 + (mi & 1)) * 16), KF[2 * p][ks][0], KF[2 * p][ks][1],
+                    KF[2 * p + 1][ks][0], KF[2 * p + 1][ks][1]);
+        };
+        auto load_v_pair = [&](int kk, int np) {  // V fragments of key step kk, output n-tiles 2np, 2np+1 (HD >= 16)
+          const int mi = lane >> 3;
+          const int key = kb + kk * 16 + (mi & 1) * 8 + (lane & 7);
+          ldsm_x4_t(sVs + swz<SWZ>(key * PITCH + (cb + np * 2 + (mi >> 1)) * 16), VF[kk][2 * np][0], VF[kk][2 * np][1],
+                    VF[kk][2 * np + 1][0], VF[kk][2 * np + 1][1]);
+        };
+        auto load_k8 = [&](int j) {  // HD == 8: K fragments of n-tiles 4j .. 4j+3 (32 keys)
+          ldsm_x4(sKs + swz<SWZ>((kb + j * 32 + lane) * PITCH + cb * 16), KF[4 * j][0][0], KF[4 * j + 1][0][0],
+                  KF[4 * j + 2][0][0], KF[4 * j + 3][0][0]);
+        };
+        auto load_v8 = [&](int j) {  // HD == 8: V fragments of key steps 2j, 2j+1 (32 keys)
+          ldsm_x4_t(sVs + swz<SWZ>((kb + j * 32 + lane) * PITCH + cb * 16), VF[2 * j][0][0], VF[2 * j][0][1],
+                    VF[2 * j + 1][0][0], VF[2 * j + 1][0][1]);
+        };
+
+        if constexpr (HOIST) {
+          if constexpr (HD == 8) {
+#pragma unroll
+            for (int j = 0; j < KSTEP / 32; ++j) { load_k8(j); load_v8(j); }
+          } else {
+#pragma unroll
+            for (int p = 0; p < NT / 2; ++p) load_k_pair(p);
+#pragma unroll
+            for (int kk = 0; kk < KSTEP / 16; ++kk)
+#pragma unroll
+              for (int np = 0; np < NTO / 2; ++np) load_v_pair(kk, np);
+          }
+        }
+
+#pragma unroll
+        for (int r_ = 0; r_ < R; ++r_) {
+          const int row0 = (sg * R + r_) * 16;
+          if (row0 >= q_real) continue;  // slab of padding rows only
+          float S[NT][4];
+#pragma unroll
+          for (int n = 0; n < NT; ++n) S[n][0] = S[n][1] = S[n][2] = S[n][3] = 0.f;
+
+          // ---- S = Q K^T (raw dot products) ----
+          if constexpr (HD == 8) {
+#pragma unroll
+            for (int j = 0; j < KSTEP / 32; ++j) {
+              if constexpr (!HOIST) load_k8(j);
+#pragma unroll
+              for (int n = 4 * j; n < 4 * j + 4; ++n) mma_k8(S[n], QF[r_][0][0], QF[r_][0][1], KF[n][0][0]);
+            }
+          } else {
+#pragma unroll
+            for (int p = 0; p < NT / 2; ++p) {
+              if constexpr (!HOIST) load_k_pair(p);
+#pragma unroll
+              for (int ks = 0; ks < KSQ; ++ks) {
+                mma_k16(S[2 * p], QF[r_][ks][0], QF[r_][ks][1], QF[r_][ks][2], QF[r_][ks][3], KF[2 * p][ks][0],
+                        KF[2 * p][ks][1]);
+                mma_k16(S[2 * p + 1], QF[r_][ks][0], QF[r_][ks][1], QF[r_][ks][2], QF[r_][ks][3], KF[2 * p + 1][ks][0],
+                        KF[2 * p + 1][ks][1]);
+              }
+            }
+          }
+          // ---- keys past the valid length get weight exactly zero ----
+          if (ragged) {
+            const int c0 = kb + (lane & 3) * 2;
+#pragma unroll
+            for (int n = 0; n < NT; ++n) {
+              if (c0 + n * 8 >= krem) S[n][0] = S[n][2] = -INFINITY;
+              if (c0 + n * 8 + 1 >= krem) S[n][1] = S[n][3] = -INFINITY;
+            }
+          }
+          // ---- online softmax (base 2, scale folded into sl2) ----
+          float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+          for (int n = 0; n < NT; ++n) {
+            mx0 = fmaxf(mx0, fmaxf(S[n][0], S[n][1]));
+            mx1 = fmaxf(mx1, fmaxf(S[n][2], S[n][3]));
+          }
+          mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+          mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+          mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+          mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+          const float mn0 = fmaxf(m[r_][0], mx0), mn1 = fmaxf(m[r_][1], mx1);
+          const float ms0 = (mn0 == -INFINITY) ? 0.f : mn0 * sl2;
+          const float ms1 = (mn1 == -INFINITY) ? 0.f : mn1 * sl2;
+          const float al0 = ex2(fmaf(m[r_][0], sl2, -ms0)), al1 = ex2(fmaf(m[r_][1], sl2, -ms1));
+          m[r_][0] = mn0;
+          m[r_][1] = mn1;
+          float rs0 = 0.f, rs1 = 0.f;
+#pragma unroll
+          for (int n = 0; n < NT; ++n) {
+            S[n][0] = ex2(fmaf(S[n][0], sl2, -ms0));
+            S[n][1] = ex2(fmaf(S[n][1], sl2, -ms0));
+            S[n][2] = ex2(fmaf(S[n][2], sl2, -ms1));
+            S[n][3] = ex2(fmaf(S[n][3], sl2, -ms1));
+            rs0 += S[n][0] + S[n][1];
+            rs1 += S[n][2] + S[n][3];
+          }
+          l[r_][0] = fmaf(l[r_][0], al0, rs0);
+          l[r_][1] = fmaf(l[r_][1], al1, rs1);
+#pragma unroll
+          for (int n = 0; n < NTO; ++n) {
+            O[r_][n][0] *= al0; O[r_][n][1] *= al0;
+            O[r_][n][2] *= al1; O[r_][n][3] *= al1;
+          }
+          // ---- O += P V, the score registers repacked as the A operand ----
+#pragma unroll
+          for (int kk = 0; kk < KSTEP / 16; ++kk) {
+            const uint32_t a0 = pack_bf16(S[2 * kk][0], S[2 * kk][1]);
+            const uint32_t a1 = pack_bf16(S[2 * kk][2], S[2 * kk][3]);
+            const uint32_t a2 = pack_bf16(S[2 * kk + 1][0], S[2 * kk + 1][1]);
+            const uint32_t a3 = pack_bf16(S[2 * kk + 1][2], S[2 * kk + 1][3]);
+            if constexpr (HD == 8) {
+              if constexpr (!HOIST) { if ((kk & 1) == 0) load_v8(kk / 2); }
+              mma_k16(O[r_][0], a0, a1, a2, a3, VF[kk][0][0], VF[kk][0][1]);
+            } else {
+#pragma unroll
+              for (int np = 0; np < NTO / 2; ++np) {
+                if constexpr (!HOIST) load_v_pair(kk, np);
+                mma_k16(O[r_][2 * np], a0, a1, a2, a3, VF[kk][2 * np][0], VF[kk][2 * np][1]);
+                mma_k16(O[r_][2 * np + 1], a0, a1, a2, a3, VF[kk][2 * np + 1][0], VF[kk][2 * np + 1][1]);
+              }
+            }
+          }
+        }  // slabs
+      }    // steps
+      __syncthreads();  // every warp is done with this stage before it is refilled
+    }      // key tiles
+
+    // ---- normalise and stage the tile in shared memory (the Q region is free now) ----
+#pragma unroll
+    for (int r_ = 0; r_ < R; ++r_) {
+      const int row0 = (sg * R + r_) * 16;
+      if (row0 >= q_real) continue;
+      float l0 = l[r_][0], l1 = l[r_][1];
+      l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
+      l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
+      l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+      l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+      const float inv0 = l0 > 0.f ? 1.f / l0 : 0.f, inv1 = l1 > 0.f ? 1.f / l1 : 0.f;
+      const int rowA = row0 + (lane >> 2), rowB = rowA + 8;
+#pragma unroll
+      for (int n = 0; n < NTO; ++n) {
+        const int colb = (head_in_slice * HD + n * 8 + (lane & 3) * 2) * 2;  // byte column in the tile row
+        const uint32_t vA = pack_bf16(O[r_][n][0] * inv0, O[r_][n][1] * inv0);
+        const uint32_t vB = pack_bf16(O[r_][n][2] * inv1, O[r_][n][3] * inv1);
+        asm volatile("st.shared.b32 [%0], %1;" ::"r"(sQ + swz<SWZ>(rowA * PITCH + colb)), "r"(vA) : "memory");
+        asm volatile("st.shared.b32 [%0], %1;" ::"r"(sQ + swz<SWZ>(rowB * PITCH + colb)), "r"(vB) : "memory");
+      }
+      if (lse != nullptr && (lane & 3) == 0) {
+        const int head = cs * G + head_in_slice;
+        float* lp = lse + ((int64_t)b * g.heads + head) * g.L + g.seg_off[s] + q0;
+        const float ln2 = 0.6931471805599453f;
+        if (rowA < q_real) lp[rowA] = l0 > 0.f ? (m[r_][0] * sl2 + log2f(l0)) * ln2 : -INFINITY;
+        if (rowB < q_real) lp[rowB] = l1 > 0.f ? (m[r_][1] * sl2 + log2f(l1)) * ln2 : -INFINITY;
+      }
+    }
+    __syncthreads();
+  }  // T > 0
+
+  // ---- coalesced 16-byte stores; padded rows are written as +0, rows of the next segment are left alone ----
+  for (int idx = tid; idx < rows_in_tile * CPR; idx += NTHREADS) {
+    const int row = idx / CPR, ch = idx % CPR;
+    uint32_t v0 = 0, v1 = 0, v2 = 0, v3 = 0;
+    if (row < q_real)
+      asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];"
+                   : "=r"(v0), "=r"(v1), "=r"(v2), "=r"(v3) : "r"(sQ + swz<SWZ>(row * PITCH + ch * 16)) : "memory");
+    uint4* dst = reinterpret_cast<uint4*>(out + (grow0 + row) * g.d + xcol + ch * 8);
+    *dst = make_uint4(v0, v1, v2, v3);
+  }
+  if (lse != nullptr) {
+    const int npad = rows_in_tile - q_real;
+    for (int idx = tid; idx < npad * G; idx += NTHREADS) {
+      const int row = q_real + idx / G, head = cs * G + idx % G;
+      lse[((int64_t)b * g.heads + head) * g.L + g.seg_off[s] + q0 + row] = -INFINITY;
+    }
+  }
+}
+
+}  // namespace
+}  // namespace gsit

@@ -1,0 +1,81 @@
+// Shared device/host helpers of the IM attention library (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "gsit.h"
+
+namespace gsit {
+
+// Problem geometry handed to every kernel by value.
+struct Geometry {
+  int batch, L, d, heads, hd;
+  int seg_len[3];
+  int seg_off[3];
+  uint32_t allowed;          // bit (3*s + r): query segment s may attend key segment r
+  const int32_t* valid_len;  // device [B][3] or nullptr
+  unsigned int* status;      // device status word (GSIT_DEVFLAG_* bits), one per device
+};
+
+__device__ __forceinline__ void raise_flag(const Geometry& g, unsigned int f) { atomicOr(g.status, f); }
+
+// Real-row count of segment s in sample b, clamped to [0, seg_len[s]].
+__device__ __forceinline__ int valid_rows(const Geometry& g, int b, int s) {
+  if (g.valid_len == nullptr) return g.seg_len[s];
+  int n = g.valid_len[3 * b + s];
+  if (n < 0 || n > g.seg_len[s]) {
+    raise_flag(g, GSIT_DEVFLAG_CLAMPED);
+    n = n < 0 ? 0 : g.seg_len[s];
+  }
+  return n;
+}
+
+__device__ __forceinline__ int segment_of(const Geometry& g, int p) {
+  return (p >= g.seg_off[2]) ? 2 : (p >= g.seg_off[1]) ? 1 : 0;
+}
+
+// True iff row `row` of the flattened [B*L] sequence is a real (non padded) position.
+__device__ __forceinline__ bool row_is_real(const Geometry& g, int64_t row) {
+  const int b = (int)(row / g.L);
+  const int p = (int)(row - (int64_t)b * g.L);
+  const int s = segment_of(g, p);
+  return (p - g.seg_off[s]) < valid_rows(g, b, s);
+}
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+
+// ---- host-side launch entry points of the kernel files (all asynchronous on `st`) ----
+// Each returns cudaSuccess or the launch error.
+
+// fp32 attention on CUDA cores (attn_f32.cu)
+cudaError_t launch_attn_f32(const Geometry& g, const float* q, const float* k, const float* v, int64_t row_stride,
+                            float* out, float* lse, float scale, cudaStream_t st);
+// bf16 attention, mma.sync tiles fed by TMA (attn_bf16.cu); returns cudaErrorNotSupported for shapes it lacks
+cudaError_t launch_attn_bf16(const Geometry& g, const __nv_bfloat16* q, const __nv_bfloat16* k,
+                             const __nv_bfloat16* v, int64_t row_stride, __nv_bfloat16* out, float* lse,
+                             float scale, cudaStream_t st);
+
+// Linear layers  C = act(A W^T + bias) (+ residual), rows that are padding written as zero when
+// `mask_rows` is set.  A [M,K] (lda), W [N,K], C [M,N] (ldc), residual float [M,N] (ldr) or nullptr.
+struct LinearArgs {
+  const void* A; int64_t lda;
+  const void* W;
+  const float* bias;
+  const float* residual; int64_t ldr;
+  void* C; int64_t ldc;
+  int M, N, K;
+  int relu;
+  int out_f32;      // bf16 path only: write float instead of bf16
+  int mask_rows;    // zero the padded rows of C (uses geometry)
+};
+cudaError_t launch_linear_f32(const Geometry& g, const LinearArgs& a, cudaStream_t st);
+cudaError_t launch_linear_bf16(const Geometry& g, const LinearArgs& a, cudaStream_t st);
+
+// Row LayerNorm of float x (row stride ldx) into float or bf16 y [rows, d]; padded rows become zero.
+cudaError_t launch_layernorm(const Geometry& g, const float* x, int64_t ldx, const float* gamma, const float* beta,
+                             float eps, void* y, int out_bf16, cudaStream_t st);
+
+}  // namespace gsit

@@ -1,0 +1,259 @@
+// C ABI of the IM attention library: argument validation, workspace carving, kernel sequencing.
+#include <math.h>
+
+#include "common.cuh"
+
+namespace gsit {
+
+__device__ unsigned int g_device_status_word = 0;
+
+namespace {
+
+constexpr int MAX_DEVICES = 64;
+unsigned int* g_status_ptr[MAX_DEVICES] = {};
+
+// Address of this device's status word (looked up once per device).
+cudaError_t status_ptr(unsigned int** p) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= MAX_DEVICES) return cudaErrorInvalidDevice;
+  if (g_status_ptr[dev] == nullptr) {
+    void* sym = nullptr;
+    e = cudaGetSymbolAddress(&sym, g_device_status_word);
+    if (e != cudaSuccess) return e;
+    g_status_ptr[dev] = static_cast<unsigned int*>(sym);
+  }
+  *p = g_status_ptr[dev];
+  return cudaSuccess;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+gsit_status allowed_bits(const gsit_shape* s, uint32_t* bits) {
+  switch (s->phase) {
+    case GSIT_PHASE_INTER_FWD: *bits = (1u << 1) | (1u << 5) | (1u << 6); return GSIT_OK;  // 0->1, 1->2, 2->0
+    case GSIT_PHASE_INTER_BWD: *bits = (1u << 2) | (1u << 3) | (1u << 7); return GSIT_OK;  // 0->2, 1->0, 2->1
+    case GSIT_PHASE_INTRA:     *bits = (1u << 0) | (1u << 4) | (1u << 8); return GSIT_OK;  // s->s
+    case GSIT_PHASE_CUSTOM:
+      if (s->custom_mask > 0x1FFu) return GSIT_ERR_INVALID_ARG;
+      *bits = s->custom_mask;
+      return GSIT_OK;
+    default: return GSIT_ERR_INVALID_ARG;
+  }
+}
+
+// Validates the shape and fills the kernel-side geometry (without the status pointer).
+gsit_status make_geometry(const gsit_shape* s, Geometry* g) {
+  if (s == nullptr) return GSIT_ERR_INVALID_ARG;
+  if (s->batch < 1 || s->heads < 1 || s->d_model < 1 || s->d_model % s->heads != 0) return GSIT_ERR_INVALID_ARG;
+  if (s->dtype != GSIT_F32 && s->dtype != GSIT_BF16) return GSIT_ERR_INVALID_ARG;
+  int64_t L = 0;
+  for (int i = 0; i < 3; ++i) {
+    if (s->seg_len[i] < 0) return GSIT_ERR_INVALID_ARG;
+    L += s->seg_len[i];
+  }
+  if (L < 1) return GSIT_ERR_INVALID_ARG;
+  if (L * (int64_t)s->batch > 0x7fffffffLL / 4) return GSIT_ERR_UNSUPPORTED;
+  uint32_t bits = 0;
+  gsit_status st = allowed_bits(s, &bits);
+  if (st != GSIT_OK) return st;
+  g->batch = s->batch;
+  g->L = (int)L;
+  g->d = s->d_model;
+  g->heads = s->heads;
+  g->hd = s->d_model / s->heads;
+  for (int i = 0; i < 3; ++i) g->seg_len[i] = s->seg_len[i];
+  g->seg_off[0] = 0;
+  g->seg_off[1] = s->seg_len[0];
+  g->seg_off[2] = s->seg_len[0] + s->seg_len[1];
+  g->allowed = bits;
+  g->valid_len = s->valid_len;
+  g->status = nullptr;
+  if (s->dtype == GSIT_BF16) {
+    if (g->d % 16 != 0) return GSIT_ERR_UNSUPPORTED;
+    if (g->hd != 8 && g->hd != 16 && g->hd != 32 && g->hd != 64) return GSIT_ERR_UNSUPPORTED;
+    const int cw = (g->d % 64 == 0) ? 64 : (g->d % 32 == 0) ? 32 : 16;
+    if (g->hd > cw || g->batch > 65535) return GSIT_ERR_UNSUPPORTED;
+  } else {
+    if (g->hd > 256) return GSIT_ERR_UNSUPPORTED;
+  }
+  return GSIT_OK;
+}
+
+gsit_status from_cuda(cudaError_t e) {
+  if (e == cudaSuccess) return GSIT_OK;
+  return (e == cudaErrorNotSupported) ? GSIT_ERR_UNSUPPORTED : GSIT_ERR_CUDA;
+}
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Scratch layout of one layer call; every region 256-byte aligned.
+struct LayerScratch {
+  size_t h, qkv, att, y1, f, total;
+};
+LayerScratch layer_scratch(const Geometry& g, int dtype, int d_ff) {
+  const size_t rows = (size_t)g.batch * g.L, es = (dtype == GSIT_BF16) ? 2 : 4;
+  LayerScratch s;
+  size_t off = 0;
+  s.h = off;   off += align_up(rows * g.d * es, 256);       // LN1(x), later LN2(y1)
+  s.qkv = off; off += align_up(rows * 3 * g.d * es, 256);
+  s.att = off; off += align_up(rows * g.d * es, 256);
+  s.y1 = off;  off += align_up(rows * g.d * 4, 256);        // float residual stream after attention
+  s.f = off;   off += align_up(rows * (size_t)d_ff * es, 256);
+  s.total = off;
+  return s;
+}
+
+gsit_status run_linear(const Geometry& g, int dtype, const LinearArgs& a, cudaStream_t st) {
+  return from_cuda(dtype == GSIT_BF16 ? launch_linear_bf16(g, a, st) : launch_linear_f32(g, a, st));
+}
+
+gsit_status run_attention(const Geometry& g, int dtype, const void* q, const void* k, const void* v,
+                          int64_t row_stride, void* out, float* lse, float scale, cudaStream_t st) {
+  if (dtype == GSIT_BF16)
+    return from_cuda(launch_attn_bf16(g, static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k),
+                                      static_cast<const __nv_bfloat16*>(v), row_stride,
+                                      static_cast<__nv_bfloat16*>(out), lse, scale, st));
+  return from_cuda(launch_attn_f32(g, static_cast<const float*>(q), static_cast<const float*>(k),
+                                   static_cast<const float*>(v), row_stride, static_cast<float*>(out), lse, scale, st));
+}
+
+float pick_scale(const gsit_shape* s, const Geometry& g) {
+  return (s->scale > 0.f) ? s->scale : 1.0f / sqrtf((float)g.hd);
+}
+
+}  // namespace
+}  // namespace gsit
+
+using namespace gsit;
+
+extern "C" {
+
+gsit_status gsit_im_qkv_proj(const gsit_shape* shape, const void* x, int64_t x_row_stride, const void* w_qkv,
+                             const float* b_qkv, void* qkv, gsit_stream stream) {
+  Geometry g;
+  gsit_status st = make_geometry(shape, &g);
+  if (st != GSIT_OK) return st;
+  if (!x || !w_qkv || !qkv || x_row_stride < g.d) return GSIT_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(w_qkv) || !aligned16(qkv)) return GSIT_ERR_INVALID_ARG;
+  if (shape->dtype == GSIT_BF16 && x_row_stride % 8 != 0) return GSIT_ERR_INVALID_ARG;
+  if (from_cuda(status_ptr(&g.status)) != GSIT_OK) return GSIT_ERR_CUDA;
+  LinearArgs a = {};
+  a.A = x; a.lda = x_row_stride; a.W = w_qkv; a.bias = b_qkv;
+  a.C = qkv; a.ldc = 3 * (int64_t)g.d;
+  a.M = g.batch * g.L; a.N = 3 * g.d; a.K = g.d;
+  a.mask_rows = 1;
+  return run_linear(g, shape->dtype, a, static_cast<cudaStream_t>(stream));
+}
+
+gsit_status gsit_im_attention_fwd(const gsit_shape* shape, const void* q, const void* k, const void* v,
+                                  int64_t row_stride, void* out, float* lse, void* workspace,
+                                  size_t workspace_bytes, gsit_stream stream) {
+  (void)workspace; (void)workspace_bytes;  // this call needs no scratch
+  Geometry g;
+  gsit_status st = make_geometry(shape, &g);
+  if (st != GSIT_OK) return st;
+  if (!q || !k || !v || !out || row_stride < g.d) return GSIT_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return GSIT_ERR_INVALID_ARG;
+  if (shape->dtype == GSIT_BF16 && row_stride % 8 != 0) return GSIT_ERR_INVALID_ARG;
+  if (from_cuda(status_ptr(&g.status)) != GSIT_OK) return GSIT_ERR_CUDA;
+  return run_attention(g, shape->dtype, q, k, v, row_stride, out, lse, pick_scale(shape, g),
+                       static_cast<cudaStream_t>(stream));
+}
+
+gsit_status gsit_im_layer_fwd(const gsit_shape* shape, const gsit_layer_weights* w, const float* x,
+                              int64_t x_row_stride, float* y, int64_t y_row_stride, void* workspace,
+                              size_t workspace_bytes, gsit_stream stream) {
+  Geometry g;
+  gsit_status st = make_geometry(shape, &g);
+  if (st != GSIT_OK) return st;
+  if (!w || !x || !y || x_row_stride < g.d || y_row_stride < g.d) return GSIT_ERR_INVALID_ARG;
+  if (!w->w_qkv || !w->w_o || !w->w_1 || !w->w_2 || w->d_ff < 1) return GSIT_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(y) || !aligned16(w->w_qkv) || !aligned16(w->w_o) || !aligned16(w->w_1) ||
+      !aligned16(w->w_2))
+    return GSIT_ERR_INVALID_ARG;
+  if (x_row_stride % 4 != 0 || y_row_stride % 4 != 0) return GSIT_ERR_INVALID_ARG;
+  const int dtype = shape->dtype;
+  if (dtype == GSIT_BF16 && w->d_ff % 8 != 0) return GSIT_ERR_UNSUPPORTED;
+  const LayerScratch sc = layer_scratch(g, dtype, w->d_ff);
+  if (!workspace || workspace_bytes < sc.total || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+    return GSIT_ERR_WORKSPACE;
+  if (from_cuda(status_ptr(&g.status)) != GSIT_OK) return GSIT_ERR_CUDA;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  void *h = ws + sc.h, *qkv = ws + sc.qkv, *att = ws + sc.att, *f = ws + sc.f;
+  float* y1 = reinterpret_cast<float*>(ws + sc.y1);
+  const float eps = (w->ln_eps > 0.f) ? w->ln_eps : 1e-5f;
+  const int bf = (dtype == GSIT_BF16);
+  const int es = bf ? 2 : 4;
+  const int M = g.batch * g.L, d = g.d;
+
+  // h = LN1(x)
+  if ((st = from_cuda(launch_layernorm(g, x, x_row_stride, w->ln1_gamma, w->ln1_beta, eps, h, bf, cs))) != GSIT_OK) return st;
+  // qkv = h W_qkv^T + b_qkv   (shared projection of the whole concatenated sequence)
+  LinearArgs a = {};
+  a.A = h; a.lda = d; a.W = w->w_qkv; a.bias = w->b_qkv; a.C = qkv; a.ldc = 3 * (int64_t)d;
+  a.M = M; a.N = 3 * d; a.K = d; a.mask_rows = 1;
+  if ((st = run_linear(g, dtype, a, cs)) != GSIT_OK) return st;
+  // att = IM attention over the open blocks
+  const uint8_t* qb = static_cast<const uint8_t*>(qkv);
+  if ((st = run_attention(g, dtype, qb, qb + (size_t)d * es, qb + (size_t)2 * d * es, 3 * (int64_t)d, att, nullptr,
+                          pick_scale(shape, g), cs)) != GSIT_OK) return st;
+  // y1 = x + att W_o^T + b_o   (float)
+  a = LinearArgs{};
+  a.A = att; a.lda = d; a.W = w->w_o; a.bias = w->b_o; a.residual = x; a.ldr = x_row_stride;
+  a.C = y1; a.ldc = d; a.M = M; a.N = d; a.K = d; a.out_f32 = 1; a.mask_rows = 1;
+  if ((st = run_linear(g, dtype, a, cs)) != GSIT_OK) return st;
+  // h = LN2(y1)
+  if ((st = from_cuda(launch_layernorm(g, y1, d, w->ln2_gamma, w->ln2_beta, eps, h, bf, cs))) != GSIT_OK) return st;
+  // f = relu(h W_1^T + b_1)
+  a = LinearArgs{};
+  a.A = h; a.lda = d; a.W = w->w_1; a.bias = w->b_1; a.C = f; a.ldc = w->d_ff;
+  a.M = M; a.N = w->d_ff; a.K = d; a.relu = 1; a.mask_rows = 1;
+  if ((st = run_linear(g, dtype, a, cs)) != GSIT_OK) return st;
+  // y = y1 + f W_2^T + b_2   (float), padded rows zero
+  a = LinearArgs{};
+  a.A = f; a.lda = w->d_ff; a.W = w->w_2; a.bias = w->b_2; a.residual = y1; a.ldr = d;
+  a.C = y; a.ldc = y_row_stride; a.M = M; a.N = d; a.K = w->d_ff; a.out_f32 = 1; a.mask_rows = 1;
+  return run_linear(g, dtype, a, cs);
+}
+
+size_t gsit_workspace_bytes(const gsit_shape* shape, int which_call, int32_t d_ff) {
+  Geometry g;
+  if (make_geometry(shape, &g) != GSIT_OK) return (size_t)-1;
+  if (which_call == GSIT_CALL_LAYER) {
+    if (d_ff < 1) return (size_t)-1;
+    return layer_scratch(g, shape->dtype, d_ff).total;
+  }
+  if (which_call == GSIT_CALL_QKV_PROJ || which_call == GSIT_CALL_ATTENTION) return 0;
+  return (size_t)-1;
+}
+
+gsit_status gsit_last_device_status(gsit_stream stream, uint32_t* flags) {
+  unsigned int* p = nullptr;
+  if (status_ptr(&p) != cudaSuccess) return GSIT_ERR_CUDA;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  unsigned int host = 0;
+  if (cudaMemcpyAsync(&host, p, sizeof(host), cudaMemcpyDeviceToHost, cs) != cudaSuccess) return GSIT_ERR_CUDA;
+  if (cudaMemsetAsync(p, 0, sizeof(host), cs) != cudaSuccess) return GSIT_ERR_CUDA;
+  if (cudaStreamSynchronize(cs) != cudaSuccess) return GSIT_ERR_CUDA;
+  if (flags) *flags = host;
+  return (host & GSIT_DEVFLAG_TIMEOUT) ? GSIT_ERR_TIMEOUT : GSIT_OK;
+}
+
+const char* gsit_status_string(gsit_status s) {
+  switch (s) {
+    case GSIT_OK: return "ok";
+    case GSIT_ERR_INVALID_ARG: return "invalid argument";
+    case GSIT_ERR_UNSUPPORTED: return "unsupported shape or dtype";
+    case GSIT_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case GSIT_ERR_CUDA: return "CUDA error";
+    case GSIT_ERR_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+int gsit_version(void) { return 100; }
+
+}  // extern "C"

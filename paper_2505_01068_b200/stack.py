@@ -1,0 +1,52 @@
+"""The GsiT fusion stack as a sequence of library calls (Eq. "All-Modal-In-One fusion"): a forward-ring
+encoder and a backward-ring encoder, each with its own weights, both starting from the same input; their
+outputs side by side on the feature axis (width 2d); then the intra-modal encoder on that.  Only
+sequencing and buffer reuse happen here -- each layer is one gsit_im_layer_fwd call, and the feature
+concat costs nothing because the last layer of each ring writes its half of the [B, L, 2d] buffer."""
+from __future__ import annotations
+
+import torch
+
+from . import binding as B
+
+
+class GsitStack:
+    def __init__(self, fwd_layers, bwd_layers, intra_layers, seg_len, heads, intra_heads, ln_eps=1e-5):
+        self.fwd, self.bwd, self.intra = list(fwd_layers), list(bwd_layers), list(intra_layers)
+        self.seg_len, self.heads, self.intra_heads, self.ln_eps = tuple(seg_len), heads, intra_heads, ln_eps
+        self._bufs = None
+
+    def _buffers(self, x, valid_len):
+        Bn, L, d = x.shape
+        key = (Bn, L, d, x.device)
+        if self._bufs is None or self._bufs[0] != key:
+            code = B._dtype_code(self.fwd[0]["w_qkv"].dtype)
+            sh1 = B.make_shape(Bn, self.seg_len, d, self.heads, valid_len, code, B.PHASE_INTER_FWD)
+            sh2 = B.make_shape(Bn, self.seg_len, 2 * d, self.intra_heads, valid_len, code, B.PHASE_INTRA)
+            need = B.workspace_bytes(sh1, B.CALL_LAYER, self.fwd[0]["w_1"].shape[0])
+            if self.intra:
+                need = max(need, B.workspace_bytes(sh2, B.CALL_LAYER, self.intra[0]["w_1"].shape[0]))
+            f32 = dict(dtype=torch.float32, device=x.device)
+            self._bufs = (key, torch.empty(need, dtype=torch.uint8, device=x.device),
+                          torch.empty((Bn, L, d), **f32), torch.empty((Bn, L, d), **f32),
+                          torch.empty((Bn, L, 2 * d), **f32), torch.empty((Bn, L, 2 * d), **f32))
+        return self._bufs[1:]
+
+    def forward(self, x, valid_len=None):
+        """x float32 [B, L, d] -> float32 [B, L, 2d].  The result lives in a buffer owned by this object."""
+        ws, t0, t1, c0, c1 = self._buffers(x, valid_len)
+        d = x.shape[2]
+        for layers, phase, half in ((self.fwd, B.PHASE_INTER_FWD, 0), (self.bwd, B.PHASE_INTER_BWD, 1)):
+            cur, ping = x, [t0, t1]
+            for i, w in enumerate(layers):
+                dst = c0[:, :, half * d:(half + 1) * d] if i == len(layers) - 1 else ping[i % 2]
+                B.im_layer_fwd(cur, w, self.seg_len, self.heads, valid_len, phase, ln_eps=self.ln_eps, out=dst,
+                               workspace=ws)
+                cur = dst
+        cur, ping = c0, [c1, c0]
+        for i, w in enumerate(self.intra):
+            dst = ping[i % 2]
+            B.im_layer_fwd(cur, w, self.seg_len, self.intra_heads, valid_len, B.PHASE_INTRA, ln_eps=self.ln_eps,
+                           out=dst, workspace=ws)
+            cur = dst
+        return cur

@@ -1,0 +1,188 @@
+"""GPU edge cases and properties: ragged / empty segments, every supported head width and slice width,
+custom block patterns (union softmax), separate vs fused q/k/v, explicit scale, bit-exact padding,
+run-to-run determinism, device status flags and host-side argument rejection."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads as wk
+from gpu_util import check_close, pad_mask, to_dev, to_np64
+
+pytestmark = pytest.mark.gpu
+PHASES = [oracle.PHASE_INTER_FWD, oracle.PHASE_INTER_BWD, oracle.PHASE_INTRA]
+
+
+@pytest.fixture(scope="module")
+def g():
+    import paper_2505_01068_b200 as lib
+    lib.load()
+    return lib
+
+
+def _run(g, q, k, v, seg, valid, phase, dtype, custom=0, scale=0.0, nan_pad=True):
+    B = q.shape[0]
+    pm = pad_mask(seg, valid, B)
+    qd, kd, vd = (to_dev(wk.fill_padding(a, seg, valid, np.nan) if (nan_pad and valid is not None) else a, dtype)
+                  for a in (q, k, v))
+    vl = None if valid is None else torch.from_numpy(valid).cuda()
+    out, lse = g.im_attention_fwd(qd, kd, vd, seg, vl, phase, custom, scale, want_lse=True)
+    ref, ref_lse = oracle.im_attention_dense(q, k, v, seg, valid, phase, custom, scale, want_lse=True)
+    check_close(to_np64(out), ref, dtype, pm, f"seg={seg} phase={phase} custom={custom:#x}")
+    gl = to_np64(lse)
+    assert np.array_equal(np.isneginf(gl), np.isneginf(ref_lse))
+    fin = np.isfinite(ref_lse)
+    if fin.any():
+        assert np.abs(gl[fin] - ref_lse[fin]).max() <= (1e-4 if dtype == "f32" else 2e-2)
+    return out
+
+
+@pytest.mark.parametrize("H,hd", [(8, 8), (4, 16), (2, 32), (1, 64), (4, 8), (2, 16), (1, 32), (2, 8), (1, 16),
+                                  (16, 8), (8, 16), (4, 64), (12, 8), (6, 16), (3, 32), (10, 8)])
+def test_bf16_every_head_and_slice_width(g, H, hd):
+    """d = H*hd covers slice widths 64, 32 and 16 and every supported head_dim; ragged lengths, several key
+    tiles, a ragged last tile, a one-row segment."""
+    rng = np.random.default_rng(100 + H * 64 + hd)
+    seg, B = (37, 150, 1), 3
+    q, k, v = wk.draw_qkv(rng, B, sum(seg), H, hd, "bf16")
+    valid = np.array([[37, 150, 1], [20, 65, 1], [1, 129, 0]], dtype=np.int32)
+    for ph in PHASES:
+        _run(g, q, k, v, seg, valid, ph, "bf16")
+
+
+@pytest.mark.parametrize("seg", [(0, 70, 33), (64, 0, 128), (5, 5, 0), (130, 1, 1), (1, 1, 1), (200, 0, 0)])
+def test_bf16_empty_and_tiny_segments(g, seg):
+    rng = np.random.default_rng(sum(seg))
+    B, H, hd = 2, 8, 8
+    q, k, v = wk.draw_qkv(rng, B, sum(seg), H, hd, "bf16")
+    valid = np.stack([rng.integers(0, s + 1, size=B) for s in seg], axis=1).astype(np.int32)
+    for ph in PHASES:
+        _run(g, q, k, v, seg, None, ph, "bf16")
+        _run(g, q, k, v, seg, valid, ph, "bf16")
+
+
+def test_random_shapes_property(g):
+    rng = np.random.default_rng(2024)
+    for it in range(12):
+        H, hd = [(8, 8), (4, 16), (2, 32), (2, 64), (4, 8)][it % 5]
+        seg = tuple(int(s) for s in rng.integers(0, 180, size=3))
+        if sum(seg) == 0:
+            seg = (3, 0, 0)
+        B = int(rng.integers(1, 4))
+        q, k, v = wk.draw_qkv(rng, B, sum(seg), H, hd, "bf16")
+        valid = np.stack([rng.integers(0, s + 1, size=B) for s in seg], axis=1).astype(np.int32)
+        ph = PHASES[it % 3]
+        _run(g, q, k, v, seg, valid, ph, "bf16")
+        qf, kf, vf = (a[:, :, : max(1, H // 2)].copy() for a in (q, k, v))
+        _run(g, qf, kf, vf, seg, valid, ph, "f32")
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_custom_block_patterns_union_softmax(g, dtype):
+    rng = np.random.default_rng(31)
+    seg, B, H, hd = (40, 90, 70), 2, 4, 8
+    q, k, v = wk.draw_qkv(rng, B, sum(seg), H, hd, dtype)
+    valid = np.array([[40, 50, 70], [13, 90, 33]], dtype=np.int32)
+    # naive unmasked graph, "disorder" pattern with two open blocks in row 0, a closed row, ablation-like pattern
+    for bits in (0x1FF, 0b001100110, 0b110000000, 0b100100100, 0):
+        _run(g, q, k, v, seg, valid, oracle.PHASE_CUSTOM, dtype, custom=bits)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_explicit_scale_and_fused_vs_separate(g, dtype):
+    rng = np.random.default_rng(32)
+    seg, B, H, hd = (30, 75, 66), 2, 4, 16
+    q, k, v = wk.draw_qkv(rng, B, sum(seg), H, hd, dtype)
+    out_sep = _run(g, q, k, v, seg, None, oracle.PHASE_INTER_BWD, dtype, scale=0.4)
+    fused = torch.stack([to_dev(a, dtype) for a in (q, k, v)], dim=2).contiguous()   # [B, L, 3, H, hd]
+    out_fused = g.im_attention_fwd(fused[:, :, 0], fused[:, :, 1], fused[:, :, 2], seg, None, oracle.PHASE_INTER_BWD,
+                                   scale=0.4)
+    assert torch.equal(out_sep, out_fused)
+
+
+def test_f32_large_head_dim_and_masking(g):
+    rng = np.random.default_rng(33)
+    seg, B, H, hd = (9, 20, 14), 2, 2, 40
+    q, k, v = wk.draw_qkv(rng, B, sum(seg), H, hd, "f32")
+    valid = np.array([[9, 0, 14], [4, 20, 1]], dtype=np.int32)
+    for ph in PHASES:
+        _run(g, q, k, v, seg, valid, ph, "f32")
+
+
+def test_masked_blocks_do_not_influence_gpu_output(g):
+    """Information-disorder invariant on the GPU: keys/values of closed blocks and padded rows may hold anything."""
+    rng = np.random.default_rng(34)
+    seg, B, H, hd = (50, 100, 80), 2, 8, 8
+    q, k, v = wk.draw_qkv(rng, B, sum(seg), H, hd, "bf16")
+    valid = np.array([[50, 70, 80], [25, 100, 41]], dtype=np.int32)
+    vl = torch.from_numpy(valid).cuda()
+    off = [0, 50, 150]
+    base = g.im_attention_fwd(*(to_dev(a, "bf16") for a in (q, k, v)), seg, vl, oracle.PHASE_INTER_FWD)
+    al = oracle.allowed_blocks(oracle.PHASE_INTER_FWD)
+    for s in range(3):
+        k2, v2 = k.copy(), v.copy()
+        for r in range(3):
+            if not al[s, r]:
+                k2[:, off[r]:off[r] + seg[r]] = np.inf
+                v2[:, off[r]:off[r] + seg[r]] = np.nan
+        k2, v2 = (wk.fill_padding(a, seg, valid, np.nan) for a in (k2, v2))
+        out = g.im_attention_fwd(*(to_dev(a, "bf16") for a in (q, k2, v2)), seg, vl, oracle.PHASE_INTER_FWD)
+        assert torch.equal(out[:, off[s]:off[s] + seg[s]], base[:, off[s]:off[s] + seg[s]])
+
+
+def test_run_to_run_bit_identical(g):
+    inp = wk.make_inputs(3, batch=4)
+    wl = inp["workload"]
+    vl = torch.from_numpy(inp["valid_len"]).cuda()
+    qkv = g.im_qkv_proj(to_dev(inp["x"], "bf16"), to_dev(inp["layer"]["w_qkv"], "bf16"), None, wl.seg_len, wl.heads, vl)
+    outs = [g.im_attention_fwd(qkv[:, :, 0], qkv[:, :, 1], qkv[:, :, 2], wl.seg_len, vl, oracle.PHASE_INTRA).clone()
+            for _ in range(3)]
+    assert torch.equal(outs[0], outs[1]) and torch.equal(outs[0], outs[2])
+
+
+def test_out_of_range_valid_len_is_clamped_and_flagged(g):
+    rng = np.random.default_rng(35)
+    seg, B, H, hd = (20, 30, 25), 2, 4, 8
+    q, k, v = wk.draw_qkv(rng, B, sum(seg), H, hd, "bf16")
+    bad = np.array([[25, 30, -3], [20, 99, 25]], dtype=np.int32)
+    clamped = np.clip(bad, 0, np.array(seg)[None]).astype(np.int32)
+    g.last_device_status()
+    out = g.im_attention_fwd(*(to_dev(a, "bf16") for a in (q, k, v)), seg, torch.from_numpy(bad).cuda(),
+                             oracle.PHASE_INTER_FWD)
+    code, flags = g.last_device_status()
+    assert code == 0 and flags == g.DEVFLAG_CLAMPED
+    ref = oracle.im_attention_dense(q, k, v, seg, clamped, oracle.PHASE_INTER_FWD)
+    check_close(to_np64(out), ref, "bf16", pad_mask(seg, clamped, B), "clamped")
+    assert g.last_device_status() == (0, 0)
+
+
+def test_host_side_rejection(g):
+    lib = g.load()
+    dev = torch.device("cuda")
+    t = torch.zeros((1, 16, 64), dtype=torch.bfloat16, device=dev)
+    ok = g.make_shape(1, (4, 8, 4), 64, 8, None, g.DTYPE_BF16, g.PHASE_INTRA)
+    p = t.data_ptr()
+    o_buf = torch.zeros_like(t)
+    call = lambda sh, q=p, k=p, v=p, rs=64, o=o_buf.data_ptr(): lib.gsit_im_attention_fwd(ctypes.byref(sh), q, k, v, rs, o, None, None, 0, None)
+    assert call(ok) == 0
+    assert call(ok, q=None) == 1 and call(ok, rs=32) == 1 and call(ok, q=p + 2) == 1 and call(ok, rs=68) == 1
+    assert call(g.make_shape(1, (4, 8, 4), 64, 7, None, g.DTYPE_BF16, g.PHASE_INTRA)) == 1      # d % heads
+    assert call(g.make_shape(0, (4, 8, 4), 64, 8, None, g.DTYPE_BF16, g.PHASE_INTRA)) == 1      # batch
+    assert call(g.make_shape(1, (4, -8, 4), 64, 8, None, g.DTYPE_BF16, g.PHASE_INTRA)) == 1     # negative length
+    assert call(g.make_shape(1, (0, 0, 0), 64, 8, None, g.DTYPE_BF16, g.PHASE_INTRA)) == 1      # empty sequence
+    assert call(g.make_shape(1, (4, 8, 4), 64, 8, None, g.DTYPE_BF16, 7)) == 1                  # bad phase
+    assert call(g.make_shape(1, (4, 8, 4), 64, 8, None, g.DTYPE_BF16, g.PHASE_CUSTOM, 0x400)) == 1
+    assert call(g.make_shape(1, (4, 8, 4), 64, 8, None, 5, g.PHASE_INTRA)) == 1                 # bad dtype
+    assert call(g.make_shape(1, (4, 8, 4), 64, 16, None, g.DTYPE_BF16, g.PHASE_INTRA)) == 2     # head_dim 4 unsupported
+    assert call(g.make_shape(1, (4, 8, 4), 24, 3, None, g.DTYPE_BF16, g.PHASE_INTRA)) == 2      # d % 16
+    # layer: workspace too small / missing
+    w = {k_: torch.zeros(s, dtype=torch.bfloat16, device=dev) for k_, s in
+         (("w_qkv", (192, 64)), ("w_o", (64, 64)), ("w_1", (256, 64)), ("w_2", (64, 256)))}
+    x = torch.zeros((1, 16, 64), dtype=torch.float32, device=dev)
+    with pytest.raises(g.GsitError) as e:
+        g.im_layer_fwd(x, w, (4, 8, 4), 8, workspace=torch.empty(256, dtype=torch.uint8, device=dev))
+    assert e.value.code == 3
+    assert g.workspace_bytes(ok, g.CALL_ATTENTION) == 0 and g.workspace_bytes(ok, g.CALL_LAYER, 256) > 0
+    torch.cuda.synchronize()

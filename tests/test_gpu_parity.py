@@ -1,0 +1,144 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, element by element, on the same
+seeded inputs, at the five workload shapes (batch reduced where the oracle would take minutes)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads as wk
+from gpu_util import check_close, pad_mask, to_dev, to_np64, weights_to_dev
+
+pytestmark = pytest.mark.gpu
+PHASES = [oracle.PHASE_INTER_FWD, oracle.PHASE_INTER_BWD, oracle.PHASE_INTRA]
+
+
+@pytest.fixture(scope="module")
+def g():
+    import paper_2505_01068_b200 as lib
+    lib.load()
+    return lib
+
+
+def _attention_case(g, x, w_qkv, seg, heads, valid, dtype, phases=PHASES, nan_padding=False, check_lse=True):
+    """qkv projection + attention per phase, each compared with the oracle fed the same (rounded) arrays."""
+    B = x.shape[0]
+    pm = pad_mask(seg, valid, B)
+    x_dev_np = wk.fill_padding(x, seg, valid, np.nan) if nan_padding else x
+    vl = None if valid is None else torch.from_numpy(valid).cuda()
+    xd, wd = to_dev(x_dev_np, dtype), to_dev(w_qkv, dtype)
+    qkv = g.im_qkv_proj(xd, wd, None, seg, heads, vl)
+    ref_qkv = oracle.qkv_proj(x, w_qkv, None, seg, heads, valid)
+    check_close(to_np64(qkv).reshape(B, -1, 3 * x.shape[2]), ref_qkv.reshape(B, -1, 3 * x.shape[2]), dtype, pm, "qkv_proj")
+    # the oracle attends over exactly the q, k, v the GPU attention reads (the GPU's own rounded projection)
+    qkv64 = to_np64(qkv)
+    res = {}
+    for ph in phases:
+        out, lse = g.im_attention_fwd(qkv[:, :, 0], qkv[:, :, 1], qkv[:, :, 2], seg, vl, ph, want_lse=True)
+        ref, ref_lse = oracle.im_attention_dense(qkv64[:, :, 0], qkv64[:, :, 1], qkv64[:, :, 2], seg, valid, ph, want_lse=True)
+        res[ph] = check_close(to_np64(out), ref, dtype, pm, f"attention phase {ph}")
+        if check_lse:
+            gl = to_np64(lse)
+            fin = np.isfinite(ref_lse)
+            assert np.array_equal(np.isneginf(gl), np.isneginf(ref_lse))
+            assert np.abs(gl[fin] - ref_lse[fin]).max() <= (1e-4 if dtype == "f32" else 2e-2)
+    code, flags = g.last_device_status()
+    assert code == 0 and flags == 0
+    return res
+
+
+def test_cfg1_tiny_f32_attention_and_layers(g):
+    inp = wk.make_inputs(1)
+    wl = inp["workload"]
+    _attention_case(g, inp["x"], inp["layer"]["w_qkv"], wl.seg_len, wl.heads, None, "f32")
+    wd = weights_to_dev(inp["layer"], "f32")
+    xd = to_dev(inp["x"])
+    for ph in PHASES:
+        y = g.im_layer_fwd(xd, wd, wl.seg_len, wl.heads, None, ph)
+        ref = oracle.im_layer_fwd(inp["x"], inp["layer"], wl.seg_len, wl.heads, None, ph)
+        check_close(to_np64(y), ref, "f32", None, f"layer phase {ph}")
+
+
+def test_cfg1_f32_wo_projected_attention(g):
+    """Attention followed by the shared W_o (the layer with the MLP switched off and x = 0 residual removed)."""
+    inp = wk.make_inputs(1)
+    wl = inp["workload"]
+    w = dict(inp["layer"], w_2=np.zeros_like(inp["layer"]["w_2"]))
+    wd = weights_to_dev(w, "f32")
+    for ph in PHASES:
+        y = g.im_layer_fwd(to_dev(inp["x"]), wd, wl.seg_len, wl.heads, None, ph)
+        ref = oracle.im_layer_fwd(inp["x"], w, wl.seg_len, wl.heads, None, ph)
+        check_close(to_np64(y), ref, "f32", None, f"x + O W_o phase {ph}")
+
+
+def test_cfg2_aligned_bf16(g):
+    inp = wk.make_inputs(2)
+    wl = inp["workload"]
+    _attention_case(g, inp["x"], inp["layer"]["w_qkv"], wl.seg_len, wl.heads, None, "bf16")
+
+
+def test_cfg3_mosi_unaligned_bf16_nan_padding(g):
+    inp = wk.make_inputs(3)
+    wl = inp["workload"]
+    _attention_case(g, inp["x"], inp["layer"]["w_qkv"], wl.seg_len, wl.heads, inp["valid_len"], "bf16", nan_padding=True)
+
+
+def test_cfg4_mosei_attention_and_layer_bf16(g):
+    inp = wk.make_inputs(4, batch=8)
+    wl = inp["workload"]
+    _attention_case(g, inp["x"], inp["layer"]["w_qkv"], wl.seg_len, wl.heads, inp["valid_len"], "bf16", nan_padding=True)
+    vl = torch.from_numpy(inp["valid_len"]).cuda()
+    pm = pad_mask(wl.seg_len, inp["valid_len"], 8)
+    xd = to_dev(wk.fill_padding(inp["x"], wl.seg_len, inp["valid_len"], np.nan))
+    for ph, w in ((oracle.PHASE_INTER_FWD, inp["fwd_layers"][0]), (oracle.PHASE_INTER_BWD, inp["bwd_layers"][0])):
+        y = g.im_layer_fwd(xd, weights_to_dev(w, "bf16"), wl.seg_len, wl.heads, vl, ph)
+        ref = oracle.im_layer_fwd(inp["x"], w, wl.seg_len, wl.heads, inp["valid_len"], ph)
+        check_close(to_np64(y), ref, "bf16", pm, f"layer d=64 phase {ph}")
+    # intra layer at width 2d with 8 heads of 16
+    rng = np.random.default_rng(77)
+    x2 = rng.standard_normal((8, wl.L, 2 * wl.d_model), dtype=np.float32)
+    w = inp["intra_layers"][0]
+    y = g.im_layer_fwd(to_dev(x2), weights_to_dev(w, "bf16"), wl.seg_len, 8, vl, oracle.PHASE_INTRA)
+    ref = oracle.im_layer_fwd(x2, w, wl.seg_len, 8, inp["valid_len"], oracle.PHASE_INTRA)
+    check_close(to_np64(y), ref, "bf16", pm, "intra layer d=128")
+
+
+def test_cfg4_full_stack_bf16(g):
+    inp = wk.make_inputs(4, batch=4)
+    wl = inp["workload"]
+    n_f, n_b, n_i, ih = wl.stack
+    vl = torch.from_numpy(inp["valid_len"]).cuda()
+    stack = g.GsitStack([weights_to_dev(w, "bf16") for w in inp["fwd_layers"]],
+                        [weights_to_dev(w, "bf16") for w in inp["bwd_layers"]],
+                        [weights_to_dev(w, "bf16") for w in inp["intra_layers"]], wl.seg_len, wl.heads, ih)
+    y = stack.forward(to_dev(inp["x"]), vl)
+    ref = oracle.gsit_stack_fwd(inp["x"], inp["fwd_layers"], inp["bwd_layers"], inp["intra_layers"], wl.seg_len,
+                                wl.heads, ih, inp["valid_len"])
+    pm = pad_mask(wl.seg_len, inp["valid_len"], 4)
+    got = to_np64(y)
+    assert np.isfinite(got).all() and np.all(got[pm] == 0.0)
+    err = np.abs(got - ref)
+    # ten bf16 layers deep: report against the per-call tolerance scaled by depth (each layer alone is checked above)
+    assert err.max() <= 10 * 2e-2 and err.mean() <= 10 * 2e-3, (err.max(), err.mean())
+
+
+def test_cfg5_scaled_hd64_bf16(g):
+    """Scaled shape (L=2176, d=512, 8 heads of 64) on two samples, one of them padded to half length."""
+    wl = wk.WORKLOADS[5]
+    B = 2
+    rng = np.random.default_rng(wl.seed)
+    q, k, v = wk.draw_qkv(rng, B, wl.L, wl.heads, wl.d_model // wl.heads, "bf16")
+    valid = np.array([wl.seg_len, [s // 2 for s in wl.seg_len]], dtype=np.int32)
+    vl = torch.from_numpy(valid).cuda()
+    pm = pad_mask(wl.seg_len, valid, B)
+    qd, kd, vd = (to_dev(a, "bf16") for a in (q, k, v))
+    for ph in PHASES:
+        out = g.im_attention_fwd(qd, kd, vd, wl.seg_len, vl, ph)
+        ref = oracle.im_attention_dense(q, k, v, wl.seg_len, valid, ph)
+        check_close(to_np64(out), ref, "bf16", pm, f"cfg5 attention phase {ph}")
+    # the shared projection at d=512
+    x = wk.storage_round(rng.standard_normal((2, wl.L, wl.d_model), dtype=np.float32), "bf16")
+    w = wk.draw_layer_weights(rng, wl.d_model, 4 * wl.d_model, "bf16")["w_qkv"]
+    qkv = g.im_qkv_proj(to_dev(x, "bf16"), to_dev(w, "bf16"), None, wl.seg_len, wl.heads, vl[:2].contiguous())
+    ref = oracle.qkv_proj(x, w, None, wl.seg_len, wl.heads, valid[:2])
+    check_close(to_np64(qkv).reshape(2, wl.L, -1), ref.reshape(2, wl.L, -1), "bf16", pad_mask(wl.seg_len, valid[:2], 2),
+                "qkv_proj d=512")
