@@ -39,7 +39,7 @@ def test_workspace_query_needs_no_gpu():
     sh = g.make_shape(2, (8, 12, 10), 32, 4, None, g.DTYPE_F32, g.PHASE_INTRA)
     assert g.workspace_bytes(sh, g.CALL_ATTENTION) == 0
     rows = 2 * 30
-    assert g.workspace_bytes(sh, g.CALL_LAYER, 128) >= rows * (32 * 4 * 4 + 96 * 4 + 128 * 4)
+    assert g.workspace_bytes(sh, g.CALL_LAYER, 128) >= rows * (32 * 4 * 3 + 96 * 4 + 128 * 4)
     bad = g.make_shape(2, (8, 12, 10), 30, 4, None, g.DTYPE_F32, g.PHASE_INTRA)
     try:
         g.workspace_bytes(bad, g.CALL_LAYER, 128)
