@@ -1,0 +1,373 @@
+#!/usr/bin/env python
+"""Benchmark of the IM-attention hot path on synthetic MOSEI-shaped data.
+
+A step is one forward pass of the whole hot path over one batch: the GsiT fusion stack (forward-ring and
+backward-ring encoders at width d, intra-modal encoder at width 2d), every layer being LayerNorm -> shared
+QKV projection -> IM attention -> out-projection + residual -> LayerNorm -> MLP + residual, all inside the
+library's kernels.  `value` is valid (non padded) tokens per second with inputs resident in HBM; `e2e`
+includes the host->device copy of the batch and the device->host copy of the result every step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload 4|5]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+from pathlib import Path
+
+import numpy as np
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+import workloads as wk  # noqa: E402
+
+METRIC = "IM-attention tokens/s (valid tokens through the GsiT IM stack), MOSEI-shaped"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+L2_BYTES = 126 * 1024 * 1024
+
+
+def peaks():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        d = json.loads(p.read_text())
+        return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of the benchmark GPU through NVML while the timed region runs."""
+
+    def __init__(self, torch_device_index: int):
+        self.samples, self.reasons, self.max_mhz, self._stop = [], set(), None, threading.Event()
+        self._thread, self._h, self._nv = None, None, None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(torch_device_index).uuid)
+            uuid = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
+            self._h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode() if hasattr(uuid, "encode") else uuid)
+            self._nv = pynvml
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception as e:  # NVML missing: the clocks object then says so
+            self.error = repr(e)
+
+    def _names(self, mask: int):
+        nv = self._nv
+        table = {"sw_power_cap": "nvmlClocksThrottleReasonSwPowerCap", "hw_slowdown": "nvmlClocksThrottleReasonHwSlowdown",
+                 "hw_thermal_slowdown": "nvmlClocksThrottleReasonHwThermalSlowdown",
+                 "sw_thermal_slowdown": "nvmlClocksThrottleReasonSwThermalSlowdown",
+                 "hw_power_brake": "nvmlClocksThrottleReasonHwPowerBrakeSlowdown",
+                 "sync_boost": "nvmlClocksThrottleReasonSyncBoost"}
+        return {n for n, attr in table.items() if hasattr(nv, attr) and (mask & getattr(nv, attr))}
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                self.reasons |= self._names(int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)))
+            except Exception:
+                pass
+            self._stop.wait(0.02)
+
+    def __enter__(self):
+        if self._h is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                    "note": getattr(self, "error", "no samples")}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def stack_flops_and_tokens(wl, valid_len, batch):
+    """Valid tokens per step, and per attention call: useful pairs, useful FLOPs, compulsory bytes."""
+    seg = wl.seg_len
+    n = np.tile(np.asarray(seg)[None], (batch, 1)) if valid_len is None else valid_len
+    tokens = int(n.sum())
+    ring = np.array([[0, 1, 0], [0, 0, 1], [1, 0, 0]])
+    info = {}
+    for name, allowed, d in (("cross", ring, wl.d_model), ("intra", np.eye(3, dtype=int), 2 * wl.d_model)):
+        U = wk.useful_pairs(seg, valid_len, allowed, batch)
+        info[name] = {"pairs": U, "flops": 4.0 * d * U, "bytes": 4.0 * tokens * d * 2 + 12.0 * batch, "d": d}
+    return tokens, info
+
+
+def run_reference(args):
+    """The CPU oracle, as it stands, timed on the host cores on a bounded sample of the same workload."""
+    import oracle
+    wl = wk.WORKLOADS[args.workload]
+    sub = args.ref_batch
+    inp = wk.make_inputs(args.workload, batch=sub)
+    tokens = int(inp["valid_len"].sum()) if inp["valid_len"] is not None else sub * wl.L
+    n_f, n_b, n_i, ih = wl.stack if wl.stack else (1, 0, 0, wl.heads)
+
+    def step():
+        if wl.stack:
+            oracle.gsit_stack_fwd(inp["x"], inp["fwd_layers"], inp["bwd_layers"], inp["intra_layers"], wl.seg_len,
+                                  wl.heads, ih, inp["valid_len"])
+        else:
+            oracle.im_layer_fwd(inp["x"], inp["layer"], wl.seg_len, wl.heads, inp["valid_len"], oracle.PHASE_INTER_FWD)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / max(1, args.steps)
+    value = tokens / dt
+    sample = f"{sub} of {wl.batch} samples per step (valid tokens {tokens}), fp64 dense-mask oracle, whole stack"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"cfg{wl.index}:{wl.name}", "batch": sub, "seg_len": list(wl.seg_len),
+                       "d_model": wl.d_model, "heads": wl.heads},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def _time_graph_replays(torch, graphs, steps, dist, world):
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    beg, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    beg.record()
+    for k in range(steps):
+        graphs[k % len(graphs)].replay()
+    end.record()
+    torch.cuda.synchronize()
+    ms = beg.elapsed_time(end)
+    if world > 1:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+        dist.barrier()
+    return ms
+
+
+def time_attention_alone(torch, g, wl, valid_dev, d, heads, phase, reps=4):
+    """One IM-attention call timed alone: a CUDA graph of launches rotating over qkv/out buffer sets larger than L2."""
+    B, L = valid_dev.shape[0], wl.L
+    set_bytes = B * L * 4 * d * 2
+    nsets = max(2, int(np.ceil(1.5 * L2_BYTES / set_bytes)))
+    gen = torch.Generator(device="cuda").manual_seed(1234)
+    qkvs = [torch.randn((B, L, 3, heads, d // heads), device="cuda", generator=gen).bfloat16() for _ in range(nsets)]
+    outs = [torch.empty((B, L, d), device="cuda", dtype=torch.bfloat16) for _ in range(nsets)]
+    run = lambda i: g.im_attention_fwd(qkvs[i][:, :, 0], qkvs[i][:, :, 1], qkvs[i][:, :, 2], wl.seg_len, valid_dev, phase, out=outs[i])
+    for i in range(nsets):
+        run(i)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for _ in range(reps):
+            for i in range(nsets):
+                run(i)
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    beg, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    beg.record()
+    for _ in range(5):
+        graph.replay()
+    end.record()
+    torch.cuda.synchronize()
+    return beg.elapsed_time(end) * 1e-3 / (5 * reps * nsets), nsets
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2505_01068_b200 as g
+
+    rank, world = int(os.environ.get("RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    g.load()
+    wl = wk.WORKLOADS[args.workload]
+    assert wl.stack is not None, "the benchmark step is the full stack (workload 4)"
+    n_f, n_b, n_i, ih = wl.stack
+    # weak scaling: every rank owns an independent batch of the same shape (no data-path collective)
+    inp = wk.make_inputs(wl.index, seed=wl.seed + 1000 * rank)
+    B = wl.batch
+    valid = inp["valid_len"]
+    vl = torch.from_numpy(valid).cuda()
+    tokens, info = stack_flops_and_tokens(wl, valid, B)
+
+    def dev_w(w):
+        return {k: (None if a is None else (torch.from_numpy(a).cuda().bfloat16() if k.startswith("w_") else torch.from_numpy(a).cuda()))
+                for k, a in w.items()}
+
+    stack = g.GsitStack([dev_w(w) for w in inp["fwd_layers"]], [dev_w(w) for w in inp["bwd_layers"]],
+                        [dev_w(w) for w in inp["intra_layers"]], wl.seg_len, wl.heads, ih)
+    x_host = torch.from_numpy(inp["x"]).pin_memory()
+    nbuf = max(2, int(np.ceil(1.2 * L2_BYTES / x_host.numel() / 4)))
+    xbufs = [x_host.cuda() for _ in range(nbuf)]
+    launches_per_step = 7 * (n_f + n_b + n_i)
+
+    for i in range(max(1, min(args.warmup, 2))):           # eager warm-up (module load, attributes, buffers)
+        stack.forward(xbufs[i % nbuf], vl)
+    torch.cuda.synchronize()
+    code, flags = g.last_device_status()
+    assert code == 0 and flags == 0, (code, flags)
+    graphs = []
+    for i in range(nbuf):
+        gr = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gr):
+            y_dev = stack.forward(xbufs[i], vl)
+        graphs.append(gr)
+    for k in range(args.warmup):
+        graphs[k % nbuf].replay()
+    torch.cuda.synchronize()
+
+    with ClockSampler(local) as clocks:
+        ms = _time_graph_replays(torch, graphs, args.steps, dist, world)
+    ms_per_step = ms / args.steps
+    value = tokens * world / (ms_per_step * 1e-3)
+    if world > 1:
+        tt = torch.tensor([float(tokens)], device="cuda")
+        dist.all_reduce(tt)
+        value = float(tt.item()) / (ms_per_step * 1e-3)
+
+    # ---- end to end: pinned host batch -> device -> stack -> host, every step ----
+    y_host = torch.empty(tuple(y_dev.shape), dtype=torch.float32).pin_memory()
+    e2e_steps = max(3, min(args.steps, 30))
+
+    def e2e_step():
+        xbufs[0].copy_(x_host, non_blocking=True)
+        graphs[0].replay()
+        y_host.copy_(y_dev, non_blocking=True)
+
+    for _ in range(3):
+        e2e_step()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    torch.cuda.synchronize()
+    e2e_s = torch.tensor([(time.perf_counter() - t0) / e2e_steps], device="cuda")
+    if world > 1:
+        dist.all_reduce(e2e_s, op=dist.ReduceOp.MAX)
+    e2e_value = tokens * world / float(e2e_s.item())
+
+    # ---- per-kernel device times inside the step (eager, CUDA events around each launch) ----
+    trace_steps = max(1, min(args.steps, 10))
+    g.trace_enable(True)
+    for k in range(trace_steps):
+        stack.forward(xbufs[k % nbuf], vl)
+    torch.cuda.synchronize()
+    att = g.trace_launches(g.KERNEL_ATTENTION)
+    lin_ms, lin_n = g.trace_read(g.KERNEL_LINEAR)
+    ln_ms, ln_n = g.trace_read(g.KERNEL_LAYERNORM)
+    g.trace_enable(False)
+    per_step = n_f + n_b + n_i
+    att = np.asarray(att).reshape(trace_steps, per_step)
+    cross_s = float(att[:, : n_f + n_b].mean()) * 1e-3
+    intra_s = float(att[:, n_f + n_b:].mean()) * 1e-3 if n_i else None
+    pk, pk_kind = peaks()
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- IM attention timed alone (burst), both block patterns, against both rooflines ----
+    ex2_rate = 148 * 16 * (clocks.summary()["sm_max_mhz"] or 1965) * 1e6     # MUFU ex2 per second at max clock
+    attention = {}
+    for name, d, heads, phase in (("cross", wl.d_model, wl.heads, g.PHASE_INTER_FWD), ("intra", 2 * wl.d_model, ih, g.PHASE_INTRA)):
+        sec, nsets = time_attention_alone(torch, g, wl, vl, d, heads, phase)
+        I = info[name]
+        t_tc, t_hbm = I["flops"] / (pk["bf16_tflops"] * 1e12), I["bytes"] / (pk["hbm_gbs"] * 1e9)
+        t_exp = heads * I["pairs"] / ex2_rate
+        attention[name] = {"us": sec * 1e6, "tokens_per_s": tokens / sec, "useful_tflops": I["flops"] / sec / 1e12,
+                           "achieved_gbs": I["bytes"] / sec / 1e9, "frac_roofline": max(t_tc, t_hbm) / sec,
+                           "frac_three_way": max(t_tc, t_hbm, t_exp) / sec, "t_tensor_us": t_tc * 1e6,
+                           "t_hbm_us": t_hbm * 1e6, "t_exp_us": t_exp * 1e6, "d_model": d, "heads": heads,
+                           "buffer_sets": nsets, "in_step_us": (cross_s if name == "cross" else intra_s) * 1e6}
+
+    # ---- CPU baseline: the oracle on a bounded sample of the same workload ----
+    import oracle
+    sub = args.ref_batch
+    ref_inp = wk.make_inputs(wl.index, batch=sub)
+    ref_tokens = int(ref_inp["valid_len"].sum())
+    ref_step = lambda: oracle.gsit_stack_fwd(ref_inp["x"], ref_inp["fwd_layers"], ref_inp["bwd_layers"],
+                                             ref_inp["intra_layers"], wl.seg_len, wl.heads, ih, ref_inp["valid_len"])
+    ref_step()
+    t0 = time.perf_counter()
+    ref_step()
+    cpu_s = time.perf_counter() - t0
+
+    cross = info["cross"]
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": f"cfg{wl.index}:{wl.name}", "batch_per_gpu": B, "seg_len": list(wl.seg_len), "d_model": wl.d_model,
+                   "heads": wl.heads, "stack": f"fwd x{n_f} + bwd x{n_b} at d={wl.d_model} (hd={wl.d_model // wl.heads}), "
+                   f"intra x{n_i} at d={2 * wl.d_model} (hd={2 * wl.d_model // ih})",
+                   "valid_tokens_per_step": tokens, "padded_tokens_per_step": B * wl.L,
+                   "l2": f"inputs rotate over {nbuf} device copies ({nbuf * x_host.numel() * 4 >> 20} MiB > 126 MiB L2); "
+                         "the step's scratch alone is larger than L2", "launch": "one CUDA graph per input buffer"},
+        "clocks": clocks.summary(),
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(x_host.numel() * 4),
+                "d2h_bytes_per_step": int(y_host.numel() * 4)},
+        "gpu_launches": launches_per_step * args.steps,
+        "roofline": {"kernel": "attn_bf16_kernel<8,64> (cross-modal IM attention inside the step)", "bound": "hbm",
+                     "achieved": cross["bytes"] / cross_s / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                     "frac": cross["bytes"] / cross_s / 1e9 / pk["hbm_gbs"], "traffic": None, "peak_kind": "of " + pk_kind,
+                     "launch_us": cross_s * 1e6, "algorithmic_bytes": cross["bytes"]},
+        "cpu_baseline": {"value": ref_tokens / cpu_s, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": f"{sub} of {B} samples, one step (valid tokens {ref_tokens}) in {cpu_s:.2f} s"},
+        "attention": attention,
+        "step_kernel_ms": {"attention": float(att.sum()) / trace_steps, "linear": lin_ms / trace_steps,
+                           "layernorm": ln_ms / trace_steps, "launches": {"attention": per_step, "linear": lin_n // trace_steps,
+                                                                          "layernorm": ln_n // trace_steps}},
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="gsit", choices=["gsit", "reference"])
+    ap.add_argument("--workload", type=int, default=4)
+    ap.add_argument("--ref-batch", type=int, default=16, help="samples per step of the CPU oracle")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        args.steps = 2 if args.steps is None else args.steps
+        args.warmup = 1 if args.warmup is None else args.warmup
+        if int(os.environ.get("RANK", 0)) == 0:
+            run_reference(args)
+        return
+    args.steps = 200 if args.steps is None else args.steps
+    args.warmup = max(3, 5 if args.warmup is None else args.warmup)
+    run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

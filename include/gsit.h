@@ -137,6 +137,19 @@ size_t gsit_workspace_bytes(const gsit_shape* shape, int which_call, int32_t d_f
  * Returns GSIT_ERR_TIMEOUT if GSIT_DEVFLAG_TIMEOUT was set, GSIT_ERR_CUDA on a CUDA error, else GSIT_OK. */
 gsit_status gsit_last_device_status(gsit_stream stream, uint32_t* flags);
 
+/* Profiling aid (host state, off by default).  While enabled, every kernel launch of the library is bracketed
+ * by a pair of CUDA events on the launching stream (up to 8192 launches are kept; later ones go unrecorded).
+ * Do not enable it while a stream is being captured into a CUDA graph. */
+typedef enum { GSIT_KERNEL_ATTENTION = 0, GSIT_KERNEL_LINEAR = 1, GSIT_KERNEL_LAYERNORM = 2 } gsit_kernel_kind;
+gsit_status gsit_trace_enable(int on);
+/* Waits for the recorded events, returns the summed device time (ms) and launch count of one kernel kind since the
+ * last gsit_trace_reset(); both outputs are HOST pointers. */
+gsit_status gsit_trace_read(int kernel_kind, float* total_ms, int32_t* launches);
+/* Per-launch device times (ms) of one kernel kind, in launch order, into out_ms[0..capacity); *launches receives
+ * the number written.  HOST pointers. */
+gsit_status gsit_trace_launches(int kernel_kind, float* out_ms, int32_t capacity, int32_t* launches);
+gsit_status gsit_trace_reset(void);
+
 const char* gsit_status_string(gsit_status status);
 int gsit_version(void);
 

@@ -39,7 +39,9 @@ class LayerWeights(ctypes.Structure):
 
 
 EXPORTS = ("gsit_im_qkv_proj", "gsit_im_attention_fwd", "gsit_im_layer_fwd", "gsit_workspace_bytes",
-           "gsit_last_device_status", "gsit_status_string", "gsit_version")
+           "gsit_last_device_status", "gsit_status_string", "gsit_version", "gsit_trace_enable", "gsit_trace_read",
+           "gsit_trace_launches", "gsit_trace_reset")
+KERNEL_ATTENTION, KERNEL_LINEAR, KERNEL_LAYERNORM = 0, 1, 2
 
 
 def load():
@@ -66,6 +68,8 @@ def load():
     lib.gsit_status_string.argtypes = [ctypes.c_int]
     lib.gsit_status_string.restype = ctypes.c_char_p
     lib.gsit_version.restype = ctypes.c_int
+    lib.gsit_trace_enable.argtypes = [ctypes.c_int]
+    lib.gsit_trace_read.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]
     _lib = lib
     return lib
 
@@ -119,6 +123,25 @@ def last_device_status() -> tuple[int, int]:
     flags = ctypes.c_uint32(0)
     code = load().gsit_last_device_status(_stream(), ctypes.byref(flags))
     return int(code), int(flags.value)
+
+
+def trace_enable(on: bool):
+    _check(load().gsit_trace_enable(int(bool(on))), "gsit_trace_enable")
+    _check(load().gsit_trace_reset(), "gsit_trace_reset")
+
+
+def trace_read(kind: int) -> tuple[float, int]:
+    """(total device ms, launches) of one kernel kind since tracing was (re)enabled."""
+    ms, n = ctypes.c_float(0), ctypes.c_int32(0)
+    _check(load().gsit_trace_read(int(kind), ctypes.byref(ms), ctypes.byref(n)), "gsit_trace_read")
+    return float(ms.value), int(n.value)
+
+
+def trace_launches(kind: int, capacity: int = 8192) -> list[float]:
+    """Per-launch device times (ms) of one kernel kind, in launch order."""
+    buf, n = (ctypes.c_float * capacity)(), ctypes.c_int32(0)
+    _check(load().gsit_trace_launches(int(kind), buf, capacity, ctypes.byref(n)), "gsit_trace_launches")
+    return [float(buf[i]) for i in range(n.value)]
 
 
 def im_qkv_proj(x, w_qkv, b_qkv, seg_len, heads, valid_len=None, out=None):

@@ -105,12 +105,46 @@ LayerScratch layer_scratch(const Geometry& g, int dtype, int d_ff) {
   return s;
 }
 
+// ---- optional event tracing of the library's launches ----
+struct TraceRec { cudaEvent_t beg, end; int kind; };
+constexpr int TRACE_CAP = 8192;
+bool g_trace_on = false;
+int g_trace_n = 0;            // records in use
+int g_trace_created = 0;      // event pairs created so far (reused after a reset)
+TraceRec g_trace[TRACE_CAP];
+
+struct TraceScope {
+  cudaStream_t st;
+  TraceRec* rec = nullptr;
+  TraceScope(int kind, cudaStream_t s) : st(s) {
+    if (!g_trace_on || g_trace_n >= TRACE_CAP) return;
+    TraceRec* r = &g_trace[g_trace_n];
+    if (g_trace_n >= g_trace_created) {
+      if (cudaEventCreate(&r->beg) != cudaSuccess || cudaEventCreate(&r->end) != cudaSuccess) return;
+      ++g_trace_created;
+    }
+    r->kind = kind;
+    if (cudaEventRecord(r->beg, st) != cudaSuccess) return;
+    rec = r;
+    ++g_trace_n;
+  }
+  ~TraceScope() { if (rec) cudaEventRecord(rec->end, st); }
+};
+
 gsit_status run_linear(const Geometry& g, int dtype, const LinearArgs& a, cudaStream_t st) {
+  TraceScope t(GSIT_KERNEL_LINEAR, st);
   return from_cuda(dtype == GSIT_BF16 ? launch_linear_bf16(g, a, st) : launch_linear_f32(g, a, st));
+}
+
+gsit_status run_layernorm(const Geometry& g, const float* x, int64_t ldx, const float* gamma, const float* beta,
+                          float eps, void* y, int out_bf16, cudaStream_t st) {
+  TraceScope t(GSIT_KERNEL_LAYERNORM, st);
+  return from_cuda(launch_layernorm(g, x, ldx, gamma, beta, eps, y, out_bf16, st));
 }
 
 gsit_status run_attention(const Geometry& g, int dtype, const void* q, const void* k, const void* v,
                           int64_t row_stride, void* out, float* lse, float scale, cudaStream_t st) {
+  TraceScope t(GSIT_KERNEL_ATTENTION, st);
   if (dtype == GSIT_BF16)
     return from_cuda(launch_attn_bf16(g, static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k),
                                       static_cast<const __nv_bfloat16*>(v), row_stride,
@@ -190,7 +224,7 @@ gsit_status gsit_im_layer_fwd(const gsit_shape* shape, const gsit_layer_weights*
   const int M = g.batch * g.L, d = g.d;
 
   // h = LN1(x)
-  if ((st = from_cuda(launch_layernorm(g, x, x_row_stride, w->ln1_gamma, w->ln1_beta, eps, h, bf, cs))) != GSIT_OK) return st;
+  if ((st = run_layernorm(g, x, x_row_stride, w->ln1_gamma, w->ln1_beta, eps, h, bf, cs)) != GSIT_OK) return st;
   // qkv = h W_qkv^T + b_qkv   (shared projection of the whole concatenated sequence)
   LinearArgs a = {};
   a.A = h; a.lda = d; a.W = w->w_qkv; a.bias = w->b_qkv; a.C = qkv; a.ldc = 3 * (int64_t)d;
@@ -206,7 +240,7 @@ gsit_status gsit_im_layer_fwd(const gsit_shape* shape, const gsit_layer_weights*
   a.C = y1; a.ldc = d; a.M = M; a.N = d; a.K = d; a.out_f32 = 1; a.mask_rows = 1;
   if ((st = run_linear(g, dtype, a, cs)) != GSIT_OK) return st;
   // h = LN2(y1)
-  if ((st = from_cuda(launch_layernorm(g, y1, d, w->ln2_gamma, w->ln2_beta, eps, h, bf, cs))) != GSIT_OK) return st;
+  if ((st = run_layernorm(g, y1, d, w->ln2_gamma, w->ln2_beta, eps, h, bf, cs)) != GSIT_OK) return st;
   // f = relu(h W_1^T + b_1)
   a = LinearArgs{};
   a.A = h; a.lda = d; a.W = w->w_1; a.bias = w->b_1; a.C = f; a.ldc = w->d_ff;
@@ -240,6 +274,46 @@ gsit_status gsit_last_device_status(gsit_stream stream, uint32_t* flags) {
   if (cudaStreamSynchronize(cs) != cudaSuccess) return GSIT_ERR_CUDA;
   if (flags) *flags = host;
   return (host & GSIT_DEVFLAG_TIMEOUT) ? GSIT_ERR_TIMEOUT : GSIT_OK;
+}
+
+gsit_status gsit_trace_enable(int on) {
+  g_trace_on = (on != 0);
+  return GSIT_OK;
+}
+
+gsit_status gsit_trace_reset(void) {
+  g_trace_n = 0;
+  return GSIT_OK;
+}
+
+gsit_status gsit_trace_read(int kernel_kind, float* total_ms, int32_t* launches) {
+  if (!total_ms || !launches) return GSIT_ERR_INVALID_ARG;
+  float sum = 0.f;
+  int n = 0;
+  for (int i = 0; i < g_trace_n; ++i) {
+    if (g_trace[i].kind != kernel_kind) continue;
+    if (cudaEventSynchronize(g_trace[i].end) != cudaSuccess) return GSIT_ERR_CUDA;
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, g_trace[i].beg, g_trace[i].end) != cudaSuccess) return GSIT_ERR_CUDA;
+    sum += ms;
+    ++n;
+  }
+  *total_ms = sum;
+  *launches = n;
+  return GSIT_OK;
+}
+
+gsit_status gsit_trace_launches(int kernel_kind, float* out_ms, int32_t capacity, int32_t* launches) {
+  if (!out_ms || !launches || capacity < 0) return GSIT_ERR_INVALID_ARG;
+  int n = 0;
+  for (int i = 0; i < g_trace_n && n < capacity; ++i) {
+    if (g_trace[i].kind != kernel_kind) continue;
+    if (cudaEventSynchronize(g_trace[i].end) != cudaSuccess) return GSIT_ERR_CUDA;
+    if (cudaEventElapsedTime(&out_ms[n], g_trace[i].beg, g_trace[i].end) != cudaSuccess) return GSIT_ERR_CUDA;
+    ++n;
+  }
+  *launches = n;
+  return GSIT_OK;
 }
 
 const char* gsit_status_string(gsit_status s) {
