@@ -150,6 +150,10 @@ gsit_status gsit_trace_read(int kernel_kind, float* total_ms, int32_t* launches)
 gsit_status gsit_trace_launches(int kernel_kind, float* out_ms, int32_t capacity, int32_t* launches);
 gsit_status gsit_trace_reset(void);
 
+/* Tuning knob (host state): selects an alternative tile configuration of the bf16 attention kernel where the
+ * shape has one; 0 restores the defaults.  Results are identical up to floating-point summation order. */
+gsit_status gsit_tune_attention(int variant);
+
 const char* gsit_status_string(gsit_status status);
 int gsit_version(void);
 

@@ -40,7 +40,7 @@ class LayerWeights(ctypes.Structure):
 
 EXPORTS = ("gsit_im_qkv_proj", "gsit_im_attention_fwd", "gsit_im_layer_fwd", "gsit_workspace_bytes",
            "gsit_last_device_status", "gsit_status_string", "gsit_version", "gsit_trace_enable", "gsit_trace_read",
-           "gsit_trace_launches", "gsit_trace_reset")
+           "gsit_trace_launches", "gsit_trace_reset", "gsit_tune_attention")
 KERNEL_ATTENTION, KERNEL_LINEAR, KERNEL_LAYERNORM = 0, 1, 2
 
 
@@ -123,6 +123,10 @@ def last_device_status() -> tuple[int, int]:
     flags = ctypes.c_uint32(0)
     code = load().gsit_last_device_status(_stream(), ctypes.byref(flags))
     return int(code), int(flags.value)
+
+
+def tune_attention(variant: int):
+    _check(load().gsit_tune_attention(int(variant)), "gsit_tune_attention")
 
 
 def trace_enable(on: bool):

@@ -21,21 +21,23 @@ constexpr int STAGES = 3;
 constexpr int NTHREADS = 256;   // 8 warps
 constexpr int WAIT_SPINS = 1 << 20;
 
-template <int HD, int CW>
+// HD = head_dim, CW = features per CTA column slice, R_ = 16-row query slabs per warp, KSTEP_ = keys per softmax
+// step, MINB_ = CTAs per SM the register allocation must allow.
+template <int HD_, int CW_, int R_, int KSTEP_, int MINB_>
 struct Cfg {
+  static constexpr int HD = HD_, CW = CW_, R = R_, KSTEP = KSTEP_, MINB = MINB_;
   static constexpr int G = CW / HD;                 // heads per column slice
   static constexpr int NSG = 8 / G;                 // slab groups (warps per head)
-  static constexpr int R = (NSG >= 4) ? 1 : 4 / NSG;  // 16-row slabs per warp
   static constexpr int QT = 16 * R * NSG;           // query rows per CTA
   static constexpr int PITCH = CW * 2;              // bytes per tile row
   static constexpr int SWZ = (CW == 64) ? 7 : (CW == 32) ? 3 : 1;  // swizzle mask (128B / 64B / 32B modes)
-  static constexpr int KSTEP = (HD <= 16) ? 64 : 32;  // keys per softmax step
   static constexpr int NT = KSTEP / 8;              // score n-tiles per step
   static constexpr int KSQ = (HD == 8) ? 1 : HD / 16;  // k-steps of Q K^T
   static constexpr int NTO = HD / 8;                // output n-tiles
   static constexpr int Q_BYTES = QT * PITCH;
   static constexpr int KV_BYTES = KT * PITCH;
-  static constexpr int SMEM = Q_BYTES + 2 * STAGES * KV_BYTES + 1024 /*align slack*/ + 64 /*barriers*/;
+  static constexpr int SMEM = ((Q_BYTES + 1023) / 1024) * 1024 + 2 * STAGES * KV_BYTES + 1024 /*align slack*/ + 64 /*barriers*/;
+  static_assert(G >= 1 && G <= 8 && QT <= 256 && (KSTEP == 32 || KSTEP == 64), "unsupported tile configuration");
 };
 
 // TMA shared-memory swizzle: 16-byte chunk index bits [4, 4+B) are XORed with address bits [7, 7+B).
@@ -47,6 +49,9 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -84,12 +89,12 @@ __device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t&
 }
 __device__ __forceinline__ void mma_k16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                         uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 __device__ __forceinline__ void mma_k8(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t b0) {
-  asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};"
+  asm("mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};"
                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a0), "r"(a1), "r"(b0));
 }
 __device__ __forceinline__ float ex2(float x) {

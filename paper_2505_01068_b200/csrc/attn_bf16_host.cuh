@@ -36,10 +36,10 @@ bool make_map(CUtensorMap* tm, const void* base, int64_t rows, int d, int64_t ro
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int HD, int CW>
+template <typename C>
 cudaError_t launch_one(const Geometry& g, const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
                        int64_t row_stride, __nv_bfloat16* out, float* lse, float scale, cudaStream_t st) {
-  using C = Cfg<HD, CW>;
+  constexpr int CW = C::CW;
   const int64_t rows = (int64_t)g.batch * g.L;
   alignas(64) CUtensorMap tmQ, tmK, tmV;
   if (!make_map(&tmQ, q, rows, g.d, row_stride, CW, C::QT) || !make_map(&tmK, k, rows, g.d, row_stride, CW, KT) ||
@@ -47,7 +47,7 @@ cudaError_t launch_one(const Geometry& g, const __nv_bfloat16* q, const __nv_bfl
     return cudaErrorInvalidValue;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(attn_bf16_kernel<HD, CW>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
+    cudaError_t e = cudaFuncSetAttribute(attn_bf16_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
@@ -55,22 +55,33 @@ cudaError_t launch_one(const Geometry& g, const __nv_bfloat16* q, const __nv_bfl
   for (int s = 0; s < 3; ++s) tiles += (g.seg_len[s] + C::QT - 1) / C::QT;
   const dim3 grid((unsigned)tiles, (unsigned)(g.d / CW), (unsigned)g.batch);
   const float sl2 = scale * 1.4426950408889634f;
-  attn_bf16_kernel<HD, CW><<<grid, NTHREADS, C::SMEM, st>>>(tmQ, tmK, tmV, g, out, lse, sl2);
+  attn_bf16_kernel<C><<<grid, NTHREADS, C::SMEM, st>>>(tmQ, tmK, tmV, g, out, lse, sl2);
   return cudaGetLastError();
 }
 
 }  // namespace
+
+int g_attn_variant = 0;  // 0 = default tile configuration per shape; 1.. = alternatives (tuning knob)
 
 cudaError_t launch_attn_bf16(const Geometry& g, const __nv_bfloat16* q, const __nv_bfloat16* k,
                              const __nv_bfloat16* v, int64_t row_stride, __nv_bfloat16* out, float* lse,
                              float scale, cudaStream_t st) {
   if (g.batch > 65535 || g.d % 16 != 0) return cudaErrorNotSupported;
   const int cw = (g.d % 64 == 0) ? 64 : (g.d % 32 == 0) ? 32 : 16;
-#define GSIT_CASE(HD_, CW_) \
-  if (g.hd == HD_ && cw == CW_) return launch_one<HD_, CW_>(g, q, k, v, row_stride, out, lse, scale, st);
-  GSIT_CASE(8, 64) GSIT_CASE(16, 64) GSIT_CASE(32, 64) GSIT_CASE(64, 64)
-  GSIT_CASE(8, 32) GSIT_CASE(16, 32) GSIT_CASE(32, 32)
-  GSIT_CASE(8, 16) GSIT_CASE(16, 16)
+  const int var = g_attn_variant;
+#define GSIT_CASE(VAR_, HD_, CW_, R_, KS_, MB_)         \
+  if (g.hd == HD_ && cw == CW_ && (var == VAR_ || VAR_ == 0)) \
+    return launch_one<Cfg<HD_, CW_, R_, KS_, MB_>>(g, q, k, v, row_stride, out, lse, scale, st);
+  // alternatives first (selected only by the knob), then the defaults (VAR_ == 0 matches any knob value)
+  GSIT_CASE(1, 8, 64, 4, 64, 2) GSIT_CASE(2, 8, 64, 4, 32, 2) GSIT_CASE(3, 8, 64, 2, 64, 2)
+  GSIT_CASE(4, 8, 64, 2, 32, 3) GSIT_CASE(5, 8, 64, 2, 64, 3) GSIT_CASE(6, 8, 64, 1, 64, 3)
+  GSIT_CASE(7, 8, 64, 1, 32, 4)
+  GSIT_CASE(1, 16, 64, 2, 64, 2) GSIT_CASE(2, 16, 64, 2, 32, 2) GSIT_CASE(3, 16, 64, 1, 64, 2)
+  GSIT_CASE(4, 16, 64, 1, 32, 3)
+  GSIT_CASE(0, 8, 64, 4, 64, 2) GSIT_CASE(0, 16, 64, 2, 64, 2) GSIT_CASE(0, 32, 64, 1, 32, 2)
+  GSIT_CASE(0, 64, 64, 1, 32, 2)
+  GSIT_CASE(0, 8, 32, 2, 64, 2) GSIT_CASE(0, 16, 32, 1, 64, 2) GSIT_CASE(0, 32, 32, 1, 32, 2)
+  GSIT_CASE(0, 8, 16, 1, 64, 2) GSIT_CASE(0, 16, 16, 1, 64, 2)
 #undef GSIT_CASE
   return cudaErrorNotSupported;
 }

@@ -4,23 +4,25 @@
 namespace gsit {
 namespace {
 
-template <int HD, int CW>
-__global__ void __launch_bounds__(NTHREADS, 2)
+template <bool V> struct BoolTag { static constexpr bool value = V; };
+
+template <typename C>
+__global__ void __launch_bounds__(NTHREADS, C::MINB)
 attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, const Geometry g, __nv_bfloat16* __restrict__ out,
                  float* __restrict__ lse, const float sl2 /* scale * log2(e) */) {
-  using C = Cfg<HD, CW>;
-  constexpr int G = C::G, R = C::R, QT = C::QT, PITCH = C::PITCH, SWZ = C::SWZ, KSTEP = C::KSTEP, NT = C::NT,
-                KSQ = C::KSQ, NTO = C::NTO, CPR = CW / 8 /* 16-byte chunks per tile row */;
+  constexpr int HD = C::HD, CW = C::CW, G = C::G, R = C::R, QT = C::QT, PITCH = C::PITCH, SWZ = C::SWZ,
+                KSTEP = C::KSTEP, NT = C::NT, KSQ = C::KSQ, NTO = C::NTO, CPR = CW / 8 /* 16-byte chunks per row */;
   constexpr bool HOIST = (R > 1);  // several query slabs per warp reuse the K/V fragments of a step
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t sQ = (raw + 1023u) & ~1023u;
-  const uint32_t sK = sQ + C::Q_BYTES;
+  const uint32_t sK = sQ + ((C::Q_BYTES + 1023) / 1024) * 1024;
   const uint32_t sV = sK + STAGES * C::KV_BYTES;
-  const uint32_t bar_full = sV + STAGES * C::KV_BYTES;  // STAGES barriers, 8 bytes each
-  const uint32_t bar_q = bar_full + 8 * STAGES;
+  const uint32_t bar_full = sV + STAGES * C::KV_BYTES;  // STAGES barriers of 8 bytes: TMA bytes have landed
+  const uint32_t bar_empty = bar_full + 8 * STAGES;     // STAGES barriers: all 8 warps are done with the stage
+  const uint32_t bar_q = bar_empty + 8 * STAGES;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int head_in_slice = warp % G, sg = warp / G;
@@ -45,18 +47,19 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   const int q_real = (T > 0) ? q_real_all : 0;           // rows that receive a computed result
   const int64_t grow0 = (int64_t)b * g.L + g.seg_off[s] + q0;  // first global row of the tile
   const int xcol = cs * CW;
+  const int off1 = g.seg_off[1], off2 = g.seg_off[2];
 
-  auto locate = [&](int i, int& r, int& krem, int& yrow) {
-    int t = i;
-    r = 0;
+  auto locate = [&](int i, int& krem, int& yrow) {
+    int t = i, r = 0;
     if (t >= nk0) { t -= nk0; r = 1; if (t >= nk1) { t -= nk1; r = 2; } }
     const int kn = (r == 0) ? kn0 : (r == 1) ? kn1 : kn2;
+    const int off = (r == 0) ? 0 : (r == 1) ? off1 : off2;
     krem = kn - t * KT;
-    yrow = b * g.L + g.seg_off[r] + t * KT;
+    yrow = b * g.L + off + t * KT;
   };
   auto issue = [&](int i) {  // one thread: TMA loads of key tile i into its stage
-    int r, krem, yrow;
-    locate(i, r, krem, yrow);
+    int krem, yrow;
+    locate(i, krem, yrow);
     const int st = i % STAGES;
     mbar_expect_tx(bar_full + 8 * st, 2 * C::KV_BYTES);
     tma_load_2d(sK + st * C::KV_BYTES, &tmK, xcol, yrow, bar_full + 8 * st);
@@ -76,16 +79,20 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   if (T > 0) {
     if (tid == 0) {
 #pragma unroll
-      for (int st = 0; st < STAGES; ++st) mbar_init(bar_full + 8 * st, 1);
+      for (int st = 0; st < STAGES; ++st) {
+        mbar_init(bar_full + 8 * st, 1);
+        mbar_init(bar_empty + 8 * st, NTHREADS / 32);
+      }
       mbar_init(bar_q, 1);
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncthreads();
+    int next_issue = 0;  // meaningful in thread 0 only: next key tile to request
     if (tid == 0) {
       mbar_expect_tx(bar_q, C::Q_BYTES);
       tma_load_2d(sQ, &tmQ, xcol, (int)grow0, bar_q);
-      for (int i = 0; i < STAGES - 1 && i < T; ++i) issue(i);
+      for (; next_issue < STAGES && next_issue < T; ++next_issue) issue(next_issue);
     }
 
     // ---- query fragments, kept in registers for the whole key walk ----
@@ -108,29 +115,24 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       }
     }
 
-    for (int i = 0; i < T; ++i) {
-      const int st = i % STAGES;
-      if (tid == 0 && i + STAGES - 1 < T) issue(i + STAGES - 1);
-      mbar_wait(g, bar_full + 8 * st, (i / STAGES) & 1);
-      int r, krem, yrow;
-      locate(i, r, krem, yrow);
-      const uint32_t sKs = sK + st * C::KV_BYTES, sVs = sV + st * C::KV_BYTES;
-      if (krem < KT) {
-        // Rows past the valid length hold whatever follows in memory: clear them in V so that a zero weight
-        // times a NaN/Inf value cannot poison the accumulator (their scores are replaced by -inf below).
-        for (int idx = tid; idx < (KT - krem) * CPR; idx += NTHREADS) {
-          const uint32_t a = sVs + (krem + idx / CPR) * PITCH + (idx % CPR) * 16;
-          asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0) : "memory");
+    // One pipeline stage (KT keys) for all query slabs of this warp.  RAGGED: the stage holds fewer than KT real keys.
+    auto process = [&](auto ragged_tag, const uint32_t sKs, const uint32_t sVs, const int krem) {
+      constexpr bool RAGGED = decltype(ragged_tag)::value;
+      if constexpr (RAGGED) {
+        // Rows past the valid length hold whatever follows in memory: clear this head's part of them in V so that a
+        // zero weight times a NaN/Inf value cannot poison the accumulator (their scores become -inf below).  Warps
+        // sharing the head write the same zeros.
+        for (int idx = lane; idx < (KT - krem) * (HD / 8); idx += 32) {
+          const int row = krem + idx / (HD / 8), ch = cb + idx % (HD / 8);
+          asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(sVs + swz<SWZ>(row * PITCH + ch * 16)), "r"(0) : "memory");
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        __syncthreads();
+        __syncwarp();
       }
-
 #pragma unroll
       for (int stp = 0; stp < KT / KSTEP; ++stp) {
         const int kb = stp * KSTEP;
-        if (kb >= krem) break;
-        const bool ragged = (krem - kb) < KSTEP;
+        if (RAGGED && kb >= krem) break;
         uint32_t KF[NT][KSQ][2];
         uint32_t VF[KSTEP / 16][NTO][2];
 
@@ -201,7 +203,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             }
           }
           // ---- keys past the valid length get weight exactly zero ----
-          if (ragged) {
+          if constexpr (RAGGED) {
             const int c0 = kb + (lane & 3) * 2;
 #pragma unroll
             for (int n = 0; n < NT; ++n) {
@@ -209,13 +211,15 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
               if (c0 + n * 8 + 1 >= krem) S[n][1] = S[n][3] = -INFINITY;
             }
           }
-          // ---- online softmax (base 2, scale folded into sl2) ----
-          float mx0 = -INFINITY, mx1 = -INFINITY;
+          // ---- online softmax (base 2, scale folded into sl2); pairwise trees keep dependency chains short ----
+          float t0[NT], t1[NT];
 #pragma unroll
-          for (int n = 0; n < NT; ++n) {
-            mx0 = fmaxf(mx0, fmaxf(S[n][0], S[n][1]));
-            mx1 = fmaxf(mx1, fmaxf(S[n][2], S[n][3]));
-          }
+          for (int n = 0; n < NT; ++n) { t0[n] = fmaxf(S[n][0], S[n][1]); t1[n] = fmaxf(S[n][2], S[n][3]); }
+#pragma unroll
+          for (int w = NT / 2; w >= 1; w >>= 1)
+#pragma unroll
+            for (int n = 0; n < w; ++n) { t0[n] = fmaxf(t0[n], t0[n + w]); t1[n] = fmaxf(t1[n], t1[n + w]); }
+          float mx0 = t0[0], mx1 = t1[0];
           mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
           mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
           mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
@@ -226,18 +230,21 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           const float al0 = ex2(fmaf(m[r_][0], sl2, -ms0)), al1 = ex2(fmaf(m[r_][1], sl2, -ms1));
           m[r_][0] = mn0;
           m[r_][1] = mn1;
-          float rs0 = 0.f, rs1 = 0.f;
 #pragma unroll
           for (int n = 0; n < NT; ++n) {
             S[n][0] = ex2(fmaf(S[n][0], sl2, -ms0));
             S[n][1] = ex2(fmaf(S[n][1], sl2, -ms0));
             S[n][2] = ex2(fmaf(S[n][2], sl2, -ms1));
             S[n][3] = ex2(fmaf(S[n][3], sl2, -ms1));
-            rs0 += S[n][0] + S[n][1];
-            rs1 += S[n][2] + S[n][3];
+            t0[n] = S[n][0] + S[n][1];
+            t1[n] = S[n][2] + S[n][3];
           }
-          l[r_][0] = fmaf(l[r_][0], al0, rs0);
-          l[r_][1] = fmaf(l[r_][1], al1, rs1);
+#pragma unroll
+          for (int w = NT / 2; w >= 1; w >>= 1)
+#pragma unroll
+            for (int n = 0; n < w; ++n) { t0[n] += t0[n + w]; t1[n] += t1[n + w]; }
+          l[r_][0] = fmaf(l[r_][0], al0, t0[0]);
+          l[r_][1] = fmaf(l[r_][1], al1, t1[0]);
 #pragma unroll
           for (int n = 0; n < NTO; ++n) {
             O[r_][n][0] *= al0; O[r_][n][1] *= al0;
@@ -264,10 +271,33 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           }
         }  // slabs
       }    // steps
-      __syncthreads();  // every warp is done with this stage before it is refilled
-    }      // key tiles
+    };
 
-    // ---- normalise and stage the tile in shared memory (the Q region is free now) ----
+    for (int i = 0; i < T; ++i) {
+      const int st = i % STAGES;
+      if (tid == 0) {
+        // request further key tiles whose stage every warp has released; never block unless tile i itself is missing
+        while (next_issue < T) {
+          const uint32_t eb = bar_empty + 8 * (next_issue % STAGES);
+          const uint32_t par = ((next_issue / STAGES) - 1) & 1;
+          if (next_issue <= i) mbar_wait(g, eb, par);
+          else if (!mbar_test(eb, par)) break;
+          issue(next_issue);
+          ++next_issue;
+        }
+      }
+      __syncwarp();
+      mbar_wait(g, bar_full + 8 * st, (i / STAGES) & 1);
+      int krem, yrow;
+      locate(i, krem, yrow);
+      const uint32_t sKs = sK + st * C::KV_BYTES, sVs = sV + st * C::KV_BYTES;
+      if (krem < KT) process(BoolTag<true>{}, sKs, sVs, krem);
+      else process(BoolTag<false>{}, sKs, sVs, KT);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_empty + 8 * st);  // this warp is done with the stage
+    }
+
+    // ---- normalise and stage the tile in shared memory.  A warp overwrites only the Q bytes it alone read. ----
 #pragma unroll
     for (int r_ = 0; r_ < R; ++r_) {
       const int row0 = (sg * R + r_) * 16;

@@ -5,6 +5,7 @@
 
 namespace gsit {
 
+extern int g_attn_variant;  // attn_bf16.cu
 __device__ unsigned int g_device_status_word = 0;
 
 namespace {
@@ -326,6 +327,12 @@ const char* gsit_status_string(gsit_status s) {
     case GSIT_ERR_TIMEOUT: return "device-side wait timed out";
     default: return "unknown status";
   }
+}
+
+gsit_status gsit_tune_attention(int variant) {
+  if (variant < 0) return GSIT_ERR_INVALID_ARG;
+  g_attn_variant = variant;
+  return GSIT_OK;
 }
 
 int gsit_version(void) { return 100; }
