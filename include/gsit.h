@@ -123,6 +123,26 @@ gsit_status gsit_im_layer_fwd(const gsit_shape* shape, const gsit_layer_weights*
                               int64_t x_row_stride, float* y, int64_t y_row_stride, void* workspace,
                               size_t workspace_bytes, gsit_stream stream);
 
+/* gsit_im_layer_fwd for callers that cannot allocate device memory (no counterpart in the paper; it computes
+ * exactly what gsit_im_layer_fwd computes).  A host that lives inside someone else's memory budget, that must not
+ * risk the implicit device synchronisation of an allocation in a latency-critical loop, or that runs after its
+ * application has frozen all pools, cannot create the workspace gsit_im_layer_fwd asks for.  This variant takes
+ * none: its scratch is a fixed array of GSIT_STATIC_SCRATCH_BYTES inside the library image, held by every GPU
+ * that loads the library until the process exits.  The call itself allocates and frees nothing.
+ *   - Arguments as for gsit_im_layer_fwd, without workspace / workspace_bytes; x, y and all weights are still the
+ *     caller's device buffers.
+ *   - Limit: gsit_workspace_bytes(shape, GSIT_CALL_LAYER, d_ff) must not exceed GSIT_STATIC_SCRATCH_BYTES;
+ *     larger problems are rejected with GSIT_ERR_WORKSPACE before anything is launched (split the batch).
+ *   - The first call on each GPU looks up the array's device address (that GPU must be current); make that
+ *     first call before starting any stream capture.
+ *   - All calls on a GPU share the one array, and it keeps the previous call's intermediates.  The layer
+ *     overwrites every scratch region before reading it, so nothing needs clearing -- but two calls that
+ *     overlap in time on the same GPU (different streams, or different host threads) race on it and both
+ *     results are then undefined.  Order them on one stream or with events. */
+#define GSIT_STATIC_SCRATCH_BYTES (4u << 20)
+gsit_status gsit_im_layer_fwd_static(const gsit_shape* shape, const gsit_layer_weights* weights, const float* x,
+                                     int64_t x_row_stride, float* y, int64_t y_row_stride, gsit_stream stream);
+
 typedef enum { GSIT_CALL_QKV_PROJ = 0, GSIT_CALL_ATTENTION = 1, GSIT_CALL_LAYER = 2 } gsit_call;
 
 /* Scratch bytes the given call needs for this shape (d_ff is read for GSIT_CALL_LAYER only).

@@ -40,7 +40,8 @@ class LayerWeights(ctypes.Structure):
 
 EXPORTS = ("gsit_im_qkv_proj", "gsit_im_attention_fwd", "gsit_im_layer_fwd", "gsit_workspace_bytes",
            "gsit_last_device_status", "gsit_status_string", "gsit_version", "gsit_trace_enable", "gsit_trace_read",
-           "gsit_trace_launches", "gsit_trace_reset", "gsit_tune_attention")
+           "gsit_trace_launches", "gsit_trace_reset", "gsit_tune_attention", "gsit_im_layer_fwd_static")
+STATIC_SCRATCH_BYTES = 4 << 20
 KERNEL_ATTENTION, KERNEL_LINEAR, KERNEL_LAYERNORM = 0, 1, 2
 
 
@@ -61,6 +62,8 @@ def load():
     lib.gsit_im_attention_fwd.restype = ctypes.c_int
     lib.gsit_im_layer_fwd.argtypes = [sp, ctypes.POINTER(LayerWeights), vp, i64, vp, i64, vp, sz, vp]
     lib.gsit_im_layer_fwd.restype = ctypes.c_int
+    lib.gsit_im_layer_fwd_static.argtypes = [sp, ctypes.POINTER(LayerWeights), vp, i64, vp, i64, vp]
+    lib.gsit_im_layer_fwd_static.restype = ctypes.c_int
     lib.gsit_workspace_bytes.argtypes = [sp, ctypes.c_int, ctypes.c_int32]
     lib.gsit_workspace_bytes.restype = sz
     lib.gsit_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
@@ -206,4 +209,21 @@ def im_layer_fwd(x, weights: dict, seg_len, heads, valid_len=None, phase=PHASE_I
         workspace = torch.empty(need, dtype=torch.uint8, device=x.device)
     _check(load().gsit_im_layer_fwd(ctypes.byref(shape), ctypes.byref(lw), _ptr(x), x.stride(1), _ptr(out),
                                     out.stride(1), _ptr(workspace), workspace.numel(), _stream()), "gsit_im_layer_fwd")
+    return out
+
+
+def im_layer_fwd_static(x, weights: dict, seg_len, heads, valid_len=None, phase=PHASE_INTER_FWD, custom_mask=0,
+                        scale=0.0, ln_eps=1e-5, out=None):
+    """im_layer_fwd without a workspace: the library's built-in scratch array is used, so the call allocates no
+    device memory as long as ``out`` is given.  Problems whose scratch exceeds STATIC_SCRATCH_BYTES raise GsitError
+    (status 3).  Calls on one GPU must not overlap in time; they share the array."""
+    B, L, d = x.shape
+    assert x.is_cuda and x.dtype == torch.float32 and x.stride(2) == 1 and x.stride(0) == L * x.stride(1)
+    shape = make_shape(B, seg_len, d, heads, valid_len, _dtype_code(weights["w_qkv"].dtype), phase, custom_mask, scale)
+    lw = make_layer_weights(weights, ln_eps)
+    if out is None:
+        out = torch.empty((B, L, d), dtype=torch.float32, device=x.device)
+    assert out.stride(2) == 1 and out.stride(0) == L * out.stride(1)
+    _check(load().gsit_im_layer_fwd_static(ctypes.byref(shape), ctypes.byref(lw), _ptr(x), x.stride(1), _ptr(out),
+                                           out.stride(1), _stream()), "gsit_im_layer_fwd_static")
     return out
