@@ -4,38 +4,6 @@
 namespace gsit {
 namespace {
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_tiled_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (fn == nullptr) {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
-        qres == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(p);
-  }
-  return fn;
-}
-
-// 2-D map over a [rows, d] bf16 view with row pitch `row_stride` elements; box = [CW columns, box_rows rows],
-// shared-memory swizzle matched to the box width.  Out-of-range rows read as zero.
-bool make_map(CUtensorMap* tm, const void* base, int64_t rows, int d, int64_t row_stride, int cw, int box_rows) {
-  EncodeTiledFn fn = encode_tiled_fn();
-  if (fn == nullptr) return false;
-  const cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
-  const cuuint64_t strides[1] = {(cuuint64_t)row_stride * 2};
-  const cuuint32_t box[2] = {(cuuint32_t)cw, (cuuint32_t)box_rows};
-  const cuuint32_t estr[2] = {1, 1};
-  const CUtensorMapSwizzle sw = (cw == 64) ? CU_TENSOR_MAP_SWIZZLE_128B
-                                : (cw == 32) ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
-  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 template <typename C>
 cudaError_t launch_one(const Geometry& g, const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
                        int64_t row_stride, __nv_bfloat16* out, float* lse, float scale, cudaStream_t st) {
@@ -69,6 +37,8 @@ cudaError_t launch_attn_bf16(const Geometry& g, const __nv_bfloat16* q, const __
   if (g.batch > 65535 || g.d % 16 != 0) return cudaErrorNotSupported;
   const int cw = (g.d % 64 == 0) ? 64 : (g.d % 32 == 0) ? 32 : 16;
   const int var = g_attn_variant;
+  // head_dim 64 is a dense contraction: tcgen05 / TMEM kernel (variant 9 keeps the mma.sync kernel for comparison)
+  if (g.hd == 64 && var != 9) return launch_attn_tc_hd64(g, q, k, v, row_stride, out, lse, scale, st);
 #define GSIT_CASE(VAR_, HD_, CW_, R_, KS_, MB_)         \
   if (g.hd == HD_ && cw == CW_ && (var == VAR_ || VAR_ == 0)) \
     return launch_one<Cfg<HD_, CW_, R_, KS_, MB_>>(g, q, k, v, row_stride, out, lse, scale, st);

@@ -58,6 +58,11 @@ cudaError_t launch_attn_bf16(const Geometry& g, const __nv_bfloat16* q, const __
                              const __nv_bfloat16* v, int64_t row_stride, __nv_bfloat16* out, float* lse,
                              float scale, cudaStream_t st);
 
+// bf16 attention for head_dim 64 on tcgen05 tensor cores with TMEM accumulators (attn_tc.cu)
+cudaError_t launch_attn_tc_hd64(const Geometry& g, const __nv_bfloat16* q, const __nv_bfloat16* k,
+                                const __nv_bfloat16* v, int64_t row_stride, __nv_bfloat16* out, float* lse,
+                                float scale, cudaStream_t st);
+
 // Linear layers  C = act(A W^T + bias) (+ residual), rows that are padding written as zero when
 // `mask_rows` is set.  A [M,K] (lda), W [N,K], C [M,N] (ldc), residual float [M,N] (ldr) or nullptr.
 struct LinearArgs {
