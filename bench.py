@@ -4,7 +4,7 @@
 A step is one forward pass of the whole hot path over one batch: the GsiT fusion stack (forward-ring and
 backward-ring encoders at width d, intra-modal encoder at width 2d), every layer being LayerNorm -> shared
 QKV projection -> IM attention -> out-projection + residual -> LayerNorm -> MLP + residual, all inside the
-library's kernels.  `value` is valid (non padded) tokens per second with inputs resident in HBM; `e2e`
+library's kernels (three launches per layer).  `value` is valid (non padded) tokens per second with inputs resident in HBM; `e2e`
 includes the host->device copy of the batch and the device->host copy of the result every step.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload 4|5]
@@ -222,7 +222,7 @@ def run_gpu(args):
     x_host = torch.from_numpy(inp["x"]).pin_memory()
     nbuf = max(2, int(np.ceil(1.2 * L2_BYTES / x_host.numel() / 4)))
     xbufs = [x_host.cuda() for _ in range(nbuf)]
-    launches_per_step = 7 * (n_f + n_b + n_i)
+    launches_per_step = 3 * (n_f + n_b + n_i)   # per layer: LN1+QKV, IM attention, out-proj+LN2+MLP (fused kernels)
 
     for i in range(max(1, min(args.warmup, 2))):           # eager warm-up (module load, attributes, buffers)
         stack.forward(xbufs[i % nbuf], vl)

@@ -79,6 +79,17 @@ struct LinearArgs {
 cudaError_t launch_linear_f32(const Geometry& g, const LinearArgs& a, cudaStream_t st);
 cudaError_t launch_linear_bf16(const Geometry& g, const LinearArgs& a, cudaStream_t st);
 
+// Fused halves of the layer for bf16 at d_model 64 / 128 with d_ff a multiple of 64 (fused_layer.cu):
+//   qkv = LN1(x) W_qkv^T + b_qkv, and  y = y1 + relu(LN2(y1) W_1^T + b_1) W_2^T + b_2 with y1 = x + att W_o^T + b_o.
+bool fused_layer_supported(const Geometry& g, int d_ff);
+cudaError_t launch_ln_qkv_bf16(const Geometry& g, const float* x, int64_t ldx, const float* gamma, const float* beta,
+                               float eps, const __nv_bfloat16* w_qkv, const float* b_qkv, __nv_bfloat16* qkv,
+                               cudaStream_t st);
+cudaError_t launch_proj_mlp_bf16(const Geometry& g, const __nv_bfloat16* att, const float* x, int64_t ldx,
+                                 const __nv_bfloat16* w_o, const float* b_o, const float* gamma, const float* beta, float eps,
+                                 const __nv_bfloat16* w_1, const float* b_1, const __nv_bfloat16* w_2, const float* b_2,
+                                 int d_ff, float* y, int64_t ldy, cudaStream_t st);
+
 // Row LayerNorm of float x (row stride ldx) into float or bf16 y [rows, d]; padded rows become zero.
 cudaError_t launch_layernorm(const Geometry& g, const float* x, int64_t ldx, const float* gamma, const float* beta,
                              float eps, void* y, int out_bf16, cudaStream_t st);

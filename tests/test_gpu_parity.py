@@ -142,3 +142,26 @@ def test_cfg5_scaled_hd64_bf16(g):
     ref = oracle.qkv_proj(x, w, None, wl.seg_len, wl.heads, valid[:2])
     check_close(to_np64(qkv).reshape(2, wl.L, -1), ref.reshape(2, wl.L, -1), "bf16", pad_mask(wl.seg_len, valid[:2], 2),
                 "qkv_proj d=512")
+
+
+@pytest.mark.parametrize("d,heads,d_ff,seg,B", [(64, 8, 256, (50, 170, 93), 3), (128, 8, 512, (37, 150, 64), 2),
+                                                (64, 4, 64, (50, 30, 90), 2), (64, 8, 128, (5, 0, 9), 3),
+                                                (32, 4, 128, (40, 33, 20), 2)])
+def test_layer_bf16_affine_biases_ragged(g, d, heads, d_ff, seg, B):
+    """One IM layer with LayerNorm affine parameters and every bias set, ragged valid lengths, NaN in the padded input
+    rows and a row count that is not a multiple of any tile: d = 64 / 128 take the fused kernels, d = 32 the separate
+    LayerNorm / linear kernels."""
+    rng = np.random.default_rng(d * 1000 + d_ff)
+    x = rng.standard_normal((B, sum(seg), d), dtype=np.float32)
+    w = wk.draw_layer_weights(rng, d, d_ff, "bf16", affine=True)
+    valid = np.stack([rng.integers(0, s + 1, size=B) for s in seg], axis=1).astype(np.int32)
+    valid[0] = seg
+    pm = pad_mask(seg, valid, B)
+    xd = to_dev(wk.fill_padding(x, seg, valid, np.nan))
+    vl = torch.from_numpy(valid).cuda()
+    for ph in PHASES:
+        y = g.im_layer_fwd(xd, weights_to_dev(w, "bf16"), seg, heads, vl, ph)
+        ref = oracle.im_layer_fwd(x, w, seg, heads, valid, ph)
+        check_close(to_np64(y), ref, "bf16", pm, f"affine layer d={d} phase {ph}")
+    code, flags = g.last_device_status()
+    assert code == 0 and flags == 0
