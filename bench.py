@@ -30,6 +30,9 @@ METRIC = "IM-attention tokens/s (valid tokens through the GsiT IM stack), MOSEI-
 UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 L2_BYTES = 126 * 1024 * 1024
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the cross-modal attention kernel at this workload
+# (ncu capture summarised in profiles/attn_bf16_hd8_cfg4_cross.md; the kernel has not changed since)
+ATTN_HD8_DRAM_BYTES = 21.43e6
 
 
 def peaks():
@@ -164,7 +167,7 @@ def _time_graph_replays(torch, graphs, steps, dist, world):
 
 def time_attention_alone(torch, g, wl, valid_dev, d, heads, phase, reps=4):
     """One IM-attention call timed alone: a CUDA graph of launches rotating over qkv/out buffer sets larger than L2."""
-    B, L = valid_dev.shape[0], wl.L
+    B, L = (wl.batch if valid_dev is None else valid_dev.shape[0]), wl.L
     set_bytes = B * L * 4 * d * 2
     nsets = max(2, int(np.ceil(1.5 * L2_BYTES / set_bytes)))
     gen = torch.Generator(device="cuda").manual_seed(1234)
@@ -306,6 +309,24 @@ def run_gpu(args):
                            "t_hbm_us": t_hbm * 1e6, "t_exp_us": t_exp * 1e6, "d_model": d, "heads": heads,
                            "buffer_sets": nsets, "in_step_us": (cross_s if name == "cross" else intra_s) * 1e6}
 
+    # ---- the scaled shape (head_dim 64, tcgen05 kernel), attention alone: context for the tensor-bound case ----
+    scaled = {}
+    if not args.no_scaled:
+        wl5 = wk.WORKLOADS[5]
+        v5 = wk.draw_valid_len(np.random.default_rng(wl5.seed), wl5)
+        vl5 = torch.from_numpy(v5).cuda()
+        tok5 = int(v5.sum())
+        for name, phase, allowed in (("cross", g.PHASE_INTER_FWD, [[0, 1, 0], [0, 0, 1], [1, 0, 0]]), ("intra", g.PHASE_INTRA, np.eye(3, dtype=int))):
+            sec, nsets = time_attention_alone(torch, g, wl5, vl5, wl5.d_model, wl5.heads, phase, reps=1)
+            U = wk.useful_pairs(wl5.seg_len, v5, allowed, wl5.batch)
+            fl, by = 4.0 * wl5.d_model * U, 4.0 * tok5 * wl5.d_model * 2
+            t_tc, t_hbm = fl / (pk["bf16_tflops"] * 1e12), by / (pk["hbm_gbs"] * 1e9)
+            scaled[name] = {"us": sec * 1e6, "tokens_per_s": tok5 / sec, "useful_tflops": fl / sec / 1e12,
+                            "frac_roofline": max(t_tc, t_hbm) / sec, "t_tensor_us": t_tc * 1e6, "t_hbm_us": t_hbm * 1e6,
+                            "t_exp_us": wl5.heads * U / ex2_rate * 1e6, "batch": wl5.batch, "buffer_sets": nsets}
+        del vl5
+        torch.cuda.empty_cache()
+
     # ---- CPU baseline: the oracle on a bounded sample of the same workload ----
     import oracle
     sub = args.ref_batch
@@ -335,11 +356,12 @@ def run_gpu(args):
         "gpu_launches": launches_per_step * args.steps,
         "roofline": {"kernel": "attn_bf16_kernel<8,64> (cross-modal IM attention inside the step)", "bound": "hbm",
                      "achieved": cross["bytes"] / cross_s / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s",
-                     "frac": cross["bytes"] / cross_s / 1e9 / pk["hbm_gbs"], "traffic": None, "peak_kind": "of " + pk_kind,
+                     "frac": cross["bytes"] / cross_s / 1e9 / pk["hbm_gbs"], "traffic": ATTN_HD8_DRAM_BYTES, "peak_kind": "of " + pk_kind,
                      "launch_us": cross_s * 1e6, "algorithmic_bytes": cross["bytes"]},
         "cpu_baseline": {"value": ref_tokens / cpu_s, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
                          "sample": f"{sub} of {B} samples, one step (valid tokens {ref_tokens}) in {cpu_s:.2f} s"},
         "attention": attention,
+        "scaled_attention_hd64": scaled,
         "step_kernel_ms": {"attention": float(att.sum()) / trace_steps, "linear": lin_ms / trace_steps,
                            "layernorm": ln_ms / trace_steps, "launches": {"attention": per_step, "linear": lin_n // trace_steps,
                                                                           "layernorm": ln_n // trace_steps}},
@@ -357,6 +379,7 @@ def main():
     ap.add_argument("--impl", default="gsit", choices=["gsit", "reference"])
     ap.add_argument("--workload", type=int, default=4)
     ap.add_argument("--ref-batch", type=int, default=16, help="samples per step of the CPU oracle")
+    ap.add_argument("--no-scaled", action="store_true", help="skip the extra timing of the head_dim-64 attention")
     args = ap.parse_args()
     if args.impl == "reference":
         args.steps = 2 if args.steps is None else args.steps
