@@ -324,7 +324,25 @@ def run_gpu(args):
             scaled[name] = {"us": sec * 1e6, "tokens_per_s": tok5 / sec, "useful_tflops": fl / sec / 1e12,
                             "frac_roofline": max(t_tc, t_hbm) / sec, "t_tensor_us": t_tc * 1e6, "t_hbm_us": t_hbm * 1e6,
                             "t_exp_us": wl5.heads * U / ex2_rate * 1e6, "batch": wl5.batch, "buffer_sets": nsets}
-        del vl5
+        # the shared QKV projection at the same shape (tcgen05 GEMM, d=512): x [B, L, 512] -> qkv [B, L, 3, 8, 64]
+        xs5 = [torch.randn((wl5.batch, wl5.L, wl5.d_model), device="cuda").bfloat16() for _ in range(2)]
+        w5 = (torch.randn((3 * wl5.d_model, wl5.d_model), device="cuda") * wl5.d_model ** -0.5).bfloat16()
+        qs5 = [torch.empty((wl5.batch, wl5.L, 3, wl5.heads, wl5.d_model // wl5.heads), device="cuda", dtype=torch.bfloat16) for _ in range(2)]
+        for i in range(2):
+            g.im_qkv_proj(xs5[i], w5, None, wl5.seg_len, wl5.heads, vl5, out=qs5[i])
+        torch.cuda.synchronize()
+        beg, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        beg.record()
+        for _ in range(5):
+            for i in range(2):
+                g.im_qkv_proj(xs5[i], w5, None, wl5.seg_len, wl5.heads, vl5, out=qs5[i])
+        end.record()
+        torch.cuda.synchronize()
+        sec = beg.elapsed_time(end) * 1e-3 / 10
+        fl = 2.0 * wl5.batch * wl5.L * wl5.d_model * 3 * wl5.d_model
+        scaled["qkv_proj"] = {"us": sec * 1e6, "tflops": fl / sec / 1e12, "frac_tensor_peak": fl / sec / 1e12 / pk["bf16_tflops"],
+                              "note": "all B*L rows multiplied (padded rows are zeroed in the epilogue)"}
+        del vl5, xs5, qs5
         torch.cuda.empty_cache()
 
     # ---- CPU baseline: the oracle on a bounded sample of the same workload ----

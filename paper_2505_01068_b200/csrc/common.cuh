@@ -77,6 +77,9 @@ struct LinearArgs {
   int mask_rows;    // zero the padded rows of C (uses geometry)
 };
 cudaError_t launch_linear_f32(const Geometry& g, const LinearArgs& a, cudaStream_t st);
+// bf16 linear layer on tcgen05 tensor cores with TMEM accumulators (gemm_tc.cu): K a multiple of 64, N a multiple of 8
+bool linear_tc_supported(const LinearArgs& a);
+cudaError_t launch_linear_tc_bf16(const Geometry& g, const LinearArgs& a, cudaStream_t st);
 cudaError_t launch_linear_bf16(const Geometry& g, const LinearArgs& a, cudaStream_t st);
 
 // Fused halves of the layer for bf16 at d_model 64 / 128 with d_ff a multiple of 64 (fused_layer.cu):

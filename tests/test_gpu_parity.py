@@ -146,11 +146,12 @@ def test_cfg5_scaled_hd64_bf16(g):
 
 @pytest.mark.parametrize("d,heads,d_ff,seg,B", [(64, 8, 256, (50, 170, 93), 3), (128, 8, 512, (37, 150, 64), 2),
                                                 (64, 4, 64, (50, 30, 90), 2), (64, 8, 128, (5, 0, 9), 3),
-                                                (32, 4, 128, (40, 33, 20), 2)])
+                                                (32, 4, 128, (40, 33, 20), 2), (192, 3, 768, (70, 129, 33), 2)])
 def test_layer_bf16_affine_biases_ragged(g, d, heads, d_ff, seg, B):
     """One IM layer with LayerNorm affine parameters and every bias set, ragged valid lengths, NaN in the padded input
     rows and a row count that is not a multiple of any tile: d = 64 / 128 take the fused kernels, d = 32 the separate
-    LayerNorm / linear kernels."""
+    LayerNorm / mma.sync linear kernels, d = 192 the separate kernels with every linear layer on the tcgen05 GEMM (bias,
+    ReLU, float output with residual, TMA-stored bf16 output)."""
     rng = np.random.default_rng(d * 1000 + d_ff)
     x = rng.standard_normal((B, sum(seg), d), dtype=np.float32)
     w = wk.draw_layer_weights(rng, d, d_ff, "bf16", affine=True)
@@ -163,5 +164,31 @@ def test_layer_bf16_affine_biases_ragged(g, d, heads, d_ff, seg, B):
         y = g.im_layer_fwd(xd, weights_to_dev(w, "bf16"), seg, heads, vl, ph)
         ref = oracle.im_layer_fwd(x, w, seg, heads, valid, ph)
         check_close(to_np64(y), ref, "bf16", pm, f"affine layer d={d} phase {ph}")
+    code, flags = g.last_device_status()
+    assert code == 0 and flags == 0
+
+
+def test_qkv_proj_tcgen05_matches_mma_sync_kernel(g):
+    """The shared projection through the tcgen05 GEMM and through the mma.sync kernel (tuning knob 9) on the same inputs:
+    both within the bf16 tolerance of the oracle, and within rounding of each other."""
+    rng = np.random.default_rng(31)
+    seg, B, d, H = (37, 300, 129), 3, 256, 4
+    x = wk.storage_round(rng.standard_normal((B, sum(seg), d), dtype=np.float32), "bf16")
+    w = wk.draw_layer_weights(rng, d, 4 * d, "bf16", affine=True)
+    valid = np.array([[37, 300, 129], [1, 150, 0], [20, 299, 64]], dtype=np.int32)
+    vl = torch.from_numpy(valid).cuda()
+    xd = to_dev(wk.fill_padding(x, seg, valid, np.nan), "bf16")
+    wd, bd = to_dev(w["w_qkv"], "bf16"), to_dev(w["b_qkv"])
+    new = to_np64(g.im_qkv_proj(xd, wd, bd, seg, H, vl)).reshape(B, sum(seg), -1)
+    g.tune_attention(9)
+    try:
+        old = to_np64(g.im_qkv_proj(xd, wd, bd, seg, H, vl)).reshape(B, sum(seg), -1)
+    finally:
+        g.tune_attention(0)
+    ref = oracle.qkv_proj(x, w["w_qkv"], w["b_qkv"], seg, H, valid).reshape(B, sum(seg), -1)
+    pm = pad_mask(seg, valid, B)
+    check_close(new, ref, "bf16", pm, "tcgen05 projection")
+    check_close(old, ref, "bf16", pm, "mma.sync projection")
+    assert np.abs(new - old).max() <= 2.0 ** -6
     code, flags = g.last_device_status()
     assert code == 0 and flags == 0
