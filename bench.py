@@ -199,6 +199,7 @@ def run_gpu(args):
     import torch.distributed as dist
 
     import paper_2505_01068_b200 as g
+    from paper_2505_01068_b200 import shard
 
     rank, world = int(os.environ.get("RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
     local = int(os.environ.get("LOCAL_RANK", 0))
@@ -210,7 +211,7 @@ def run_gpu(args):
     assert wl.stack is not None, "the benchmark step is the full stack (workload 4)"
     n_f, n_b, n_i, ih = wl.stack
     # weak scaling: every rank owns an independent batch of the same shape (no data-path collective)
-    inp = wk.make_inputs(wl.index, seed=wl.seed + 1000 * rank)
+    inp = wk.make_inputs(wl.index, seed=shard.rank_seed(wl.seed, rank))
     B = wl.batch
     valid = inp["valid_len"]
     vl = torch.from_numpy(valid).cuda()
@@ -245,11 +246,8 @@ def run_gpu(args):
     with ClockSampler(local) as clocks:
         ms = _time_graph_replays(torch, graphs, args.steps, dist, world)
     ms_per_step = ms / args.steps
-    value = tokens * world / (ms_per_step * 1e-3)
-    if world > 1:
-        tt = torch.tensor([float(tokens)], device="cuda")
-        dist.all_reduce(tt)
-        value = float(tt.item()) / (ms_per_step * 1e-3)
+    # whole job: tokens of all ranks over the slowest rank's time (ms is already the maximum over ranks)
+    _, _, value = shard.job_throughput(tokens, ms_per_step, device="cuda")
 
     # ---- end to end: pinned host batch -> device -> stack -> host, every step ----
     y_host = torch.empty(tuple(y_dev.shape), dtype=torch.float32).pin_memory()
@@ -269,10 +267,7 @@ def run_gpu(args):
     for _ in range(e2e_steps):
         e2e_step()
     torch.cuda.synchronize()
-    e2e_s = torch.tensor([(time.perf_counter() - t0) / e2e_steps], device="cuda")
-    if world > 1:
-        dist.all_reduce(e2e_s, op=dist.ReduceOp.MAX)
-    e2e_value = tokens * world / float(e2e_s.item())
+    _, _, e2e_value = shard.job_throughput(tokens, (time.perf_counter() - t0) / e2e_steps * 1e3, device="cuda")
 
     # ---- per-kernel device times inside the step (eager, CUDA events around each launch) ----
     trace_steps = max(1, min(args.steps, 10))
