@@ -1,0 +1,636 @@
+// The two fused halves of the IM encoder layer at d_model 64 on the 5th-generation tensor cores (tcgen05 / TMEM):
+//
+//   ln_qkv_tc_kernel     qkv = LN1(x) W_qkv^T + b_qkv          (the shared projection of the concatenated sequence)
+//   proj_mlp_tc_kernel   y1 = x + att W_o^T + b_o ;  y = y1 + relu(LN2(y1) W_1^T + b_1) W_2^T + b_2   (d_ff <= 256)
+//
+// Persistent, one CTA per SM, tiles of 128 sequence rows, six warps:
+//   warp 0      producer: weights once (TMA, 128-byte swizzle, resident for the whole kernel), then per tile the x rows
+//               (per-row bulk copies into padded float rows) and the attention tile (TMA)
+//   warp 1      owns 512 TMEM columns and issues every tcgen05.mma (M 128, K 16, operands from shared memory)
+//   warps 2..5  thread = sequence row = TMEM lane.  LayerNorm needs no shuffles: a thread holds its whole row.  Rows
+//               are written back to shared memory as bf16 in the 128-byte swizzle the MMA expects (the A operand of the
+//               next product), so the normalised rows, the float residual y1 (registers) and the 256 hidden units per
+//               row never leave the SM.  Outputs leave through swizzled staging rows and TMA stores.
+// Every wait is bounded (GSIT_DEVFLAG_TIMEOUT instead of a hang) and TMEM is always released.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "tensor_map.cuh"
+#include "tmem_ldst.cuh"
+
+namespace gsit {
+namespace {
+
+constexpr int TD = 64;            // d_model
+constexpr int TM = 128;           // rows per tile
+constexpr int T_THREADS = 192;
+constexpr int T_SPIN = 1 << 16;
+constexpr int XBOX = TM * 128;     // a float input tile is two TMA boxes of 32 columns x 128 rows (128-byte rows, swizzled)
+
+__device__ __forceinline__ void t_mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void t_mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void t_mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void t_mbar_wait(const Geometry& g, uint32_t bar, uint32_t parity) {
+  for (int it = 0; it < T_SPIN; ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    if (ok) return;
+    if ((it & 63) == 63 && (*reinterpret_cast<volatile unsigned int*>(g.status) & GSIT_DEVFLAG_TIMEOUT)) return;
+  }
+  raise_flag(g, GSIT_DEVFLAG_TIMEOUT);
+}
+__device__ __forceinline__ void t_tma_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void t_tma_store_2d(const CUtensorMap* tm, uint32_t src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(src) : "memory");
+}
+__device__ __forceinline__ bool t_elect() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
+}
+// K-major operand tile with 128-byte rows and 128-byte swizzle: 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t t_desc(uint32_t addr) {
+  return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+__host__ __device__ constexpr uint32_t t_idesc(int n) {  // D = f32, A = B = bf16 K-major, M = 128, N = n
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+__device__ __forceinline__ void t_umma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void t_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void t_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void t_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void t_fence_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void t_bar_rows() { asm volatile("bar.sync 1, 128;" ::: "memory"); }  // the four row warps
+__device__ __forceinline__ uint32_t t_bf2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+// 16-byte chunk `ch` (0..7) of row r in a tile of 128-byte rows with the 128-byte swizzle.
+__device__ __forceinline__ uint32_t sw128(uint32_t tile, int r, int ch) { return tile + r * 128 + ((ch ^ (r & 7)) << 4); }
+__device__ __forceinline__ void st_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
+__device__ __forceinline__ float4 ld_v4f(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+  return v;
+}
+// Reads the thread's float row r (64 values) from a two-box swizzled float tile.
+__device__ __forceinline__ void load_row64(uint32_t tile, int r, float (&v)[TD]) {
+#pragma unroll
+  for (int j = 0; j < 2; ++j)
+#pragma unroll
+    for (int ch = 0; ch < 8; ++ch) {
+      const float4 t = ld_v4f(sw128(tile + j * XBOX, r, ch));
+      const int e = 32 * j + 4 * ch;
+      v[e] = t.x; v[e + 1] = t.y; v[e + 2] = t.z; v[e + 3] = t.w;
+    }
+}
+// Copies n floats of a per-feature vector into shared memory (or `fill` when the pointer is null): vectors such as
+// gamma, beta and the biases are read by every thread for every row, as 16-byte broadcasts.
+__device__ __forceinline__ void stage_vector(float* dst, const float* src, int n, float fill, int tid, int nthreads) {
+  for (int i = tid; i < n; i += nthreads) dst[i] = (src != nullptr) ? src[i] : fill;
+}
+// Row validity with 32-bit arithmetic (the library limits B * L to 2^29).
+__device__ __forceinline__ bool row_real32(const Geometry& g, int row, int rows) {
+  if (row >= rows) return false;
+  const int b = row / g.L, p = row - b * g.L;
+  const int sgm = segment_of(g, p);
+  return (p - g.seg_off[sgm]) < valid_rows(g, b, sgm);
+}
+// LayerNorm of one row held by one thread -> bf16 row r of a swizzled 128-byte-row tile (zeros when !real).
+__device__ __forceinline__ void layernorm_row_to_tile(const float (&v)[TD], bool real, uint32_t s_gamma, uint32_t s_beta,
+                                                      float eps, uint32_t tile, int r) {
+  float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+  for (int e = 0; e < TD; e += 4) { s0 += v[e]; s1 += v[e + 1]; s2 += v[e + 2]; s3 += v[e + 3]; }
+  const float mean = ((s0 + s1) + (s2 + s3)) * (1.f / TD);
+  float q0 = 0.f, q1 = 0.f, q2 = 0.f, q3 = 0.f;
+#pragma unroll
+  for (int e = 0; e < TD; e += 4) {
+    const float a = v[e] - mean, b = v[e + 1] - mean, c = v[e + 2] - mean, d = v[e + 3] - mean;
+    q0 = fmaf(a, a, q0); q1 = fmaf(b, b, q1); q2 = fmaf(c, c, q2); q3 = fmaf(d, d, q3);
+  }
+  const float rstd = real ? rsqrtf(((q0 + q1) + (q2 + q3)) * (1.f / TD) + eps) : 0.f;
+#pragma unroll
+  for (int ch = 0; ch < 8; ++ch) {
+    const float4 g0 = ld_v4f(s_gamma + ch * 32), g1 = ld_v4f(s_gamma + ch * 32 + 16);
+    const float4 b0 = ld_v4f(s_beta + ch * 32), b1 = ld_v4f(s_beta + ch * 32 + 16);
+    const float gm[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+    const float bt[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+    uint32_t pk[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int e = ch * 8 + 2 * k;
+      float a = fmaf((v[e] - mean) * rstd, gm[2 * k], bt[2 * k]), b = fmaf((v[e + 1] - mean) * rstd, gm[2 * k + 1], bt[2 * k + 1]);
+      if (!real) { a = 0.f; b = 0.f; }
+      pk[k] = t_bf2(a, b);
+    }
+    st_v4(sw128(tile, r, ch), pk[0], pk[1], pk[2], pk[3]);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------ LN1 + shared QKV
+namespace qk {
+constexpr int NQ = 3 * TD;                       // 192 output columns
+constexpr int OFF_W = 0;                         // W_qkv: 192 rows x 128 B, swizzled
+constexpr int OFF_H = OFF_W + NQ * 128;          // normalised rows (A operand)
+constexpr int OFF_OUT = OFF_H + TM * 128;        // 3 boxes of 64 columns x 128 rows
+constexpr int OFF_X = OFF_OUT + 3 * TM * 128;    // 2 float input tiles (2 boxes each)
+constexpr int OFF_P = OFF_X + 2 * 2 * XBOX;      // gamma[64], beta[64], bias[192] as floats
+constexpr int OFF_BAR = OFF_P + (2 * TD + NQ) * 4;
+constexpr int B_W = 0, B_XFULL = 8, B_XFREE = 24, B_HREADY = 40, B_ACCFULL = 48, B_ACCFREE = 56, SLOT = 64;
+constexpr int SMEM = OFF_BAR + 80 + 1024;
+constexpr int TMEM_COLS = 256;
+}  // namespace qk
+
+__global__ void __launch_bounds__(T_THREADS, 1)
+ln_qkv_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
+                 const __grid_constant__ CUtensorMap tmOut, const Geometry g, const float* __restrict__ gamma,
+                 const float* __restrict__ beta, const float eps, const float* __restrict__ bias) {
+  using namespace qk;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t bars = base + OFF_BAR;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int rows = g.batch * g.L;
+  const int ntiles = (rows + TM - 1) / TM;
+
+  float* prm = reinterpret_cast<float*>(base_ptr + OFF_P);
+  stage_vector(prm, gamma, TD, 1.f, tid, T_THREADS);
+  stage_vector(prm + TD, beta, TD, 0.f, tid, T_THREADS);
+  stage_vector(prm + 2 * TD, bias, NQ, 0.f, tid, T_THREADS);
+  if (tid == 0) {
+    t_mbar_init(bars + B_W, 1);
+    for (int i = 0; i < 2; ++i) { t_mbar_init(bars + B_XFULL + 8 * i, 1); t_mbar_init(bars + B_XFREE + 8 * i, 4); }
+    t_mbar_init(bars + B_HREADY, 4);
+    t_mbar_init(bars + B_ACCFULL, 1);
+    t_mbar_init(bars + B_ACCFREE, 4);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    t_fence_async();
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(bars + SLOT), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  t_fence_before();
+  __syncthreads();
+  t_fence_after();
+  uint32_t tmem;
+  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tmem) : "r"(bars + SLOT) : "memory");
+
+  if (warp == 0) {
+    // ================================ producer ================================
+    if (t_elect()) {
+      t_mbar_expect_tx(bars + B_W, NQ * 128);
+      t_tma_2d(base + OFF_W, &tmW, 0, 0, bars + B_W);
+    }
+    __syncwarp();
+    int i = 0;
+    for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
+      const int xb = i & 1;
+      if (i >= 2) t_mbar_wait(g, bars + B_XFREE + 8 * xb, ((i >> 1) - 1) & 1);  // the row warps hold that tile in registers
+      if (t_elect()) {
+        t_mbar_expect_tx(bars + B_XFULL + 8 * xb, 2 * XBOX);
+        t_tma_2d(base + OFF_X + xb * 2 * XBOX, &tmX, 0, t * TM, bars + B_XFULL + 8 * xb);
+        t_tma_2d(base + OFF_X + xb * 2 * XBOX + XBOX, &tmX, 32, t * TM, bars + B_XFULL + 8 * xb);
+      }
+      __syncwarp();
+    }
+  } else if (warp == 1) {
+    // ================================ MMA issuer ================================
+    constexpr uint32_t IDESC = t_idesc(NQ);
+    t_mbar_wait(g, bars + B_W, 0);
+    int i = 0;
+    for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
+      t_mbar_wait(g, bars + B_HREADY, i & 1);
+      if (i > 0) t_mbar_wait(g, bars + B_ACCFREE, (i - 1) & 1);
+      t_fence_after();
+      if (t_elect()) {
+#pragma unroll
+        for (int k = 0; k < TD / 16; ++k)
+          t_umma(tmem, t_desc(base + OFF_H + 32 * k), t_desc(base + OFF_W + 32 * k), IDESC, k > 0);
+        t_commit(bars + B_ACCFULL);
+      }
+      __syncwarp();
+    }
+  } else {
+    // ================================ one thread per sequence row ================================
+    const int r = ((warp & 3) << 5) + lane;
+    const uint32_t tl = tmem + ((uint32_t)((warp & 3) << 5) << 16);
+    const uint32_t s_gamma = base + OFF_P, s_beta = s_gamma + TD * 4, s_bias = s_beta + TD * 4;
+    int i = 0;
+    bool real = row_real32(g, (int)blockIdx.x * TM + r, rows);
+    for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
+      const int row0 = t * TM, xb = i & 1;
+      t_mbar_wait(g, bars + B_XFULL + 8 * xb, (i >> 1) & 1);
+      float v[TD];
+      if (real) {
+        load_row64(base + OFF_X + xb * 2 * XBOX, r, v);
+      } else {  // padded input rows may hold anything (NaN included): never read them
+#pragma unroll
+        for (int e = 0; e < TD; ++e) v[e] = 0.f;
+      }
+      __syncwarp();
+      if (lane == 0) t_mbar_arrive(bars + B_XFREE + 8 * xb);
+      // the MMA of the previous tile finished reading the normalised rows before its accumulator was handed over
+      layernorm_row_to_tile(v, real, s_gamma, s_beta, eps, base + OFF_H, r);
+      t_fence_async();
+      __syncwarp();
+      if (lane == 0) t_mbar_arrive(bars + B_HREADY);
+      const bool real_next = row_real32(g, (t + (int)gridDim.x) * TM + r, rows);  // overlaps the MMA
+
+      t_mbar_wait(g, bars + B_ACCFULL, i & 1);
+      t_fence_after();
+      if (i > 0) {  // the previous tile's stores must have finished reading the staging rows
+        if (tid == 64) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        t_bar_rows();
+      }
+#pragma unroll 1
+      for (int c0 = 0; c0 < NQ; c0 += 32) {
+        uint32_t a[32];
+        tmem_ld32(tl + c0, a);
+        tmem_wait_ld();
+        uint32_t pk[16];
+#pragma unroll
+        for (int e = 0; e < 32; e += 4) {
+          const float4 bb = ld_v4f(s_bias + (c0 + e) * 4);
+          float f0 = __uint_as_float(a[e]) + bb.x, f1 = __uint_as_float(a[e + 1]) + bb.y;
+          float f2 = __uint_as_float(a[e + 2]) + bb.z, f3 = __uint_as_float(a[e + 3]) + bb.w;
+          if (!real) { f0 = 0.f; f1 = 0.f; f2 = 0.f; f3 = 0.f; }
+          pk[e >> 1] = t_bf2(f0, f1);
+          pk[(e >> 1) + 1] = t_bf2(f2, f3);
+        }
+        const uint32_t box = base + OFF_OUT + (c0 >> 6) * (TM * 128);
+        const int ch0 = (c0 & 32) >> 3;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) st_v4(sw128(box, r, ch0 + q), pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+      }
+      t_fence_before();
+      __syncwarp();
+      if (lane == 0) t_mbar_arrive(bars + B_ACCFREE);
+      t_fence_async();
+      t_bar_rows();
+      if (tid == 64) {
+#pragma unroll
+        for (int j = 0; j < 3; ++j) t_tma_store_2d(&tmOut, base + OFF_OUT + j * (TM * 128), 64 * j, row0);
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+      }
+      real = real_next;
+    }
+    if (tid == 64) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  }
+
+  t_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    t_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------------------------------------ out-proj + MLP
+namespace pm {
+constexpr int OFF_WO = 0;                          // W_o: 64 rows x 128 B
+constexpr int OFF_W1 = OFF_WO + TD * 128;          // W_1: up to 256 rows x 128 B
+constexpr int OFF_W2 = OFF_W1 + 256 * 128;         // W_2: up to 4 k-blocks of 64 rows x 128 B
+constexpr int OFF_ATT = OFF_W2 + 4 * TD * 128;     // 2 attention tiles
+constexpr int OFF_H = OFF_ATT + 2 * TM * 128;      // LN2 output
+constexpr int OFF_F = OFF_H + TM * 128;            // hidden units: up to 4 k-blocks of 128 rows x 128 B; later the y staging
+constexpr int OFF_X = OFF_F + 4 * TM * 128;        // float residual input tile (2 boxes)
+constexpr int OFF_P = OFF_X + 2 * XBOX;            // b_o[64], gamma[64], beta[64], b_2[64], b_1[256] as floats
+constexpr int OFF_BAR = OFF_P + (4 * TD + 256) * 4;
+constexpr int B_W = 0, B_ATTFULL = 8, B_ATTFREE = 24, B_XFULL = 40, B_XFREE = 48, B_ACC1 = 56, B_HREADY = 64, B_ACCF = 72,
+              B_FREADY = 80, B_ACCY = 88, SLOT = 96;
+constexpr int SMEM = OFF_BAR + 112 + 1024;
+constexpr int COL_1 = 0, COL_F = 64, COL_Y = 320, TMEM_COLS = 512;
+static_assert(SMEM <= 227 * 1024, "shared memory budget");
+}  // namespace pm
+
+__global__ void __launch_bounds__(T_THREADS, 1)
+proj_mlp_tc_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_constant__ CUtensorMap tmX,
+                   const __grid_constant__ CUtensorMap tmWo, const __grid_constant__ CUtensorMap tmW1,
+                   const __grid_constant__ CUtensorMap tmW2, const __grid_constant__ CUtensorMap tmY, const Geometry g,
+                   const float* __restrict__ bo, const float* __restrict__ gamma, const float* __restrict__ beta,
+                   const float eps, const float* __restrict__ b1, const float* __restrict__ b2, const int d_ff) {
+  using namespace pm;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t bars = base + OFF_BAR;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int rows = g.batch * g.L;
+  const int ntiles = (rows + TM - 1) / TM;
+  const int nh = d_ff / 64;  // k-blocks of hidden units
+
+  float* prm = reinterpret_cast<float*>(base_ptr + OFF_P);
+  stage_vector(prm, bo, TD, 0.f, tid, T_THREADS);
+  stage_vector(prm + TD, gamma, TD, 1.f, tid, T_THREADS);
+  stage_vector(prm + 2 * TD, beta, TD, 0.f, tid, T_THREADS);
+  stage_vector(prm + 3 * TD, b2, TD, 0.f, tid, T_THREADS);
+  stage_vector(prm + 4 * TD, b1, d_ff, 0.f, tid, T_THREADS);
+  if (tid == 0) {
+    t_mbar_init(bars + B_W, 1);
+    for (int i = 0; i < 2; ++i) { t_mbar_init(bars + B_ATTFULL + 8 * i, 1); t_mbar_init(bars + B_ATTFREE + 8 * i, 1); }
+    t_mbar_init(bars + B_XFULL, 1);
+    t_mbar_init(bars + B_XFREE, 4);
+    t_mbar_init(bars + B_ACC1, 1);
+    t_mbar_init(bars + B_HREADY, 4);
+    t_mbar_init(bars + B_ACCF, 1);
+    t_mbar_init(bars + B_FREADY, 4);
+    t_mbar_init(bars + B_ACCY, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    t_fence_async();
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(bars + SLOT), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  t_fence_before();
+  __syncthreads();
+  t_fence_after();
+  uint32_t tmem;
+  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tmem) : "r"(bars + SLOT) : "memory");
+
+  if (warp == 0) {
+    // ================================ producer ================================
+    if (t_elect()) {
+      t_mbar_expect_tx(bars + B_W, (uint32_t)(TD * 128 + d_ff * 128 + nh * TD * 128));
+      t_tma_2d(base + OFF_WO, &tmWo, 0, 0, bars + B_W);
+      t_tma_2d(base + OFF_W1, &tmW1, 0, 0, bars + B_W);
+      for (int kb = 0; kb < nh; ++kb) t_tma_2d(base + OFF_W2 + kb * TD * 128, &tmW2, 64 * kb, 0, bars + B_W);
+    }
+    __syncwarp();
+    int i = 0;
+    for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
+      const int row0 = t * TM;
+      const int b = i & 1;
+      if (i >= 2) t_mbar_wait(g, bars + B_ATTFREE + 8 * b, ((i >> 1) - 1) & 1);
+      if (t_elect()) {
+        t_mbar_expect_tx(bars + B_ATTFULL + 8 * b, TM * 128);
+        t_tma_2d(base + OFF_ATT + b * TM * 128, &tmAtt, 0, row0, bars + B_ATTFULL + 8 * b);
+      }
+      __syncwarp();
+      if (i > 0) t_mbar_wait(g, bars + B_XFREE, (i - 1) & 1);
+      if (t_elect()) {
+        t_mbar_expect_tx(bars + B_XFULL, 2 * XBOX);
+        t_tma_2d(base + OFF_X, &tmX, 0, row0, bars + B_XFULL);
+        t_tma_2d(base + OFF_X + XBOX, &tmX, 32, row0, bars + B_XFULL);
+      }
+      __syncwarp();
+    }
+  } else if (warp == 1) {
+    // ================================ MMA issuer ================================
+    constexpr uint32_t IDESC_D = t_idesc(TD);
+    const uint32_t idesc_f = t_idesc(d_ff);
+    t_mbar_wait(g, bars + B_W, 0);
+    int i = 0;
+    for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
+      const int b = i & 1;
+      // y1 accumulator = att W_o^T
+      t_mbar_wait(g, bars + B_ATTFULL + 8 * b, (i >> 1) & 1);
+      t_fence_after();
+      if (t_elect()) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          t_umma(tmem + COL_1, t_desc(base + OFF_ATT + b * TM * 128 + 32 * k), t_desc(base + OFF_WO + 32 * k), IDESC_D, k > 0);
+        t_commit(bars + B_ATTFREE + 8 * b);
+        t_commit(bars + B_ACC1);
+      }
+      __syncwarp();
+      // hidden accumulator = LN2(y1) W_1^T
+      t_mbar_wait(g, bars + B_HREADY, i & 1);
+      t_fence_after();
+      if (t_elect()) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          t_umma(tmem + COL_F, t_desc(base + OFF_H + 32 * k), t_desc(base + OFF_W1 + 32 * k), idesc_f, k > 0);
+        t_commit(bars + B_ACCF);
+      }
+      __syncwarp();
+      // output accumulator = relu(hidden) W_2^T
+      t_mbar_wait(g, bars + B_FREADY, i & 1);
+      t_fence_after();
+      if (t_elect()) {
+        for (int kb = 0; kb < nh; ++kb)
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            t_umma(tmem + COL_Y, t_desc(base + OFF_F + kb * TM * 128 + 32 * k), t_desc(base + OFF_W2 + kb * TD * 128 + 32 * k),
+                   IDESC_D, (kb > 0 || k > 0) ? 1u : 0u);
+        t_commit(bars + B_ACCY);
+      }
+      __syncwarp();
+    }
+  } else {
+    // ================================ one thread per sequence row ================================
+    const int r = ((warp & 3) << 5) + lane;
+    const uint32_t tl = tmem + ((uint32_t)((warp & 3) << 5) << 16);
+    const uint32_t s_bo = base + OFF_P, s_gamma = s_bo + TD * 4, s_beta = s_gamma + TD * 4, s_b2 = s_beta + TD * 4,
+                   s_b1 = s_b2 + TD * 4;
+    int i = 0;
+    bool real = row_real32(g, (int)blockIdx.x * TM + r, rows);
+    for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
+      const int row0 = t * TM;
+      // ---- y1 = x + att W_o^T + b_o (registers) ----
+      t_mbar_wait(g, bars + B_XFULL, i & 1);
+      float v[TD];
+      if (real) {
+        load_row64(base + OFF_X, r, v);
+      } else {
+#pragma unroll
+        for (int e = 0; e < TD; ++e) v[e] = 0.f;
+      }
+      __syncwarp();
+      if (lane == 0) t_mbar_arrive(bars + B_XFREE);
+      t_mbar_wait(g, bars + B_ACC1, i & 1);
+      t_fence_after();
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t a[32];
+        tmem_ld32(tl + COL_1 + 32 * c, a);
+        tmem_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 32; e += 4) {
+          const float4 bb = ld_v4f(s_bo + (32 * c + e) * 4);
+          v[32 * c + e] += __uint_as_float(a[e]) + bb.x;
+          v[32 * c + e + 1] += __uint_as_float(a[e + 1]) + bb.y;
+          v[32 * c + e + 2] += __uint_as_float(a[e + 2]) + bb.z;
+          v[32 * c + e + 3] += __uint_as_float(a[e + 3]) + bb.w;
+        }
+      }
+      // ---- h = LN2(y1) -> A operand of the first MLP product ----
+      layernorm_row_to_tile(v, real, s_gamma, s_beta, eps, base + OFF_H, r);
+      t_fence_async();
+      t_fence_before();
+      __syncwarp();
+      if (lane == 0) t_mbar_arrive(bars + B_HREADY);
+      const bool real_next = row_real32(g, (t + (int)gridDim.x) * TM + r, rows);  // overlaps the MMA
+      // ---- f = relu(h W_1^T + b_1) -> A operand of the second MLP product ----
+      t_mbar_wait(g, bars + B_ACCF, i & 1);
+      t_fence_after();
+      if (i > 0) {  // the previous tile's output stores must have finished reading the staging rows (they overlay f)
+        if (tid == 64) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        t_bar_rows();
+      }
+#pragma unroll 1
+      for (int c0 = 0; c0 < d_ff; c0 += 32) {
+        uint32_t a[32];
+        tmem_ld32(tl + COL_F + c0, a);
+        tmem_wait_ld();
+        uint32_t pk[16];
+#pragma unroll
+        for (int e = 0; e < 32; e += 4) {
+          const float4 bb = ld_v4f(s_b1 + (c0 + e) * 4);
+          pk[e >> 1] = t_bf2(fmaxf(__uint_as_float(a[e]) + bb.x, 0.f), fmaxf(__uint_as_float(a[e + 1]) + bb.y, 0.f));
+          pk[(e >> 1) + 1] = t_bf2(fmaxf(__uint_as_float(a[e + 2]) + bb.z, 0.f), fmaxf(__uint_as_float(a[e + 3]) + bb.w, 0.f));
+        }
+        const uint32_t blk = base + OFF_F + (c0 >> 6) * (TM * 128);
+        const int ch0 = (c0 & 32) >> 3;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) st_v4(sw128(blk, r, ch0 + q), pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+      }
+      t_fence_async();
+      t_fence_before();
+      __syncwarp();
+      if (lane == 0) t_mbar_arrive(bars + B_FREADY);
+      // ---- y = y1 + f W_2^T + b_2 -> staging rows (two boxes of 32 floats) -> TMA stores; padded rows +0 ----
+      t_mbar_wait(g, bars + B_ACCY, i & 1);
+      t_fence_after();
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t a[32];
+        tmem_ld32(tl + COL_Y + 32 * c, a);
+        tmem_wait_ld();
+        const uint32_t box = base + OFF_F + c * (TM * 128);
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) {
+          const int e = 32 * c + 4 * ch;
+          const float4 bb = ld_v4f(s_b2 + e * 4);
+          float o0 = v[e] + __uint_as_float(a[4 * ch]) + bb.x, o1 = v[e + 1] + __uint_as_float(a[4 * ch + 1]) + bb.y;
+          float o2 = v[e + 2] + __uint_as_float(a[4 * ch + 2]) + bb.z, o3 = v[e + 3] + __uint_as_float(a[4 * ch + 3]) + bb.w;
+          if (!real) { o0 = 0.f; o1 = 0.f; o2 = 0.f; o3 = 0.f; }
+          st_v4(sw128(box, r, ch), __float_as_uint(o0), __float_as_uint(o1), __float_as_uint(o2), __float_as_uint(o3));
+        }
+      }
+      t_fence_before();
+      t_fence_async();
+      t_bar_rows();
+      if (tid == 64) {
+        t_tma_store_2d(&tmY, base + OFF_F, 0, row0);
+        t_tma_store_2d(&tmY, base + OFF_F + TM * 128, 32, row0);
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+      }
+      real = real_next;
+    }
+    if (tid == 64) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  }
+
+  t_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    t_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+// 2-D map over a [rows, cols] float view with row pitch `row_stride` elements; box = [32 columns, box_rows rows] (128
+// bytes wide), 128-byte swizzle.
+bool make_map_f32(CUtensorMap* tm, const void* basep, int64_t rows, int cols, int64_t row_stride, int box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (fn == nullptr) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)row_stride * 4};
+  const cuuint32_t box[2] = {32u, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(basep), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int t_sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n = 0;
+  }
+  return n;
+}
+
+}  // namespace
+
+bool fused_layer_tc_supported(const Geometry& g, int d_ff) { return g.d == TD && d_ff >= 64 && d_ff <= 256 && d_ff % 64 == 0; }
+
+cudaError_t launch_ln_qkv_tc(const Geometry& g, const float* x, int64_t ldx, const float* gamma, const float* beta, float eps,
+                             const __nv_bfloat16* w_qkv, const float* b_qkv, __nv_bfloat16* qkv, cudaStream_t st) {
+  if (g.d != TD) return cudaErrorNotSupported;
+  const int64_t rows = (int64_t)g.batch * g.L;
+  const int ntiles = (int)((rows + TM - 1) / TM), nsm = t_sm_count();
+  if (nsm == 0) return cudaErrorUnknown;
+  alignas(64) CUtensorMap tmW, tmX, tmOut;
+  if (!make_map(&tmW, w_qkv, 3 * TD, TD, TD, 64, 3 * TD) || !make_map_f32(&tmX, x, rows, TD, ldx, TM) ||
+      !make_map(&tmOut, qkv, rows, 3 * TD, 3 * TD, 64, TM))
+    return cudaErrorInvalidValue;
+  static bool done = false;
+  if (!done) {
+    cudaError_t e = cudaFuncSetAttribute(ln_qkv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, qk::SMEM);
+    if (e != cudaSuccess) return e;
+    done = true;
+  }
+  ln_qkv_tc_kernel<<<min(ntiles, nsm), T_THREADS, qk::SMEM, st>>>(tmW, tmX, tmOut, g, gamma, beta, eps, b_qkv);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_proj_mlp_tc(const Geometry& g, const __nv_bfloat16* att, const float* x, int64_t ldx,
+                               const __nv_bfloat16* w_o, const float* b_o, const float* gamma, const float* beta, float eps,
+                               const __nv_bfloat16* w_1, const float* b_1, const __nv_bfloat16* w_2, const float* b_2, int d_ff,
+                               float* y, int64_t ldy, cudaStream_t st) {
+  if (!fused_layer_tc_supported(g, d_ff)) return cudaErrorNotSupported;
+  const int64_t rows = (int64_t)g.batch * g.L;
+  const int ntiles = (int)((rows + TM - 1) / TM), nsm = t_sm_count();
+  if (nsm == 0) return cudaErrorUnknown;
+  alignas(64) CUtensorMap tmAtt, tmX, tmWo, tmW1, tmW2, tmY;
+  if (!make_map(&tmAtt, att, rows, TD, TD, 64, TM) || !make_map_f32(&tmX, x, rows, TD, ldx, TM) || !make_map(&tmWo, w_o, TD, TD, TD, 64, TD) ||
+      !make_map(&tmW1, w_1, d_ff, TD, TD, 64, d_ff) || !make_map(&tmW2, w_2, TD, d_ff, d_ff, 64, TD) ||
+      !make_map_f32(&tmY, y, rows, TD, ldy, TM))
+    return cudaErrorInvalidValue;
+  static bool done = false;
+  if (!done) {
+    cudaError_t e = cudaFuncSetAttribute(proj_mlp_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, pm::SMEM);
+    if (e != cudaSuccess) return e;
+    done = true;
+  }
+  proj_mlp_tc_kernel<<<min(ntiles, nsm), T_THREADS, pm::SMEM, st>>>(tmAtt, tmX, tmWo, tmW1, tmW2, tmY, g, b_o, gamma, beta, eps,
+                                                                   b_1, b_2, d_ff);
+  return cudaGetLastError();
+}
+
+}  // namespace gsit

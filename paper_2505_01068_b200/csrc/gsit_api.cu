@@ -226,17 +226,27 @@ gsit_status gsit_im_layer_fwd(const gsit_shape* shape, const gsit_layer_weights*
 
   if (bf && fused_layer_supported(g, w->d_ff)) {
     // three launches: LN1 + shared projection, IM attention, out-projection + residual + LN2 + MLP + residual
+    // d_model 64 runs both halves on tcgen05 (tuning knob 9 keeps the mma.sync kernels)
+    const bool tc = fused_layer_tc_supported(g, w->d_ff) && g_attn_variant != 9;
     {
       TraceScope t(GSIT_KERNEL_LINEAR, cs);
-      st = from_cuda(launch_ln_qkv_bf16(g, x, x_row_stride, w->ln1_gamma, w->ln1_beta, eps,
-                                        static_cast<const __nv_bfloat16*>(w->w_qkv), w->b_qkv,
-                                        static_cast<__nv_bfloat16*>(qkv), cs));
+      st = from_cuda(tc ? launch_ln_qkv_tc(g, x, x_row_stride, w->ln1_gamma, w->ln1_beta, eps,
+                                           static_cast<const __nv_bfloat16*>(w->w_qkv), w->b_qkv,
+                                           static_cast<__nv_bfloat16*>(qkv), cs)
+                        : launch_ln_qkv_bf16(g, x, x_row_stride, w->ln1_gamma, w->ln1_beta, eps,
+                                             static_cast<const __nv_bfloat16*>(w->w_qkv), w->b_qkv,
+                                             static_cast<__nv_bfloat16*>(qkv), cs));
     }
     if (st != GSIT_OK) return st;
     const uint8_t* qb = static_cast<const uint8_t*>(qkv);
     if ((st = run_attention(g, dtype, qb, qb + (size_t)d * es, qb + (size_t)2 * d * es, 3 * (int64_t)d, att, nullptr,
                             pick_scale(shape, g), cs)) != GSIT_OK) return st;
     TraceScope t(GSIT_KERNEL_LINEAR, cs);
+    if (tc)
+      return from_cuda(launch_proj_mlp_tc(g, static_cast<const __nv_bfloat16*>(att), x, x_row_stride,
+                                          static_cast<const __nv_bfloat16*>(w->w_o), w->b_o, w->ln2_gamma, w->ln2_beta, eps,
+                                          static_cast<const __nv_bfloat16*>(w->w_1), w->b_1,
+                                          static_cast<const __nv_bfloat16*>(w->w_2), w->b_2, w->d_ff, y, y_row_stride, cs));
     return from_cuda(launch_proj_mlp_bf16(g, static_cast<const __nv_bfloat16*>(att), x, x_row_stride,
                                           static_cast<const __nv_bfloat16*>(w->w_o), w->b_o, w->ln2_gamma, w->ln2_beta, eps,
                                           static_cast<const __nv_bfloat16*>(w->w_1), w->b_1,
