@@ -102,6 +102,15 @@ cudaError_t launch_proj_mlp_tc(const Geometry& g, const __nv_bfloat16* att, cons
                                const __nv_bfloat16* w_1, const float* b_1, const __nv_bfloat16* w_2, const float* b_2, int d_ff,
                                float* y, int64_t ldy, cudaStream_t st);
 
+// ... and at d_model 128 (d_ff <= 512), with the MLP weights streamed in chunks (fused_layer_tc128.cu)
+bool fused_layer_tc128_supported(const Geometry& g, int d_ff);
+cudaError_t launch_ln_qkv_tc128(const Geometry& g, const float* x, int64_t ldx, const float* gamma, const float* beta, float eps,
+                                const __nv_bfloat16* w_qkv, const float* b_qkv, __nv_bfloat16* qkv, cudaStream_t st);
+cudaError_t launch_proj_mlp_tc128(const Geometry& g, const __nv_bfloat16* att, const float* x, int64_t ldx,
+                                  const __nv_bfloat16* w_o, const float* b_o, const float* gamma, const float* beta, float eps,
+                                  const __nv_bfloat16* w_1, const float* b_1, const __nv_bfloat16* w_2, const float* b_2, int d_ff,
+                                  float* y, int64_t ldy, cudaStream_t st);
+
 // Row LayerNorm of float x (row stride ldx) into float or bf16 y [rows, d]; padded rows become zero.
 cudaError_t launch_layernorm(const Geometry& g, const float* x, int64_t ldx, const float* gamma, const float* beta,
                              float eps, void* y, int out_bf16, cudaStream_t st);

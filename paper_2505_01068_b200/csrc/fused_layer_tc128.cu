@@ -1,0 +1,543 @@
+// The fused halves of the IM encoder layer at d_model 128 (the intra-modal encoder on the feature concat of the two
+// ring encoders) on tcgen05 / TMEM.  Same structure as fused_layer_tc.cu (one CTA per SM, 128-row tiles, thread = row
+// for LayerNorm and epilogues, operands in the 128-byte swizzle); what differs is the budget: rows are two k-blocks of
+// 64 features wide, the 384 QKV columns need two MMA groups (N 256 + N 128), and the MLP weights (2 x 128 KB at
+// d_ff 512) no longer fit in shared memory, so W_1 / W_2 stream through a two-stage TMA ring in chunks of 64 hidden
+// units while the hidden accumulator is double-buffered in TMEM.
+#include "fused_tc_common.cuh"
+
+namespace gsit {
+namespace {
+
+constexpr int D2 = 128;  // d_model
+
+// Reads the thread's float row r (128 values) from a four-box swizzled float tile.
+__device__ __forceinline__ void load_row128(uint32_t tile, int r, float (&v)[D2]) {
+#pragma unroll
+  for (int j = 0; j < 4; ++j)
+#pragma unroll
+    for (int ch = 0; ch < 8; ++ch) {
+      const float4 t = ld_v4f(sw128(tile + j * XBOX, r, ch));
+      const int e = 32 * j + 4 * ch;
+      v[e] = t.x; v[e + 1] = t.y; v[e + 2] = t.z; v[e + 3] = t.w;
+    }
+}
+// LayerNorm of one 128-feature row held by one thread -> bf16 row r of two swizzled k-block tiles (zeros when !real).
+__device__ __forceinline__ void layernorm_row128_to_tiles(const float (&v)[D2], bool real, uint32_t s_gamma, uint32_t s_beta,
+                                                          float eps, uint32_t tiles, int r) {
+  float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+  for (int e = 0; e < D2; e += 4) { s0 += v[e]; s1 += v[e + 1]; s2 += v[e + 2]; s3 += v[e + 3]; }
+  const float mean = ((s0 + s1) + (s2 + s3)) * (1.f / D2);
+  float q0 = 0.f, q1 = 0.f, q2 = 0.f, q3 = 0.f;
+#pragma unroll
+  for (int e = 0; e < D2; e += 4) {
+    const float a = v[e] - mean, b = v[e + 1] - mean, c = v[e + 2] - mean, d = v[e + 3] - mean;
+    q0 = fmaf(a, a, q0); q1 = fmaf(b, b, q1); q2 = fmaf(c, c, q2); q3 = fmaf(d, d, q3);
+  }
+  const float rstd = real ? rsqrtf(((q0 + q1) + (q2 + q3)) * (1.f / D2) + eps) : 0.f;
+#pragma unroll
+  for (int c8 = 0; c8 < D2 / 8; ++c8) {  // 16 chunks of 8 features: k-block c8 / 8, chunk c8 % 8
+    const float4 g0 = ld_v4f(s_gamma + c8 * 32), g1 = ld_v4f(s_gamma + c8 * 32 + 16);
+    const float4 b0 = ld_v4f(s_beta + c8 * 32), b1 = ld_v4f(s_beta + c8 * 32 + 16);
+    const float gm[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+    const float bt[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+    uint32_t pk[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int e = c8 * 8 + 2 * k;
+      float a = fmaf((v[e] - mean) * rstd, gm[2 * k], bt[2 * k]), b = fmaf((v[e + 1] - mean) * rstd, gm[2 * k + 1], bt[2 * k + 1]);
+      if (!real) { a = 0.f; b = 0.f; }
+      pk[k] = t_bf2(a, b);
+    }
+    st_v4(sw128(tiles + (c8 >> 3) * XBOX, r, c8 & 7), pk[0], pk[1], pk[2], pk[3]);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------ LN1 + shared QKV
+namespace qk2 {
+constexpr int NQ = 3 * D2;                        // 384 output columns
+constexpr int OFF_W = 0;                          // W_qkv: 2 k-blocks x 384 rows x 128 B
+constexpr int OFF_X = OFF_W + 2 * NQ * 128;       // float input tile (4 boxes); the normalised rows (2 k-blocks) overlay it
+constexpr int OFF_OUT = OFF_X + 4 * XBOX;         // 3 boxes of 64 columns: the output leaves in two passes
+constexpr int OFF_P = OFF_OUT + 3 * XBOX;         // gamma[128], beta[128], bias[384]
+constexpr int OFF_BAR = OFF_P + (2 * D2 + NQ) * 4;
+constexpr int B_W = 0, B_XFULL = 8, B_XFREE = 16, B_HREADY = 24, B_ACCFULL = 32, B_ACCFREE = 40, SLOT = 48;
+constexpr int SMEM = OFF_BAR + 64 + 1024;
+constexpr int TMEM_COLS = 512;
+static_assert(SMEM <= 227 * 1024, "shared memory budget");
+}  // namespace qk2
+
+__global__ void __launch_bounds__(T_THREADS, 1)
+ln_qkv_tc128_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
+                    const __grid_constant__ CUtensorMap tmOut, const Geometry g, const float* __restrict__ gamma,
+                    const float* __restrict__ beta, const float eps, const float* __restrict__ bias) {
+  using namespace qk2;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t bars = base + OFF_BAR;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int rows = g.batch * g.L;
+  const int ntiles = (rows + TM - 1) / TM;
+
+  float* prm = reinterpret_cast<float*>(base_ptr + OFF_P);
+  stage_vector(prm, gamma, D2, 1.f, tid, T_THREADS);
+  stage_vector(prm + D2, beta, D2, 0.f, tid, T_THREADS);
+  stage_vector(prm + 2 * D2, bias, NQ, 0.f, tid, T_THREADS);
+  if (tid == 0) {
+    t_mbar_init(bars + B_W, 1);
+    t_mbar_init(bars + B_XFULL, 1);
+    t_mbar_init(bars + B_XFREE, 4);
+    t_mbar_init(bars + B_HREADY, 4);
+    t_mbar_init(bars + B_ACCFULL, 1);
+    t_mbar_init(bars + B_ACCFREE, 4);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    t_fence_async();
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(bars + SLOT), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  t_fence_before();
+  __syncthreads();
+  t_fence_after();
+  uint32_t tmem;
+  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tmem) : "r"(bars + SLOT) : "memory");
+
+  if (warp == 0) {
+    // ================================ producer ================================
+    if (t_elect()) {
+      t_mbar_expect_tx(bars + B_W, 2 * NQ * 128);
+      for (int kb = 0; kb < 2; ++kb)
+        for (int j = 0; j < 3; ++j)  // boxes of 128 weight rows
+          t_tma_2d(base + OFF_W + kb * NQ * 128 + j * XBOX, &tmW, 64 * kb, 128 * j, bars + B_W);
+    }
+    __syncwarp();
+    int i = 0;
+    for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
+      // the tile buffer also held the previous tile's normalised rows: wait until the MMA has consumed them
+      if (i > 0) t_mbar_wait(g, bars + B_XFREE, (i - 1) & 1);
+      if (t_elect()) {
+        t_mbar_expect_tx(bars + B_XFULL, 4 * XBOX);
+        for (int j = 0; j < 4; ++j) t_tma_2d(base + OFF_X + j * XBOX, &tmX, 32 * j, t * TM, bars + B_XFULL);
+      }
+      __syncwarp();
+    }
+  } else if (warp == 1) {
+    // ================================ MMA issuer ================================
+    constexpr uint32_t IDESC_256 = t_idesc(256), IDESC_128 = t_idesc(128);
+    t_mbar_wait(g, bars + B_W, 0);
+    int i = 0;
+    for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
+      t_mbar_wait(g, bars + B_HREADY, i & 1);
+      if (i > 0) t_mbar_wait(g, bars + B_ACCFREE, (i - 1) & 1);
+      t_fence_after();
+      if (t_elect()) {
+#pragma unroll
+        for (int kb = 0; kb < 2; ++kb)
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const uint64_t a = t_desc(base + OFF_X + kb * XBOX + 32 * k);
+            const uint32_t w = base + OFF_W + kb * NQ * 128 + 32 * k;
+            t_umma(tmem, a, t_desc(w), IDESC_256, (kb > 0 || k > 0) ? 1u : 0u);                    // columns 0..255
+            t_umma(tmem + 256, a, t_desc(w + 256 * 128), IDESC_128, (kb > 0 || k > 0) ? 1u : 0u);  // columns 256..383
+          }
+        t_commit(bars + B_ACCFULL);
+      }
+      __syncwarp();
+    }
+  } else {
+    // ================================ one thread per sequence row ================================
+    const int r = ((warp & 3) << 5) + lane;
+    const uint32_t tl = tmem + ((uint32_t)((warp & 3) << 5) << 16);
+    const uint32_t s_gamma = base + OFF_P, s_beta = s_gamma + D2 * 4, s_bias = s_beta + D2 * 4;
+    int i = 0;
+    bool real = row_real32(g, (int)blockIdx.x * TM + r, rows);
+    for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
+      const int row0 = t * TM;
+      t_mbar_wait(g, bars + B_XFULL, i & 1);
+      float v[D2];
+      if (real) {
+        load_row128(base + OFF_X, r, v);
+      } else {  // padded input rows may hold anything (NaN included): never read them
+#pragma unroll
+        for (int e = 0; e < D2; ++e) v[e] = 0.f;
+      }
+      t_bar_rows();  // every row is in registers: the normalised rows may overwrite the tile
+      layernorm_row128_to_tiles(v, real, s_gamma, s_beta, eps, base + OFF_X, r);
+      t_fence_async();
+      __syncwarp();
+      if (lane == 0) t_mbar_arrive(bars + B_HREADY);
+      const bool real_next = row_real32(g, (t + (int)gridDim.x) * TM + r, rows);  // overlaps the MMA
+
+      t_mbar_wait(g, bars + B_ACCFULL, i & 1);
+      t_fence_after();
+      __syncwarp();
+      if (lane == 0) t_mbar_arrive(bars + B_XFREE);  // the MMA has read the normalised rows: the next tile may land
+#pragma unroll 1
+      for (int pass = 0; pass < 2; ++pass) {
+        if (i > 0 || pass > 0) {  // earlier stores must have finished reading the staging rows
+          if (tid == 64) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+          t_bar_rows();
+        }
+#pragma unroll 1
+        for (int c0 = 0; c0 < NQ / 2; c0 += 32) {
+          const int col = pass * (NQ / 2) + c0;
+          uint32_t a[32];
+          tmem_ld32(tl + col, a);
+          tmem_wait_ld();
+          uint32_t pk[16];
+#pragma unroll
+          for (int e = 0; e < 32; e += 4) {
+            const float4 bb = ld_v4f(s_bias + (col + e) * 4);
+            float f0 = __uint_as_float(a[e]) + bb.x, f1 = __uint_as_float(a[e + 1]) + bb.y;
+            float f2 = __uint_as_float(a[e + 2]) + bb.z, f3 = __uint_as_float(a[e + 3]) + bb.w;
+            if (!real) { f0 = 0.f; f1 = 0.f; f2 = 0.f; f3 = 0.f; }
+            pk[e >> 1] = t_bf2(f0, f1);
+            pk[(e >> 1) + 1] = t_bf2(f2, f3);
+          }
+          const uint32_t box = base + OFF_OUT + (c0 >> 6) * XBOX;
+          const int ch0 = (c0 & 32) >> 3;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) st_v4(sw128(box, r, ch0 + q), pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+        }
+        if (pass == 1) {
+          t_fence_before();
+          __syncwarp();
+          if (lane == 0) t_mbar_arrive(bars + B_ACCFREE);
+        }
+        t_fence_async();
+        t_bar_rows();
+        if (tid == 64) {
+#pragma unroll
+          for (int j = 0; j < 3; ++j) t_tma_store_2d(&tmOut, base + OFF_OUT + j * XBOX, pass * (NQ / 2) + 64 * j, row0);
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        }
+      }
+      real = real_next;
+    }
+    if (tid == 64) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  }
+
+  t_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    t_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------------------------------------ out-proj + MLP
+namespace pm2 {
+constexpr int OFF_WO = 0;                          // W_o: 2 k-blocks x 128 rows x 128 B
+constexpr int OFF_ATT = OFF_WO + 2 * XBOX;         // attention tile (2 k-blocks); LN2 output overlays it
+constexpr int OFF_X = OFF_ATT + 2 * XBOX;          // float residual input tile (4 boxes)
+constexpr int WC_STAGE = 2 * 64 * 128 + XBOX;      // W_1 chunk: 2 k-blocks x 64 rows; W_2 chunk: 128 rows x 128 B
+constexpr int OFF_WC = OFF_X + 4 * XBOX;           // 2 stages
+constexpr int OFF_F = OFF_WC + 2 * WC_STAGE;       // hidden chunk: 128 rows x 64 units, bf16
+constexpr int OFF_P = OFF_F + XBOX;                // b_o[128], gamma[128], beta[128], b_2[128], b_1[512]
+constexpr int OFF_BAR = OFF_P + (4 * D2 + 512) * 4;
+constexpr int B_WO = 0, B_ATTFULL = 8, B_ATTFREE = 16, B_XFULL = 24, B_XFREE = 32, B_ACC1 = 40, B_HREADY = 48,
+              B_WCFULL = 56, B_WCFREE = 72, B_ACCF = 88, B_FREADY = 104, B_FFREE = 112, B_ACCY = 120, SLOT = 128;
+constexpr int SMEM = OFF_BAR + 144 + 1024;
+constexpr int COL_1 = 0, COL_F = 128, COL_Y = 256, TMEM_COLS = 512;
+static_assert(SMEM <= 227 * 1024, "shared memory budget");
+}  // namespace pm2
+
+__global__ void __launch_bounds__(T_THREADS, 1)
+proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_constant__ CUtensorMap tmX,
+                      const __grid_constant__ CUtensorMap tmWo, const __grid_constant__ CUtensorMap tmW1,
+                      const __grid_constant__ CUtensorMap tmW2, const Geometry g, const float* __restrict__ bo,
+                      const float* __restrict__ gamma, const float* __restrict__ beta, const float eps,
+                      const float* __restrict__ b1, const float* __restrict__ b2, const int d_ff, float* __restrict__ y,
+                      const int64_t ldy) {
+  using namespace pm2;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t bars = base + OFF_BAR;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int rows = g.batch * g.L;
+  const int ntiles = (rows + TM - 1) / TM;
+  const int nc = d_ff / 64;  // chunks of 64 hidden units
+
+  float* prm = reinterpret_cast<float*>(base_ptr + OFF_P);
+  stage_vector(prm, bo, D2, 0.f, tid, T_THREADS);
+  stage_vector(prm + D2, gamma, D2, 1.f, tid, T_THREADS);
+  stage_vector(prm + 2 * D2, beta, D2, 0.f, tid, T_THREADS);
+  stage_vector(prm + 3 * D2, b2, D2, 0.f, tid, T_THREADS);
+  stage_vector(prm + 4 * D2, b1, d_ff, 0.f, tid, T_THREADS);
+  if (tid == 0) {
+    t_mbar_init(bars + B_WO, 1);
+    t_mbar_init(bars + B_ATTFULL, 1);
+    t_mbar_init(bars + B_ATTFREE, 1);
+    t_mbar_init(bars + B_XFULL, 1);
+    t_mbar_init(bars + B_XFREE, 4);
+    t_mbar_init(bars + B_ACC1, 1);
+    t_mbar_init(bars + B_HREADY, 4);
+    for (int i = 0; i < 2; ++i) {
+      t_mbar_init(bars + B_WCFULL + 8 * i, 1);
+      t_mbar_init(bars + B_WCFREE + 8 * i, 1);
+      t_mbar_init(bars + B_ACCF + 8 * i, 1);
+    }
+    t_mbar_init(bars + B_FREADY, 4);
+    t_mbar_init(bars + B_FFREE, 1);
+    t_mbar_init(bars + B_ACCY, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    t_fence_async();
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(bars + SLOT), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  t_fence_before();
+  __syncthreads();
+  t_fence_after();
+  uint32_t tmem;
+  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tmem) : "r"(bars + SLOT) : "memory");
+
+  if (warp == 0) {
+    // ================================ producer ================================
+    if (t_elect()) {
+      t_mbar_expect_tx(bars + B_WO, 2 * XBOX);
+      for (int kb = 0; kb < 2; ++kb) t_tma_2d(base + OFF_WO + kb * XBOX, &tmWo, 64 * kb, 0, bars + B_WO);
+    }
+    __syncwarp();
+    int i = 0, n = 0;  // tiles, weight chunks requested so far
+    for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
+      const int row0 = t * TM;
+      // the attention buffer also holds the LN2 rows of the previous tile until its last first-MLP product is done
+      if (i > 0) t_mbar_wait(g, bars + B_ATTFREE, (i - 1) & 1);
+      if (t_elect()) {
+        t_mbar_expect_tx(bars + B_ATTFULL, 2 * XBOX);
+        for (int kb = 0; kb < 2; ++kb) t_tma_2d(base + OFF_ATT + kb * XBOX, &tmAtt, 64 * kb, row0, bars + B_ATTFULL);
+      }
+      __syncwarp();
+      if (i > 0) t_mbar_wait(g, bars + B_XFREE, (i - 1) & 1);
+      if (t_elect()) {
+        t_mbar_expect_tx(bars + B_XFULL, 4 * XBOX);
+        for (int j = 0; j < 4; ++j) t_tma_2d(base + OFF_X + j * XBOX, &tmX, 32 * j, row0, bars + B_XFULL);
+      }
+      __syncwarp();
+      for (int c = 0; c < nc; ++c, ++n) {
+        const int st = n & 1, use = n >> 1;
+        if (use > 0) t_mbar_wait(g, bars + B_WCFREE + 8 * st, (use - 1) & 1);
+        if (t_elect()) {
+          const uint32_t dst = base + OFF_WC + st * WC_STAGE;
+          t_mbar_expect_tx(bars + B_WCFULL + 8 * st, WC_STAGE);
+          t_tma_2d(dst, &tmW1, 0, 64 * c, bars + B_WCFULL + 8 * st);                // W_1[64c .. 64c+63, 0..63]
+          t_tma_2d(dst + 64 * 128, &tmW1, 64, 64 * c, bars + B_WCFULL + 8 * st);    // W_1[64c .. 64c+63, 64..127]
+          t_tma_2d(dst + 2 * 64 * 128, &tmW2, 64 * c, 0, bars + B_WCFULL + 8 * st); // W_2[0..127, 64c .. 64c+63]
+        }
+        __syncwarp();
+      }
+    }
+  } else if (warp == 1) {
+    // ================================ MMA issuer ================================
+    constexpr uint32_t IDESC_128 = t_idesc(128), IDESC_64 = t_idesc(64);
+    t_mbar_wait(g, bars + B_WO, 0);
+    int i = 0, n = 0;  // tiles done, chunks whose first product has been issued
+    for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
+      // y1 accumulator = att W_o^T
+      t_mbar_wait(g, bars + B_ATTFULL, i & 1);
+      t_fence_after();
+      if (t_elect()) {
+#pragma unroll
+        for (int kb = 0; kb < 2; ++kb)
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            t_umma(tmem + COL_1, t_desc(base + OFF_ATT + kb * XBOX + 32 * k), t_desc(base + OFF_WO + kb * XBOX + 32 * k),
+                   IDESC_128, (kb > 0 || k > 0) ? 1u : 0u);
+        t_commit(bars + B_ACC1);
+      }
+      __syncwarp();
+      t_mbar_wait(g, bars + B_HREADY, i & 1);
+      // second product of chunk m (global index): accY += relu-hidden(m) W_2c^T
+      auto second = [&](int m, bool first_of_tile, bool last_of_tile) {
+        t_mbar_wait(g, bars + B_FREADY, m & 1);
+        t_fence_after();
+        if (t_elect()) {
+          const uint32_t w2 = base + OFF_WC + (m & 1) * WC_STAGE + 2 * 64 * 128;
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            t_umma(tmem + COL_Y, t_desc(base + OFF_F + 32 * k), t_desc(w2 + 32 * k), IDESC_128, (!first_of_tile || k > 0) ? 1u : 0u);
+          t_commit(bars + B_WCFREE + 8 * (m & 1));
+          t_commit(bars + B_FFREE);
+          if (last_of_tile) t_commit(bars + B_ACCY);
+        }
+        __syncwarp();
+      };
+      for (int c = 0; c < nc; ++c, ++n) {
+        // first product of chunk n: hidden accumulator (n & 1) = LN2(y1) W_1c^T
+        const int st = n & 1;
+        t_mbar_wait(g, bars + B_WCFULL + 8 * st, (n >> 1) & 1);
+        t_fence_after();
+        if (t_elect()) {
+          const uint32_t w1 = base + OFF_WC + st * WC_STAGE;
+#pragma unroll
+          for (int kb = 0; kb < 2; ++kb)
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              t_umma(tmem + COL_F + 64 * st, t_desc(base + OFF_ATT + kb * XBOX + 32 * k), t_desc(w1 + kb * 64 * 128 + 32 * k),
+                     IDESC_64, (kb > 0 || k > 0) ? 1u : 0u);
+          t_commit(bars + B_ACCF + 8 * st);
+          if (c + 1 == nc) t_commit(bars + B_ATTFREE);  // LN2 rows no longer needed: the next attention tile may land
+        }
+        __syncwarp();
+        if (c > 0) second(n - 1, c == 1, false);
+      }
+      second(n - 1, nc == 1, true);
+    }
+  } else {
+    // ================================ one thread per sequence row ================================
+    const int r = ((warp & 3) << 5) + lane;
+    const uint32_t tl = tmem + ((uint32_t)((warp & 3) << 5) << 16);
+    const uint32_t s_bo = base + OFF_P, s_gamma = s_bo + D2 * 4, s_beta = s_gamma + D2 * 4, s_b2 = s_beta + D2 * 4,
+                   s_b1 = s_b2 + D2 * 4;
+    int i = 0, n = 0;
+    bool real = row_real32(g, (int)blockIdx.x * TM + r, rows);
+    for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
+      const int row0 = t * TM;
+      // ---- y1 = x + att W_o^T + b_o (registers) ----
+      t_mbar_wait(g, bars + B_XFULL, i & 1);
+      float v[D2];
+      if (real) {
+        load_row128(base + OFF_X, r, v);
+      } else {
+#pragma unroll
+        for (int e = 0; e < D2; ++e) v[e] = 0.f;
+      }
+      __syncwarp();
+      if (lane == 0) t_mbar_arrive(bars + B_XFREE);
+      t_mbar_wait(g, bars + B_ACC1, i & 1);
+      t_fence_after();
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t a[32];
+        tmem_ld32(tl + COL_1 + 32 * c, a);
+        tmem_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 32; e += 4) {
+          const float4 bb = ld_v4f(s_bo + (32 * c + e) * 4);
+          v[32 * c + e] += __uint_as_float(a[e]) + bb.x;
+          v[32 * c + e + 1] += __uint_as_float(a[e + 1]) + bb.y;
+          v[32 * c + e + 2] += __uint_as_float(a[e + 2]) + bb.z;
+          v[32 * c + e + 3] += __uint_as_float(a[e + 3]) + bb.w;
+        }
+      }
+      // ---- h = LN2(y1) over the attention tile (its product has completed) ----
+      layernorm_row128_to_tiles(v, real, s_gamma, s_beta, eps, base + OFF_ATT, r);
+      t_fence_async();
+      t_fence_before();
+      __syncwarp();
+      if (lane == 0) t_mbar_arrive(bars + B_HREADY);
+      const bool real_next = row_real32(g, (t + (int)gridDim.x) * TM + r, rows);
+      // ---- hidden chunks: f = relu(h W_1c^T + b_1c) -> A operand of the second product ----
+#pragma unroll 1
+      for (int c = 0; c < nc; ++c, ++n) {
+        t_mbar_wait(g, bars + B_ACCF + 8 * (n & 1), (n >> 1) & 1);
+        t_fence_after();
+        uint32_t pk[32];
+#pragma unroll
+        for (int hlf = 0; hlf < 2; ++hlf) {
+          uint32_t a[32];
+          tmem_ld32(tl + COL_F + 64 * (n & 1) + 32 * hlf, a);
+          tmem_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; e += 4) {
+            const float4 bb = ld_v4f(s_b1 + (64 * c + 32 * hlf + e) * 4);
+            pk[16 * hlf + (e >> 1)] = t_bf2(fmaxf(__uint_as_float(a[e]) + bb.x, 0.f), fmaxf(__uint_as_float(a[e + 1]) + bb.y, 0.f));
+            pk[16 * hlf + (e >> 1) + 1] = t_bf2(fmaxf(__uint_as_float(a[e + 2]) + bb.z, 0.f), fmaxf(__uint_as_float(a[e + 3]) + bb.w, 0.f));
+          }
+        }
+        if (n > 0) t_mbar_wait(g, bars + B_FFREE, (n - 1) & 1);  // the previous second product has read the hidden chunk
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) st_v4(sw128(base + OFF_F, r, ch), pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
+        t_fence_async();
+        t_fence_before();
+        __syncwarp();
+        if (lane == 0) t_mbar_arrive(bars + B_FREADY);
+      }
+      // ---- y = y1 + f W_2^T + b_2: each thread stores its own 512-byte row; padded rows +0 ----
+      t_mbar_wait(g, bars + B_ACCY, i & 1);
+      t_fence_after();
+      float4* dst = reinterpret_cast<float4*>(y + (int64_t)(row0 + r) * ldy);
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t a[32];
+        tmem_ld32(tl + COL_Y + 32 * c, a);
+        tmem_wait_ld();
+        if (row0 + r < rows) {
+#pragma unroll
+          for (int e = 0; e < 32; e += 4) {
+            const float4 bb = ld_v4f(s_b2 + (32 * c + e) * 4);
+            float4 o = make_float4(v[32 * c + e] + __uint_as_float(a[e]) + bb.x, v[32 * c + e + 1] + __uint_as_float(a[e + 1]) + bb.y,
+                                   v[32 * c + e + 2] + __uint_as_float(a[e + 2]) + bb.z, v[32 * c + e + 3] + __uint_as_float(a[e + 3]) + bb.w);
+            if (!real) o = make_float4(0.f, 0.f, 0.f, 0.f);
+            dst[8 * c + (e >> 2)] = o;
+          }
+        }
+      }
+      t_fence_before();  // orders these TMEM reads before the next tile's products (which wait for this thread's arrivals)
+      real = real_next;
+    }
+  }
+
+  t_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    t_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+}  // namespace
+
+bool fused_layer_tc128_supported(const Geometry& g, int d_ff) { return g.d == D2 && d_ff >= 64 && d_ff <= 512 && d_ff % 64 == 0; }
+
+cudaError_t launch_ln_qkv_tc128(const Geometry& g, const float* x, int64_t ldx, const float* gamma, const float* beta, float eps,
+                                const __nv_bfloat16* w_qkv, const float* b_qkv, __nv_bfloat16* qkv, cudaStream_t st) {
+  if (g.d != D2) return cudaErrorNotSupported;
+  const int64_t rows = (int64_t)g.batch * g.L;
+  const int ntiles = (int)((rows + TM - 1) / TM), nsm = t_sm_count();
+  if (nsm == 0) return cudaErrorUnknown;
+  alignas(64) CUtensorMap tmW, tmX, tmOut;
+  if (!make_map(&tmW, w_qkv, 3 * D2, D2, D2, 64, 128) || !make_map_f32(&tmX, x, rows, D2, ldx, TM) ||
+      !make_map(&tmOut, qkv, rows, 3 * D2, 3 * D2, 64, TM))
+    return cudaErrorInvalidValue;
+  static bool done = false;
+  if (!done) {
+    cudaError_t e = cudaFuncSetAttribute(ln_qkv_tc128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, qk2::SMEM);
+    if (e != cudaSuccess) return e;
+    done = true;
+  }
+  ln_qkv_tc128_kernel<<<min(ntiles, nsm), T_THREADS, qk2::SMEM, st>>>(tmW, tmX, tmOut, g, gamma, beta, eps, b_qkv);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_proj_mlp_tc128(const Geometry& g, const __nv_bfloat16* att, const float* x, int64_t ldx,
+                                  const __nv_bfloat16* w_o, const float* b_o, const float* gamma, const float* beta, float eps,
+                                  const __nv_bfloat16* w_1, const float* b_1, const __nv_bfloat16* w_2, const float* b_2, int d_ff,
+                                  float* y, int64_t ldy, cudaStream_t st) {
+  if (!fused_layer_tc128_supported(g, d_ff)) return cudaErrorNotSupported;
+  const int64_t rows = (int64_t)g.batch * g.L;
+  const int ntiles = (int)((rows + TM - 1) / TM), nsm = t_sm_count();
+  if (nsm == 0) return cudaErrorUnknown;
+  alignas(64) CUtensorMap tmAtt, tmX, tmWo, tmW1, tmW2;
+  if (!make_map(&tmAtt, att, rows, D2, D2, 64, TM) || !make_map_f32(&tmX, x, rows, D2, ldx, TM) ||
+      !make_map(&tmWo, w_o, D2, D2, D2, 64, D2) || !make_map(&tmW1, w_1, d_ff, D2, D2, 64, 64) ||
+      !make_map(&tmW2, w_2, D2, d_ff, d_ff, 64, D2))
+    return cudaErrorInvalidValue;
+  static bool done = false;
+  if (!done) {
+    cudaError_t e = cudaFuncSetAttribute(proj_mlp_tc128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, pm2::SMEM);
+    if (e != cudaSuccess) return e;
+    done = true;
+  }
+  proj_mlp_tc128_kernel<<<min(ntiles, nsm), T_THREADS, pm2::SMEM, st>>>(tmAtt, tmX, tmWo, tmW1, tmW2, g, b_o, gamma, beta, eps,
+                                                                       b_1, b_2, d_ff, y, ldy);
+  return cudaGetLastError();
+}
+
+}  // namespace gsit

@@ -224,15 +224,19 @@ gsit_status gsit_im_layer_fwd(const gsit_shape* shape, const gsit_layer_weights*
   const int es = bf ? 2 : 4;
   const int M = g.batch * g.L, d = g.d;
 
-  if (bf && fused_layer_supported(g, w->d_ff)) {
+  if (bf && fused_layer_supported(g, w->d_ff) && g_attn_variant != 8) {
     // three launches: LN1 + shared projection, IM attention, out-projection + residual + LN2 + MLP + residual
-    // d_model 64 runs both halves on tcgen05 (tuning knob 9 keeps the mma.sync kernels)
+    // d_model 64 and 128 run both halves on tcgen05 (tuning knob 9 keeps the mma.sync kernels)
     const bool tc = fused_layer_tc_supported(g, w->d_ff) && g_attn_variant != 9;
+    const bool tc128 = fused_layer_tc128_supported(g, w->d_ff) && g_attn_variant != 9;
     {
       TraceScope t(GSIT_KERNEL_LINEAR, cs);
       st = from_cuda(tc ? launch_ln_qkv_tc(g, x, x_row_stride, w->ln1_gamma, w->ln1_beta, eps,
                                            static_cast<const __nv_bfloat16*>(w->w_qkv), w->b_qkv,
                                            static_cast<__nv_bfloat16*>(qkv), cs)
+                     : tc128 ? launch_ln_qkv_tc128(g, x, x_row_stride, w->ln1_gamma, w->ln1_beta, eps,
+                                                   static_cast<const __nv_bfloat16*>(w->w_qkv), w->b_qkv,
+                                                   static_cast<__nv_bfloat16*>(qkv), cs)
                         : launch_ln_qkv_bf16(g, x, x_row_stride, w->ln1_gamma, w->ln1_beta, eps,
                                              static_cast<const __nv_bfloat16*>(w->w_qkv), w->b_qkv,
                                              static_cast<__nv_bfloat16*>(qkv), cs));
@@ -247,6 +251,11 @@ gsit_status gsit_im_layer_fwd(const gsit_shape* shape, const gsit_layer_weights*
                                           static_cast<const __nv_bfloat16*>(w->w_o), w->b_o, w->ln2_gamma, w->ln2_beta, eps,
                                           static_cast<const __nv_bfloat16*>(w->w_1), w->b_1,
                                           static_cast<const __nv_bfloat16*>(w->w_2), w->b_2, w->d_ff, y, y_row_stride, cs));
+    if (tc128)
+      return from_cuda(launch_proj_mlp_tc128(g, static_cast<const __nv_bfloat16*>(att), x, x_row_stride,
+                                             static_cast<const __nv_bfloat16*>(w->w_o), w->b_o, w->ln2_gamma, w->ln2_beta, eps,
+                                             static_cast<const __nv_bfloat16*>(w->w_1), w->b_1,
+                                             static_cast<const __nv_bfloat16*>(w->w_2), w->b_2, w->d_ff, y, y_row_stride, cs));
     return from_cuda(launch_proj_mlp_bf16(g, static_cast<const __nv_bfloat16*>(att), x, x_row_stride,
                                           static_cast<const __nv_bfloat16*>(w->w_o), w->b_o, w->ln2_gamma, w->ln2_beta, eps,
                                           static_cast<const __nv_bfloat16*>(w->w_1), w->b_1,

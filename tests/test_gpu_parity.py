@@ -146,10 +146,11 @@ def test_cfg5_scaled_hd64_bf16(g):
 
 @pytest.mark.parametrize("d,heads,d_ff,seg,B", [(64, 8, 256, (50, 170, 93), 3), (128, 8, 512, (37, 150, 64), 2),
                                                 (64, 4, 64, (50, 30, 90), 2), (64, 8, 128, (5, 0, 9), 3),
-                                                (32, 4, 128, (40, 33, 20), 2), (192, 3, 768, (70, 129, 33), 2)])
+                                                (32, 4, 128, (40, 33, 20), 2), (192, 3, 768, (70, 129, 33), 2), (128, 4, 64, (5, 0, 9), 3),
+                                                (128, 8, 320, (50, 201, 93), 2), (64, 8, 192, (300, 20, 333), 2)])
 def test_layer_bf16_affine_biases_ragged(g, d, heads, d_ff, seg, B):
     """One IM layer with LayerNorm affine parameters and every bias set, ragged valid lengths, NaN in the padded input
-    rows and a row count that is not a multiple of any tile: d = 64 / 128 take the fused kernels, d = 32 the separate
+    rows and a row count that is not a multiple of any tile: d = 64 / 128 take the fused tcgen05 kernels, d = 32 the separate
     LayerNorm / mma.sync linear kernels, d = 192 the separate kernels with every linear layer on the tcgen05 GEMM (bias,
     ReLU, float output with residual, TMA-stored bf16 output)."""
     rng = np.random.default_rng(d * 1000 + d_ff)
@@ -190,5 +191,28 @@ def test_qkv_proj_tcgen05_matches_mma_sync_kernel(g):
     check_close(new, ref, "bf16", pm, "tcgen05 projection")
     check_close(old, ref, "bf16", pm, "mma.sync projection")
     assert np.abs(new - old).max() <= 2.0 ** -6
+    code, flags = g.last_device_status()
+    assert code == 0 and flags == 0
+
+
+@pytest.mark.parametrize("d,heads,d_ff", [(64, 8, 256), (128, 8, 512)])
+def test_fused_layer_tcgen05_matches_mma_sync_fused_kernels(g, d, heads, d_ff):
+    """The tcgen05 fused halves and the mma.sync fused halves (tuning knob 9) compute the same layer."""
+    rng = np.random.default_rng(d)
+    seg, B = (50, 333, 190), 2
+    x = rng.standard_normal((B, sum(seg), d), dtype=np.float32)
+    w = weights_to_dev(wk.draw_layer_weights(rng, d, d_ff, "bf16", affine=True), "bf16")
+    valid = np.array([[50, 333, 190], [25, 170, 1]], dtype=np.int32)
+    vl = torch.from_numpy(valid).cuda()
+    xd = to_dev(wk.fill_padding(x, seg, valid, np.nan))
+    new = to_np64(g.im_layer_fwd(xd, w, seg, heads, vl, oracle.PHASE_INTER_BWD))
+    g.tune_attention(9)
+    try:
+        old = to_np64(g.im_layer_fwd(xd, w, seg, heads, vl, oracle.PHASE_INTER_BWD))
+    finally:
+        g.tune_attention(0)
+    assert np.isfinite(new).all() and np.abs(new - old).max() <= 2e-2 and np.abs(new - old).mean() <= 1e-3
+    pm = pad_mask(seg, valid, B)
+    assert np.all(new[pm] == 0.0)
     code, flags = g.last_device_status()
     assert code == 0 and flags == 0
