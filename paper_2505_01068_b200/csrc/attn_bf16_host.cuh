@@ -21,9 +21,21 @@ cudaError_t launch_one(const Geometry& g, const __nv_bfloat16* q, const __nv_bfl
   }
   int tiles = 0;
   for (int s = 0; s < 3; ++s) tiles += (g.seg_len[s] + C::QT - 1) / C::QT;
-  const dim3 grid((unsigned)tiles, (unsigned)(g.d / CW), (unsigned)g.batch);
+  if ((int64_t)tiles * g.batch > 0x7fffffffLL) return cudaErrorNotSupported;
+  // query segments in descending order of the keys their tiles walk (longest work first)
+  int cost[3], ord[3] = {0, 1, 2};
+  for (int s = 0; s < 3; ++s) {
+    cost[s] = 0;
+    for (int r = 0; r < 3; ++r)
+      if ((g.allowed >> (3 * s + r)) & 1u) cost[s] += g.seg_len[r];
+  }
+  for (int i = 0; i < 3; ++i)
+    for (int j = i + 1; j < 3; ++j)
+      if (cost[ord[j]] > cost[ord[i]]) { const int t = ord[i]; ord[i] = ord[j]; ord[j] = t; }
+  const int seg_order = ord[0] | (ord[1] << 2) | (ord[2] << 4);
+  const dim3 grid((unsigned)(tiles * g.batch), (unsigned)(g.d / CW), 1u);
   const float sl2 = scale * 1.4426950408889634f;
-  attn_bf16_kernel<C><<<grid, NTHREADS, C::SMEM, st>>>(tmQ, tmK, tmV, g, out, lse, sl2);
+  attn_bf16_kernel<C><<<grid, NTHREADS, C::SMEM, st>>>(tmQ, tmK, tmV, g, out, lse, sl2, seg_order);
   return cudaGetLastError();
 }
 

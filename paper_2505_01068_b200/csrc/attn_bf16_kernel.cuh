@@ -10,7 +10,7 @@ template <typename C>
 __global__ void __launch_bounds__(NTHREADS, C::MINB)
 attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, const Geometry g, __nv_bfloat16* __restrict__ out,
-                 float* __restrict__ lse, const float sl2 /* scale * log2(e) */) {
+                 float* __restrict__ lse, const float sl2 /* scale * log2(e) */, const int seg_order) {
   constexpr int HD = C::HD, CW = C::CW, G = C::G, R = C::R, QT = C::QT, PITCH = C::PITCH, SWZ = C::SWZ,
                 KSTEP = C::KSTEP, NT = C::NT, KSQ = C::KSQ, NTO = C::NTO, CPR = CW / 8 /* 16-byte chunks per row */;
   constexpr bool HOIST = (R > 1);  // several query slabs per warp reuse the K/V fragments of a step
@@ -28,16 +28,19 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   const int head_in_slice = warp % G, sg = warp / G;
   const int cb = head_in_slice * (HD / 8);  // first 16-byte chunk of this warp's head inside a tile row
 
-  // ---- which tile of which block row ----
-  int tile = blockIdx.x, s = 0;
+  // ---- which tile of which block row.  blockIdx.x = (tile in cost order) * batch + sample: the query segments with
+  // the most keys to walk are launched first (seg_order packs the three segment indices, two bits each), and CTAs that
+  // run together work on the same tile of different samples, so the last wave is short and made of the cheapest tiles.
+  const int b = blockIdx.x % g.batch;
+  int tile = blockIdx.x / g.batch, s = seg_order & 3;
 #pragma unroll
-  for (int ss = 0; ss < 2; ++ss) {
+  for (int rank = 0; rank < 2; ++rank) {
     const int nts = (g.seg_len[s] + QT - 1) / QT;
-    if (tile >= nts) { tile -= nts; ++s; }
+    if (tile >= nts) { tile -= nts; s = (seg_order >> (2 * rank + 2)) & 3; }
   }
   const int q0 = tile * QT;
   const int rows_in_tile = min(QT, g.seg_len[s] - q0);
-  const int b = blockIdx.z, cs = blockIdx.y;
+  const int cs = blockIdx.y;
   const int q_real_all = max(0, min(rows_in_tile, valid_rows(g, b, s) - q0));
   const int kn0 = ((g.allowed >> (3 * s + 0)) & 1u) ? valid_rows(g, b, 0) : 0;
   const int kn1 = ((g.allowed >> (3 * s + 1)) & 1u) ? valid_rows(g, b, 1) : 0;
