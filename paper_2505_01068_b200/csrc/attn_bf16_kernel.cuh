@@ -70,11 +70,11 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   };
 
   float O[R][NTO][4];
-  float m[R][2], l[R][2];
+  float m[R][2], l[R][4];  // l: accumulator tile of P 1 (elements 0 and 2 are the sums of rows g and g + 8)
 #pragma unroll
   for (int r_ = 0; r_ < R; ++r_) {
     m[r_][0] = m[r_][1] = -INFINITY;
-    l[r_][0] = l[r_][1] = 0.f;
+    l[r_][0] = l[r_][1] = l[r_][2] = l[r_][3] = 0.f;
 #pragma unroll
     for (int n = 0; n < NTO; ++n) O[r_][n][0] = O[r_][n][1] = O[r_][n][2] = O[r_][n][3] = 0.f;
   }
@@ -233,33 +233,32 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           const float al0 = ex2(fmaf(m[r_][0], sl2, -ms0)), al1 = ex2(fmaf(m[r_][1], sl2, -ms1));
           m[r_][0] = mn0;
           m[r_][1] = mn1;
+          // Exponentials two at a time: one packed FMA forms s * sl2 - m * sl2 for a pair (both <= 0), the pair is
+          // rounded to bf16 (absolute error <= 2^-9 |x|, i.e. negligible where the weight is not) and one packed ex2
+          // yields the two bf16 weights already in the layout of the A operand of P V.  The row sum is taken by the
+          // tensor core from those same bf16 weights (a column of ones appended to V), so numerator and denominator
+          // of the softmax see identical values.
+          const float2 sl2v = make_float2(sl2, sl2), nm0 = make_float2(-ms0, -ms0), nm1 = make_float2(-ms1, -ms1);
+          uint32_t P[NT][2];
 #pragma unroll
           for (int n = 0; n < NT; ++n) {
-            S[n][0] = ex2(fmaf(S[n][0], sl2, -ms0));
-            S[n][1] = ex2(fmaf(S[n][1], sl2, -ms0));
-            S[n][2] = ex2(fmaf(S[n][2], sl2, -ms1));
-            S[n][3] = ex2(fmaf(S[n][3], sl2, -ms1));
-            t0[n] = S[n][0] + S[n][1];
-            t1[n] = S[n][2] + S[n][3];
+            const float2 x0 = __ffma2_rn(make_float2(S[n][0], S[n][1]), sl2v, nm0);
+            const float2 x1 = __ffma2_rn(make_float2(S[n][2], S[n][3]), sl2v, nm1);
+            P[n][0] = ex2_bf16x2(pack_bf16(x0.x, x0.y));
+            P[n][1] = ex2_bf16x2(pack_bf16(x1.x, x1.y));
           }
-#pragma unroll
-          for (int w = NT / 2; w >= 1; w >>= 1)
-#pragma unroll
-            for (int n = 0; n < w; ++n) { t0[n] += t0[n + w]; t1[n] += t1[n + w]; }
-          l[r_][0] = fmaf(l[r_][0], al0, t0[0]);
-          l[r_][1] = fmaf(l[r_][1], al1, t1[0]);
+          l[r_][0] *= al0;
+          l[r_][2] *= al1;
 #pragma unroll
           for (int n = 0; n < NTO; ++n) {
             O[r_][n][0] *= al0; O[r_][n][1] *= al0;
             O[r_][n][2] *= al1; O[r_][n][3] *= al1;
           }
-          // ---- O += P V, the score registers repacked as the A operand ----
+          // ---- O += P V and l += P 1, the weights being the A operand ----
 #pragma unroll
           for (int kk = 0; kk < KSTEP / 16; ++kk) {
-            const uint32_t a0 = pack_bf16(S[2 * kk][0], S[2 * kk][1]);
-            const uint32_t a1 = pack_bf16(S[2 * kk][2], S[2 * kk][3]);
-            const uint32_t a2 = pack_bf16(S[2 * kk + 1][0], S[2 * kk + 1][1]);
-            const uint32_t a3 = pack_bf16(S[2 * kk + 1][2], S[2 * kk + 1][3]);
+            const uint32_t a0 = P[2 * kk][0], a1 = P[2 * kk][1], a2 = P[2 * kk + 1][0], a3 = P[2 * kk + 1][1];
+            mma_k16(l[r_], a0, a1, a2, a3, 0x3F803F80u, 0x3F803F80u);  // B = ones: every column of the result is the row sum
             if constexpr (HD == 8) {
               if constexpr (!HOIST) { if ((kk & 1) == 0) load_v8(kk / 2); }
               mma_k16(O[r_][0], a0, a1, a2, a3, VF[kk][0][0], VF[kk][0][1]);
@@ -305,11 +304,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     for (int r_ = 0; r_ < R; ++r_) {
       const int row0 = (sg * R + r_) * 16;
       if (row0 >= q_real) continue;
-      float l0 = l[r_][0], l1 = l[r_][1];
-      l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
-      l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
-      l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
-      l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+      const float l0 = l[r_][0], l1 = l[r_][2];
       const float inv0 = l0 > 0.f ? 1.f / l0 : 0.f, inv1 = l1 > 0.f ? 1.f / l1 : 0.f;
       const int rowA = row0 + (lane >> 2), rowB = rowA + 8;
 #pragma unroll
