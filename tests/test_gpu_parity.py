@@ -216,3 +216,18 @@ def test_fused_layer_tcgen05_matches_mma_sync_fused_kernels(g, d, heads, d_ff):
     assert np.all(new[pm] == 0.0)
     code, flags = g.last_device_status()
     assert code == 0 and flags == 0
+
+
+@pytest.mark.parametrize("index", [6, 7, 8])
+def test_second_workload_family_attention_and_layer(g, index):
+    """Dataset-statistics lengths (MOSEI averages) and the CH-SIMS / MIntRec segment shapes: projection, all three
+    block patterns and one layer, NaN in the padded rows."""
+    inp = wk.make_inputs(index, batch=6)
+    wl = inp["workload"]
+    _attention_case(g, inp["x"], inp["layer"]["w_qkv"], wl.seg_len, wl.heads, inp["valid_len"], "bf16", nan_padding=True)
+    vl = torch.from_numpy(inp["valid_len"]).cuda()
+    pm = pad_mask(wl.seg_len, inp["valid_len"], 6)
+    xd = to_dev(wk.fill_padding(inp["x"], wl.seg_len, inp["valid_len"], np.nan))
+    y = g.im_layer_fwd(xd, weights_to_dev(inp["layer"], "bf16"), wl.seg_len, wl.heads, vl, oracle.PHASE_INTER_BWD)
+    ref = oracle.im_layer_fwd(inp["x"], inp["layer"], wl.seg_len, wl.heads, inp["valid_len"], oracle.PHASE_INTER_BWD)
+    check_close(to_np64(y), ref, "bf16", pm, f"workload {index} layer")

@@ -287,3 +287,12 @@ def test_workload_generators_are_seeded_and_shaped():
     assert (v5[3] == (64, 512, 512)).all() and (v5[0] == (128, 1024, 1024)).all()
     r = wk.round_to_bf16(np.array([1.0 + 2 ** -8, 1.0 + 3 * 2 ** -8, 1.00390625], np.float32))
     assert r[0] == 1.0 and r[1] == 1.015625 and r[2] == 1.0
+    # second family: lengths around the dataset averages stay inside [1, max]; the other shapes keep the half-length floor
+    v6 = wk.draw_valid_len(np.random.default_rng(1), wk.WORKLOADS[6], 4000)
+    assert (v6 >= 1).all() and (v6 <= (50, 500, 500)).all()
+    assert abs(v6[:, 0].mean() - 24) < 2 and abs(v6[:, 2].mean() - 94) < 6 and v6[:, 1].mean() < 190
+    for idx in (7, 8):
+        w = wk.WORKLOADS[idx]
+        v = wk.draw_valid_len(np.random.default_rng(2), w, 64)
+        assert (v >= (np.asarray(w.seg_len) + 1) // 2).all() and (v <= w.seg_len).all()
+        assert wk.make_inputs(idx, batch=2)["x"].shape == (2, w.L, 64)

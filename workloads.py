@@ -29,9 +29,11 @@ class Workload:
     d_model: int
     heads: int
     raw_dims: tuple | None     # raw feature widths per modality, None = draw X ~ N(0,1) directly
-    padding: str               # "none" | "uniform_half" | "quarter_half"
+    padding: str               # "none" | "uniform_half" | "quarter_half" | "stats"
     d_ff_mult: int = 4
     stack: tuple | None = None  # (n_fwd, n_bwd, n_intra, intra_heads) for the full-stack workload
+    len_mean: tuple | None = None  # "stats" padding: mean and variance of the valid length per segment
+    len_var: tuple | None = None
 
     @property
     def L(self) -> int:
@@ -49,6 +51,15 @@ WORKLOADS = {
     4: Workload(4, "mosei_unaligned_stack", "bf16", 64, (50, 500, 500), 64, 8, (768, 74, 35), "uniform_half",
                 stack=(4, 4, 2, 8)),
     5: Workload(5, "scaled_stress", "bf16", 128, (128, 1024, 1024), 512, 8, None, "quarter_half"),
+    # Second workload family: realistic sparsity and other segment-size ratios (paper, Appendix "Datasets").
+    # 6: MOSEI maxima with valid lengths drawn around the train-split averages 24 / 94 / 149 (text / vision / audio;
+    #    variances 148 / 5115 / 8105) -- far shorter than the maxima, so most key tiles are skipped.
+    6: Workload(6, "mosei_length_stats", "bf16", 32, (50, 500, 500), 64, 8, (768, 74, 35), "stats",
+                len_mean=(24.0, 149.0, 94.0), len_var=(148.0, 8105.0, 5115.0)),
+    # 7: CH-SIMS-shaped maxima 39 / 400 / 55 (text / vision / audio), raw widths 768 / 709 / 33
+    7: Workload(7, "chsims_shaped", "bf16", 32, (39, 55, 400), 64, 8, (768, 33, 709), "uniform_half"),
+    # 8: MIntRec-shaped maxima 30 / 230 / 480 (text / vision / audio), raw widths 768 / 256 / 768
+    8: Workload(8, "mintrec_shaped", "bf16", 32, (30, 480, 230), 64, 8, (768, 768, 256), "uniform_half"),
 }
 
 
@@ -84,6 +95,10 @@ def draw_valid_len(rng: np.random.Generator, wl: Workload, batch: int | None = N
     if wl.padding == "uniform_half":
         lo = (seg + 1) // 2
         return np.stack([rng.integers(lo[m], seg[m] + 1, size=B) for m in range(3)], axis=1).astype(np.int32)
+    if wl.padding == "stats":
+        mean, std = np.asarray(wl.len_mean), np.sqrt(np.asarray(wl.len_var))
+        n = np.rint(rng.normal(mean[None, :], std[None, :], size=(B, 3)))
+        return np.clip(n, 1, seg[None, :]).astype(np.int32)
     if wl.padding == "quarter_half":
         n = np.tile(seg[None, :], (B, 1))
         n[np.arange(B) % 4 == 3] = seg // 2
