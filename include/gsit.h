@@ -123,6 +123,18 @@ gsit_status gsit_im_layer_fwd(const gsit_shape* shape, const gsit_layer_weights*
                               int64_t x_row_stride, float* y, int64_t y_row_stride, void* workspace,
                               size_t workspace_bytes, gsit_stream stream);
 
+/* Read-out of the fusion stack (Eq. "All-Modal-In-One fusion": X_m = f(|| Split(a(G_intra))[-1])): the encoder output is
+ * split by the original modality lengths, the last time step of each modality is taken (with right padding inside a
+ * segment: its last real step; an empty segment contributes zeros), the three vectors are concatenated and the linear
+ * map f is applied.
+ *   shape   batch, seg_len, valid_len and dtype are read (dtype = type of w_f); d_model, heads and phase are ignored
+ *   c       float [B, L, d_c] with row stride c_row_stride elements (>= d_c): the intra encoder's output, d_c = 2 d
+ *   w_f     [out_features, 3 * d_c] row-major in shape->dtype;  b_f float [out_features] or NULL
+ *   out     float [B, out_features] contiguous
+ * Needs 3 * d_c * 4 <= 48 KiB.  Errors as for the other calls. */
+gsit_status gsit_stack_head_fwd(const gsit_shape* shape, const float* c, int64_t c_row_stride, int32_t d_c, const void* w_f,
+                                const float* b_f, float* out, int32_t out_features, gsit_stream stream);
+
 /* gsit_im_layer_fwd for callers that cannot allocate device memory (no counterpart in the paper; it computes
  * exactly what gsit_im_layer_fwd computes).  A host that lives inside someone else's memory budget, that must not
  * risk the implicit device synchronisation of an allocation in a latency-critical loop, or that runs after its

@@ -213,3 +213,29 @@ def gsit_stack_fwd(x, fwd_layers, bwd_layers, intra_layers, seg_len, heads, intr
     for w in intra_layers:
         c = im_layer_fwd(c, w, seg_len, intra_heads, valid_len, PHASE_INTRA, ln_eps=ln_eps)
     return c
+
+
+def stack_head_fwd(c, w_f, b_f, seg_len, valid_len=None) -> np.ndarray:
+    """Read-out of the fusion stack (Eq. "All-Modal-In-One fusion": X_m = f(|| Split(a(G_intra))[-1])): split the
+    encoder output by the original modality lengths, take the last time step of each modality (with right padding inside
+    a segment: its last real step; an empty segment contributes zeros), concatenate the three vectors and apply the
+    linear map f.  c [B, L, dc] -> [B, out_features], w_f [out_features, 3*dc]."""
+    c = _f64(c)
+    w = _f64(w_f)
+    B, L, dc = c.shape
+    assert L == sum(seg_len) and w.shape[1] == 3 * dc
+    out = np.zeros((B, w.shape[0]), dtype=np.float64)
+    for b in range(B):
+        z = np.zeros(3 * dc, dtype=np.float64)
+        off = 0
+        for s in range(3):
+            n = seg_len[s] if valid_len is None else int(min(max(int(valid_len[b][s]), 0), seg_len[s]))
+            if n > 0:
+                z[s * dc:(s + 1) * dc] = c[b, off + n - 1]
+            off += seg_len[s]
+        for o in range(w.shape[0]):
+            acc = 0.0 if b_f is None else float(b_f[o])
+            for i in range(3 * dc):
+                acc += w[o, i] * z[i]
+            out[b, o] = acc
+    return out

@@ -40,7 +40,7 @@ class LayerWeights(ctypes.Structure):
 
 EXPORTS = ("gsit_im_qkv_proj", "gsit_im_attention_fwd", "gsit_im_layer_fwd", "gsit_workspace_bytes",
            "gsit_last_device_status", "gsit_status_string", "gsit_version", "gsit_trace_enable", "gsit_trace_read",
-           "gsit_trace_launches", "gsit_trace_reset", "gsit_tune_attention", "gsit_im_layer_fwd_static")
+           "gsit_trace_launches", "gsit_trace_reset", "gsit_tune_attention", "gsit_im_layer_fwd_static", "gsit_stack_head_fwd")
 STATIC_SCRATCH_BYTES = 4 << 20
 KERNEL_ATTENTION, KERNEL_LINEAR, KERNEL_LAYERNORM = 0, 1, 2
 
@@ -64,6 +64,8 @@ def load():
     lib.gsit_im_layer_fwd.restype = ctypes.c_int
     lib.gsit_im_layer_fwd_static.argtypes = [sp, ctypes.POINTER(LayerWeights), vp, i64, vp, i64, vp]
     lib.gsit_im_layer_fwd_static.restype = ctypes.c_int
+    lib.gsit_stack_head_fwd.argtypes = [sp, vp, i64, ctypes.c_int32, vp, vp, vp, ctypes.c_int32, vp]
+    lib.gsit_stack_head_fwd.restype = ctypes.c_int
     lib.gsit_workspace_bytes.argtypes = [sp, ctypes.c_int, ctypes.c_int32]
     lib.gsit_workspace_bytes.restype = sz
     lib.gsit_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
@@ -225,5 +227,19 @@ def im_layer_fwd_static(x, weights: dict, seg_len, heads, valid_len=None, phase=
         out = torch.empty((B, L, d), dtype=torch.float32, device=x.device)
     assert out.stride(2) == 1 and out.stride(0) == L * out.stride(1)
     _check(load().gsit_im_layer_fwd_static(ctypes.byref(shape), ctypes.byref(lw), _ptr(x), x.stride(1), _ptr(out),
-                                           out.stride(1), _stream()), "gsit_im_layer_fwd_static")
+                                           out.stride(1), _stream()), "gsit_im_layer_fwd_static", "gsit_stack_head_fwd")
+    return out
+
+
+def stack_head_fwd(c, w_f, b_f, seg_len, valid_len=None, out=None):
+    """c float32 [B, L, dc] (row stride free) -> float32 [B, out_features]: the last real step of each modality segment,
+    concatenated, through the linear map w_f [out_features, 3*dc] (float32 or bfloat16) and bias b_f."""
+    B, L, dc = c.shape
+    assert c.is_cuda and c.dtype == torch.float32 and c.stride(2) == 1 and c.stride(0) == L * c.stride(1)
+    assert w_f.is_contiguous() and w_f.shape[1] == 3 * dc
+    shape = make_shape(B, seg_len, 16, 1, valid_len, _dtype_code(w_f.dtype), PHASE_INTRA)
+    if out is None:
+        out = torch.empty((B, w_f.shape[0]), dtype=torch.float32, device=c.device)
+    _check(load().gsit_stack_head_fwd(ctypes.byref(shape), _ptr(c), c.stride(1), dc, _ptr(w_f), _ptr(b_f), _ptr(out),
+                                      w_f.shape[0], _stream()), "gsit_stack_head_fwd")
     return out

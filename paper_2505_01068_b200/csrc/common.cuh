@@ -115,4 +115,8 @@ cudaError_t launch_proj_mlp_tc128(const Geometry& g, const __nv_bfloat16* att, c
 cudaError_t launch_layernorm(const Geometry& g, const float* x, int64_t ldx, const float* gamma, const float* beta,
                              float eps, void* y, int out_bf16, cudaStream_t st);
 
+// Stack read-out: last real step of each segment of c [B, L, dc] (row stride ldc), concatenated, times w^T + bias.
+cudaError_t launch_stack_head(const Geometry& g, int dtype, const float* c, int64_t ldc, int dc, const void* w,
+                              const float* bias, float* out, int n_out, cudaStream_t st);
+
 }  // namespace gsit

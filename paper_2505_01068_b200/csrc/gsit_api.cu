@@ -291,6 +291,20 @@ gsit_status gsit_im_layer_fwd(const gsit_shape* shape, const gsit_layer_weights*
   return run_linear(g, dtype, a, cs);
 }
 
+gsit_status gsit_stack_head_fwd(const gsit_shape* shape, const float* c, int64_t c_row_stride, int32_t d_c, const void* w_f,
+                                const float* b_f, float* out, int32_t out_features, gsit_stream stream) {
+  if (shape == nullptr || !c || !w_f || !out || d_c < 1 || out_features < 1 || c_row_stride < d_c) return GSIT_ERR_INVALID_ARG;
+  gsit_shape sh = *shape;  // only batch, seg_len, valid_len and dtype matter here: make the rest valid
+  sh.d_model = 16; sh.heads = 1; sh.phase = GSIT_PHASE_INTRA;
+  Geometry g;
+  gsit_status st = make_geometry(&sh, &g);
+  if (st != GSIT_OK) return st;
+  if ((size_t)3 * d_c * sizeof(float) > 48 * 1024) return GSIT_ERR_UNSUPPORTED;
+  if (from_cuda(status_ptr(&g.status)) != GSIT_OK) return GSIT_ERR_CUDA;
+  return from_cuda(launch_stack_head(g, shape->dtype, c, c_row_stride, d_c, w_f, b_f, out, out_features,
+                                     static_cast<cudaStream_t>(stream)));
+}
+
 size_t gsit_workspace_bytes(const gsit_shape* shape, int which_call, int32_t d_ff) {
   Geometry g;
   if (make_geometry(shape, &g) != GSIT_OK) return (size_t)-1;

@@ -11,7 +11,9 @@ from . import binding as B
 
 
 class GsitStack:
-    def __init__(self, fwd_layers, bwd_layers, intra_layers, seg_len, heads, intra_heads, ln_eps=1e-5):
+    def __init__(self, fwd_layers, bwd_layers, intra_layers, seg_len, heads, intra_heads, ln_eps=1e-5, head=None):
+        """head: optional (w_f, b_f) of the read-out X_m = f(|| Split(.)[-1]); see read_out()."""
+        self.head = head
         self.fwd, self.bwd, self.intra = list(fwd_layers), list(bwd_layers), list(intra_layers)
         self.seg_len, self.heads, self.intra_heads, self.ln_eps = tuple(seg_len), heads, intra_heads, ln_eps
         self._bufs = None
@@ -50,3 +52,10 @@ class GsitStack:
                            out=dst, workspace=ws)
             cur = dst
         return cur
+
+    def read_out(self, c, valid_len=None):
+        """X_m = f(|| Split(c)[-1]): last real step of each modality of the stack output c [B, L, 2d], through the linear
+        map given as `head` -> float32 [B, out_features] (one gsit_stack_head_fwd call)."""
+        assert self.head is not None, "no read-out weights were given"
+        w_f, b_f = self.head
+        return B.stack_head_fwd(c, w_f, b_f, self.seg_len, valid_len)

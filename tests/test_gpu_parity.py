@@ -231,3 +231,27 @@ def test_second_workload_family_attention_and_layer(g, index):
     y = g.im_layer_fwd(xd, weights_to_dev(inp["layer"], "bf16"), wl.seg_len, wl.heads, vl, oracle.PHASE_INTER_BWD)
     ref = oracle.im_layer_fwd(inp["x"], inp["layer"], wl.seg_len, wl.heads, inp["valid_len"], oracle.PHASE_INTER_BWD)
     check_close(to_np64(y), ref, "bf16", pm, f"workload {index} layer")
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_stack_head_readout(g, dtype):
+    """Last real step of each modality, concatenated, through the linear map f -- against the oracle."""
+    rng = np.random.default_rng(77)
+    seg, B, dc, n_out = (50, 300, 270), 5, 128, 192
+    c = rng.standard_normal((B, sum(seg), dc), dtype=np.float32)
+    w = wk.storage_round(wk.xavier_uniform(rng, n_out, 3 * dc), dtype)
+    bias = (0.1 * rng.standard_normal(n_out)).astype(np.float32)
+    valid = np.array([[50, 300, 270], [1, 150, 270], [25, 0, 1], [50, 1, 135], [13, 299, 200]], dtype=np.int32)
+    vl = torch.from_numpy(valid).cuda()
+    cd = to_dev(wk.fill_padding(c, seg, valid, np.nan))
+    for v_np, v_dev in ((valid, vl), (None, None)):
+        src = cd if v_np is not None else to_dev(c)
+        got = to_np64(g.stack_head_fwd(src, to_dev(w, dtype), to_dev(bias), seg, v_dev))
+        ref = oracle.stack_head_fwd(c, w, bias, seg, v_np)
+        assert np.isfinite(got).all() and np.abs(got - ref).max() <= (1e-4 if dtype == "f32" else 2e-2)
+    # a strided view (the right half of a wider buffer) gives the same result as its contiguous copy
+    wide = torch.zeros((B, sum(seg), 2 * dc), device="cuda")
+    wide[:, :, dc:] = to_dev(c)
+    a = g.stack_head_fwd(wide[:, :, dc:], to_dev(w, dtype), None, seg, vl)
+    b2 = g.stack_head_fwd(to_dev(c), to_dev(w, dtype), None, seg, vl)
+    assert torch.equal(a, b2)

@@ -296,3 +296,22 @@ def test_workload_generators_are_seeded_and_shaped():
         v = wk.draw_valid_len(np.random.default_rng(2), w, 64)
         assert (v >= (np.asarray(w.seg_len) + 1) // 2).all() and (v <= w.seg_len).all()
         assert wk.make_inputs(idx, batch=2)["x"].shape == (2, w.L, 64)
+
+
+def test_stack_head_picks_last_real_step_of_each_modality():
+    """Eq. "All-Modal-In-One fusion", X_m = f(|| Split(.)[-1]): with a selection matrix for f the read-out must return
+    exactly the last real row of each segment; without padding that is the last row of the segment; an empty segment
+    gives zeros; a general f agrees with a matrix product on the gathered rows."""
+    rng = np.random.default_rng(12)
+    seg, B, dc = (4, 7, 5), 3, 6
+    c = rng.standard_normal((B, sum(seg), dc))
+    ident = np.eye(3 * dc)
+    out = oracle.stack_head_fwd(c, ident, None, seg, None)
+    assert np.array_equal(out, np.concatenate([c[:, 3], c[:, 10], c[:, 15]], axis=1))
+    valid = np.array([[4, 7, 5], [1, 3, 2], [2, 0, 5]], dtype=np.int32)
+    out = oracle.stack_head_fwd(c, ident, None, seg, valid)
+    assert np.array_equal(out[1], np.concatenate([c[1, 0], c[1, 4 + 2], c[1, 11 + 1]]))
+    assert np.array_equal(out[2], np.concatenate([c[2, 1], np.zeros(dc), c[2, 15]]))
+    w, bias = rng.standard_normal((9, 3 * dc)), rng.standard_normal(9)
+    got = oracle.stack_head_fwd(c, w, bias, seg, valid)
+    assert np.allclose(got, oracle.stack_head_fwd(c, ident, None, seg, valid) @ w.T + bias, rtol=0, atol=1e-12)
