@@ -40,7 +40,12 @@ constexpr int OFF_Q = 0, OFF_K = OFF_Q + Q_BUFS * Q_BYTES, OFF_V = OFF_K + KV_ST
               OFF_BAR = OFF_V + KV_STAGES * KV_BYTES;
 constexpr int BAR_QFULL = 0, BAR_QEMPTY = 16, BAR_KFULL = 32, BAR_VFULL = 64, BAR_KEMPTY = 96, BAR_VEMPTY = 128,
               BAR_SFULL = 160, BAR_PFULL = 176, BAR_OFINAL = 192, SLOT_TMEM = 200;
-constexpr int TC_SMEM = OFF_BAR + 256 + 1024 /* alignment slack */;
+// Work items are decoded once, by the producer warp, and handed to the other roles through a ring of records in
+// shared memory (the decode needs the sample's valid lengths from global memory and two integer divisions).
+constexpr int ITEM_SLOTS = 8;
+constexpr int OFF_ITEMBAR = OFF_BAR + 256;                      // ITEM_SLOTS "record written" + ITEM_SLOTS "record read" barriers
+constexpr int OFF_ITEMS = OFF_ITEMBAR + 16 * ITEM_SLOTS;        // ITEM_SLOTS records of 16 ints
+constexpr int TC_SMEM = OFF_ITEMS + 64 * ITEM_SLOTS + 1024 /* alignment slack */;
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
@@ -174,6 +179,31 @@ __device__ __forceinline__ void locate(const Geometry& g, const Item& it, int i,
   yrow = it.b * g.L + g.seg_off[r] + t * TK;
 }
 
+// Producer side: lane 0 writes record k of this CTA, then the slot's "written" barrier is released.
+__device__ __forceinline__ void publish_item(uint32_t base, const Item& it, int k, int lane) {
+  if (lane == 0) {
+    const uint32_t a = base + OFF_ITEMS + 64 * (k % ITEM_SLOTS);
+    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(it.b), "r"(it.h), "r"(it.s), "r"(it.q0) : "memory");
+    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(a + 16), "r"(it.rows_in_tile), "r"(it.q_real), "r"(it.T), "r"(it.kn0) : "memory");
+    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(a + 32), "r"(it.kn1), "r"(it.kn2), "r"(it.nk0), "r"(it.nk1) : "memory");
+    mbar_arrive(base + OFF_ITEMBAR + 8 * (k % ITEM_SLOTS));
+  }
+  __syncwarp();
+}
+// Consumer side (whole warp): waits for record k, copies it to registers and releases the slot (one arrival per warp).
+__device__ __forceinline__ Item fetch_item(const Geometry& g, uint32_t base, int k, int lane) {
+  const int slot = k % ITEM_SLOTS;
+  mbar_wait(g, base + OFF_ITEMBAR + 8 * slot, (k / ITEM_SLOTS) & 1);
+  const uint32_t a = base + OFF_ITEMS + 64 * slot;
+  Item it;
+  asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(it.b), "=r"(it.h), "=r"(it.s), "=r"(it.q0) : "r"(a) : "memory");
+  asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(it.rows_in_tile), "=r"(it.q_real), "=r"(it.T), "=r"(it.kn0) : "r"(a + 16) : "memory");
+  asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(it.kn1), "=r"(it.kn2), "=r"(it.nk0), "=r"(it.nk1) : "r"(a + 32) : "memory");
+  __syncwarp();
+  if (lane == 0) mbar_arrive(base + OFF_ITEMBAR + 8 * ITEM_SLOTS + 8 * slot);
+  return it;
+}
+
 __global__ void __launch_bounds__(TC_THREADS, 2)
 attn_tc_hd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                     const __grid_constant__ CUtensorMap tmV, const Geometry g, __nv_bfloat16* __restrict__ out,
@@ -201,6 +231,10 @@ attn_tc_hd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       mbar_init(bars + BAR_VEMPTY + 8 * i, 1);
     }
     mbar_init(bars + BAR_OFINAL, 1);
+    for (int i = 0; i < ITEM_SLOTS; ++i) {
+      mbar_init(base + OFF_ITEMBAR + 8 * i, 1);                   // record written (producer)
+      mbar_init(base + OFF_ITEMBAR + 8 * ITEM_SLOTS + 8 * i, 5);  // record read (MMA warp + four softmax warps)
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -219,8 +253,11 @@ attn_tc_hd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     // ================================ TMA producer ================================
     {
       int n_q = 0, n_kv = 0;  // Q tiles and K/V tiles requested so far (ring positions and phases follow from them)
-      for (int w = blockIdx.x; w < n_items; w += gridDim.x) {
+      int k = 0;              // items of this CTA so far
+      for (int w = blockIdx.x; w < n_items; w += gridDim.x, ++k) {
         const Item it = decode_item(g, w, tiles_per_sample);
+        if (k >= ITEM_SLOTS) mbar_wait(g, base + OFF_ITEMBAR + 8 * ITEM_SLOTS + 8 * (k % ITEM_SLOTS), ((k / ITEM_SLOTS) - 1) & 1);
+        publish_item(base, it, k, lane);
         if (it.T == 0) continue;
         const int qb = n_q & 1, quse = n_q >> 1;
         if (quse > 0) mbar_wait(g, bars + BAR_QEMPTY + 8 * qb, (quse - 1) & 1);
@@ -252,8 +289,9 @@ attn_tc_hd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       constexpr uint32_t IDESC_QK = idesc_bf16(TK, false), IDESC_PV = idesc_bf16(HD64, true);
       int n_q = 0, n_kv = 0;  // Q tiles / key tiles consumed so far.  Key tile n uses S and P buffer n & 1 (phase
                               // (n >> 1) & 1 of their barriers) and ring stage n % KV_STAGES
-      for (int w = blockIdx.x; w < n_items; w += gridDim.x) {
-        const Item it = decode_item(g, w, tiles_per_sample);
+      int k = 0;
+      for (int w = blockIdx.x; w < n_items; w += gridDim.x, ++k) {
+        const Item it = fetch_item(g, base, k, lane);
         if (it.T == 0) continue;
         const int qb = n_q & 1;
         const uint32_t sQb = sQ + qb * Q_BYTES;
@@ -304,8 +342,9 @@ attn_tc_hd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const float2 sl2v = make_float2(sl2, sl2);
     int n_kv = 0, n_items_done = 0;
 
-    for (int w = blockIdx.x; w < n_items; w += gridDim.x) {
-      const Item it = decode_item(g, w, tiles_per_sample);
+    int k = 0;
+    for (int w = blockIdx.x; w < n_items; w += gridDim.x, ++k) {
+      const Item it = fetch_item(g, base, k, lane);
       const int64_t grow = (int64_t)it.b * g.L + g.seg_off[it.s] + it.q0 + r;
       uint4* dst = reinterpret_cast<uint4*>(out + grow * g.d + it.h * HD64);
       float* lse_row = (lse != nullptr) ? lse + ((int64_t)it.b * g.heads + it.h) * g.L + g.seg_off[it.s] + it.q0 + r : nullptr;
