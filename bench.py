@@ -270,11 +270,14 @@ def run_gpu(args):
     _, _, e2e_value = shard.job_throughput(tokens, (time.perf_counter() - t0) / e2e_steps * 1e3, device="cuda")
 
     # ---- per-kernel device times inside the step (eager, CUDA events around each launch) ----
+    # The two rings are issued one after the other here, so that every event pair brackets one kernel running alone.
     trace_steps = max(1, min(args.steps, 10))
+    stack.concurrent_rings = False
     g.trace_enable(True)
     for k in range(trace_steps):
         stack.forward(xbufs[k % nbuf], vl)
     torch.cuda.synchronize()
+    stack.concurrent_rings = True
     att = g.trace_launches(g.KERNEL_ATTENTION)
     lin_ms, lin_n = g.trace_read(g.KERNEL_LINEAR)
     ln_ms, ln_n = g.trace_read(g.KERNEL_LAYERNORM)
@@ -362,7 +365,7 @@ def run_gpu(args):
                    f"intra x{n_i} at d={2 * wl.d_model} (hd={2 * wl.d_model // ih})",
                    "valid_tokens_per_step": tokens, "padded_tokens_per_step": B * wl.L,
                    "l2": f"inputs rotate over {nbuf} device copies ({nbuf * x_host.numel() * 4 >> 20} MiB > 126 MiB L2); "
-                         "the step's scratch alone is larger than L2", "launch": "one CUDA graph per input buffer"},
+                         "the step's scratch alone is larger than L2", "launch": "one CUDA graph per input buffer; the forward and backward rings on two streams inside it"},
         "clocks": clocks.summary(),
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(x_host.numel() * 4),
                 "d2h_bytes_per_step": int(y_host.numel() * 4)},
@@ -370,7 +373,12 @@ def run_gpu(args):
         "roofline": {"kernel": "attn_bf16_kernel<8,64> (cross-modal IM attention inside the step)", "bound": "hbm",
                      "achieved": cross["bytes"] / cross_s / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s",
                      "frac": cross["bytes"] / cross_s / 1e9 / pk["hbm_gbs"], "traffic": ATTN_HD8_DRAM_BYTES, "peak_kind": "of " + pk_kind,
-                     "launch_us": cross_s * 1e6, "algorithmic_bytes": cross["bytes"]},
+                     "launch_us": cross_s * 1e6, "algorithmic_bytes": cross["bytes"],
+                     "timed": "event pair around each launch, rings issued serially for this pass",
+                     # the same launch against the exponential unit: one ex2 per useful (query, key) pair per head
+                     "alu": {"bound": "ex2 (special-function unit)", "achieved": wl.heads * cross["pairs"] / cross_s / 1e9,
+                             "peak": ex2_rate / 1e9, "unit": "Gex2/s", "frac": wl.heads * cross["pairs"] / cross_s / ex2_rate,
+                             "peak_kind": "148 SMs x 16 ex2/clk x max SM clock"}},
         "cpu_baseline": {"value": ref_tokens / cpu_s, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
                          "sample": f"{sub} of {B} samples, one step (valid tokens {ref_tokens}) in {cpu_s:.2f} s"},
         "attention": attention,

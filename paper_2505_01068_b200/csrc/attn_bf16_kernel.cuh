@@ -244,8 +244,8 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           for (int n = 0; n < NT; ++n) {
             const float2 x0 = __ffma2_rn(make_float2(S[n][0], S[n][1]), sl2v, nm0);
             const float2 x1 = __ffma2_rn(make_float2(S[n][2], S[n][3]), sl2v, nm1);
-            P[n][0] = ex2_bf16x2(pack_bf16(x0.x, x0.y));
-            P[n][1] = ex2_bf16x2(pack_bf16(x1.x, x1.y));
+            P[n][0] = pack_bf16(ex2(x0.x), ex2(x0.y));
+            P[n][1] = pack_bf16(ex2(x1.x), ex2(x1.y));
           }
           l[r_][0] *= al0;
           l[r_][2] *= al1;
