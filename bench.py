@@ -249,25 +249,25 @@ def run_gpu(args):
     # whole job: tokens of all ranks over the slowest rank's time (ms is already the maximum over ranks)
     _, _, value = shard.job_throughput(tokens, ms_per_step, device="cuda")
 
-    # ---- end to end: pinned host batch -> device -> stack -> host, every step ----
-    y_host = torch.empty(tuple(y_dev.shape), dtype=torch.float32).pin_memory()
+    # ---- end to end: pinned host batch -> device -> stack -> pinned host result, every step, through the package's
+    # host pipeline (the three legs of neighbouring steps overlap; every step moves its own input and output) ----
+    from paper_2505_01068_b200.hostio import HostPipeline
+    vl_host = torch.from_numpy(valid).pin_memory()
+    y_hosts = [torch.empty((B, wl.L, 2 * wl.d_model), dtype=torch.float32).pin_memory() for _ in range(2)]
+    pipe = HostPipeline(stack, tuple(x_host.shape), depth=2)
     e2e_steps = max(3, min(args.steps, 30))
-
-    def e2e_step():
-        xbufs[0].copy_(x_host, non_blocking=True)
-        graphs[0].replay()
-        y_host.copy_(y_dev, non_blocking=True)
-
-    for _ in range(3):
-        e2e_step()
+    for k in range(3):
+        pipe.step(x_host, y_hosts[k % 2], vl_host)
+    pipe.wait()
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
     t0 = time.perf_counter()
-    for _ in range(e2e_steps):
-        e2e_step()
-    torch.cuda.synchronize()
+    for k in range(e2e_steps):
+        pipe.step(x_host, y_hosts[k % 2], vl_host)
+    pipe.wait()
     _, _, e2e_value = shard.job_throughput(tokens, (time.perf_counter() - t0) / e2e_steps * 1e3, device="cuda")
+    y_host = y_hosts[0]
 
     # ---- per-kernel device times inside the step (eager, CUDA events around each launch) ----
     # The two rings are issued one after the other here, so that every event pair brackets one kernel running alone.
@@ -368,7 +368,8 @@ def run_gpu(args):
                          "the step's scratch alone is larger than L2", "launch": "one CUDA graph per input buffer; the forward and backward rings on two streams inside it"},
         "clocks": clocks.summary(),
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(x_host.numel() * 4),
-                "d2h_bytes_per_step": int(y_host.numel() * 4)},
+                "d2h_bytes_per_step": int(y_host.numel() * 4) ,
+                "how": "HostPipeline, 2 steps in flight: copy-in, kernels and copy-out of neighbouring steps overlap"},
         "gpu_launches": launches_per_step * args.steps,
         "roofline": {"kernel": "attn_bf16_kernel<8,64> (cross-modal IM attention inside the step)", "bound": "hbm",
                      "achieved": cross["bytes"] / cross_s / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s",

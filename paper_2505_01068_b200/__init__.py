@@ -9,5 +9,6 @@ from .binding import (CALL_ATTENTION, CALL_LAYER, CALL_QKV_PROJ, DEVFLAG_CLAMPED
                       status_string, trace_enable, trace_launches, trace_read, tune_attention, version, workspace_bytes,
                       KERNEL_ATTENTION, KERNEL_LINEAR, KERNEL_LAYERNORM)
 from .stack import GsitStack
+from .hostio import HostPipeline
 
 __all__ = [n for n in dir() if not n.startswith("_")]

@@ -233,11 +233,11 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           const float al0 = ex2(fmaf(m[r_][0], sl2, -ms0)), al1 = ex2(fmaf(m[r_][1], sl2, -ms1));
           m[r_][0] = mn0;
           m[r_][1] = mn1;
-          // Exponentials two at a time: one packed FMA forms s * sl2 - m * sl2 for a pair (both <= 0), the pair is
-          // rounded to bf16 (absolute error <= 2^-9 |x|, i.e. negligible where the weight is not) and one packed ex2
-          // yields the two bf16 weights already in the layout of the A operand of P V.  The row sum is taken by the
-          // tensor core from those same bf16 weights (a column of ones appended to V), so numerator and denominator
-          // of the softmax see identical values.
+          // One packed FMA forms s * sl2 - m * sl2 for a pair of scores (both <= 0); each gets its own f32 ex2 (the
+          // packed bf16 form of ex2 issues two special-function operations as well, plus unpacking), and the pair is
+          // rounded once into the bf16x2 layout of the A operand of P V.  The row sum is taken by the tensor core from
+          // those same bf16 weights (a column of ones appended to V), so numerator and denominator of the softmax see
+          // identical values.
           const float2 sl2v = make_float2(sl2, sl2), nm0 = make_float2(-ms0, -ms0), nm1 = make_float2(-ms1, -ms1);
           uint32_t P[NT][2];
 #pragma unroll

@@ -255,3 +255,52 @@ def test_stack_head_readout(g, dtype):
     a = g.stack_head_fwd(wide[:, :, dc:], to_dev(w, dtype), None, seg, vl)
     b2 = g.stack_head_fwd(to_dev(c), to_dev(w, dtype), None, seg, vl)
     assert torch.equal(a, b2)
+
+
+def test_stack_rings_on_two_streams_match_serial_issue(g):
+    """Issuing the forward and backward rings on two streams changes the order of launches, not a single bit."""
+    inp = wk.make_inputs(4, batch=6)
+    wl = inp["workload"]
+    n_f, n_b, n_i, ih = wl.stack
+    vl = torch.from_numpy(inp["valid_len"]).cuda()
+    mk = lambda conc: g.GsitStack([weights_to_dev(w, "bf16") for w in inp["fwd_layers"]],
+                                  [weights_to_dev(w, "bf16") for w in inp["bwd_layers"]],
+                                  [weights_to_dev(w, "bf16") for w in inp["intra_layers"]], wl.seg_len, wl.heads, ih,
+                                  concurrent_rings=conc)
+    x = to_dev(inp["x"])
+    a = mk(True).forward(x, vl).clone()
+    b = mk(False).forward(x, vl).clone()
+    torch.cuda.synchronize()
+    assert torch.equal(a, b)
+    assert g.last_device_status() == (0, 0)
+
+
+def test_host_pipeline_delivers_every_step(g):
+    """Overlapped host->device / kernels / device->host legs: each step's result equals the plain forward of its own
+    input (bit for bit), for more steps than the pipeline is deep, and one of them is held to the oracle."""
+    from paper_2505_01068_b200.hostio import HostPipeline
+    inp = wk.make_inputs(4, batch=3)
+    wl = inp["workload"]
+    n_f, n_b, n_i, ih = wl.stack
+    stack = g.GsitStack([weights_to_dev(w, "bf16") for w in inp["fwd_layers"]],
+                        [weights_to_dev(w, "bf16") for w in inp["bwd_layers"]],
+                        [weights_to_dev(w, "bf16") for w in inp["intra_layers"]], wl.seg_len, wl.heads, ih)
+    rng = np.random.default_rng(5)
+    steps = 5
+    xs = [inp["x"]] + [rng.standard_normal(inp["x"].shape).astype(np.float32) for _ in range(steps - 1)]
+    vs = [inp["valid_len"]] + [wk.draw_valid_len(rng, wl, 3) for _ in range(steps - 1)]
+    x_host = [torch.from_numpy(x).pin_memory() for x in xs]
+    v_host = [torch.from_numpy(v).pin_memory() for v in vs]
+    y_host = [torch.empty((3, wl.L, 2 * wl.d_model), dtype=torch.float32).pin_memory() for _ in range(steps)]
+    pipe = HostPipeline(stack, inp["x"].shape, depth=2)
+    for i in range(steps):
+        pipe.step(x_host[i], y_host[i], v_host[i])
+    pipe.wait()
+    for i in range(steps):
+        want = stack.forward(x_host[i].cuda(), v_host[i].cuda())
+        torch.cuda.synchronize()
+        assert torch.equal(want.cpu(), y_host[i]), i
+    ref = oracle.gsit_stack_fwd(xs[0], inp["fwd_layers"], inp["bwd_layers"], inp["intra_layers"], wl.seg_len, wl.heads, ih, vs[0])
+    err = np.abs(y_host[0].numpy().astype(np.float64) - ref)
+    assert err.max() <= 10 * 2e-2 and err.mean() <= 10 * 2e-3, (err.max(), err.mean())
+    assert g.last_device_status() == (0, 0)
