@@ -16,33 +16,52 @@ from . import binding as B
 
 class GsitStack:
     def __init__(self, fwd_layers, bwd_layers, intra_layers, seg_len, heads, intra_heads, ln_eps=1e-5, head=None,
-                 concurrent_rings=True):
+                 concurrent_rings=True, batch_chunks=1):
         """head: optional (w_f, b_f) of the read-out X_m = f(|| Split(.)[-1]); see read_out().
-        concurrent_rings: issue the forward and the backward ring on two streams (False: one after the other)."""
+        concurrent_rings: issue independent work on several streams (False: every launch on the caller's stream, whole
+        batch per launch).  batch_chunks: with concurrent issue, the batch is cut into this many groups of samples, each
+        with its own pair of streams; samples never interact, so the result does not depend on it.  (At B = 64, L = 1050
+        one chunk is fastest: the persistent fused kernels pay their per-CTA set-up once per launch.)"""
         self.head = head
         self.concurrent_rings = concurrent_rings
-        self._side = None  # second stream and fork/join events, created on first use
+        self.batch_chunks = max(1, int(batch_chunks))
         self.fwd, self.bwd, self.intra = list(fwd_layers), list(bwd_layers), list(intra_layers)
         self.seg_len, self.heads, self.intra_heads, self.ln_eps = tuple(seg_len), heads, intra_heads, ln_eps
         self._bufs = None
+        self._lanes = None  # streams and events of the concurrent issue, created on first use
+
+    def _chunks(self, Bn):
+        nch = min(self.batch_chunks, Bn) if (self.concurrent_rings and self.fwd and self.bwd) else 1
+        q, r = divmod(Bn, nch)
+        out, lo = [], 0
+        for c in range(nch):
+            hi = lo + q + (1 if c < r else 0)
+            out.append(slice(lo, hi))
+            lo = hi
+        return out
 
     def _buffers(self, x, valid_len):
         Bn, L, d = x.shape
-        key = (Bn, L, d, x.device)
-        if self._bufs is None or self._bufs[0] != key:
+        chunks = self._chunks(Bn)
+        key = (Bn, L, d, x.device, len(chunks))
+        if self._bufs is None:
+            self._bufs = {}
+        if key not in self._bufs:
             code = B._dtype_code(self.fwd[0]["w_qkv"].dtype)
-            sh1 = B.make_shape(Bn, self.seg_len, d, self.heads, valid_len, code, B.PHASE_INTER_FWD)
-            sh2 = B.make_shape(Bn, self.seg_len, 2 * d, self.intra_heads, valid_len, code, B.PHASE_INTRA)
-            need = B.workspace_bytes(sh1, B.CALL_LAYER, self.fwd[0]["w_1"].shape[0])
-            if self.intra:
-                need = max(need, B.workspace_bytes(sh2, B.CALL_LAYER, self.intra[0]["w_1"].shape[0]))
+            ws = []
+            for sl in chunks:  # two workspaces per chunk of the batch: one per ring (the intra encoder reuses the first)
+                n = sl.stop - sl.start
+                vl = None if valid_len is None else valid_len[sl]
+                sh1 = B.make_shape(n, self.seg_len, d, self.heads, vl, code, B.PHASE_INTER_FWD)
+                need = B.workspace_bytes(sh1, B.CALL_LAYER, self.fwd[0]["w_1"].shape[0])
+                if self.intra:
+                    sh2 = B.make_shape(n, self.seg_len, 2 * d, self.intra_heads, vl, code, B.PHASE_INTRA)
+                    need = max(need, B.workspace_bytes(sh2, B.CALL_LAYER, self.intra[0]["w_1"].shape[0]))
+                ws.append([torch.empty(need, dtype=torch.uint8, device=x.device) for _ in range(2)])
             f32 = dict(dtype=torch.float32, device=x.device)
-            self._bufs = (key, torch.empty(need, dtype=torch.uint8, device=x.device),
-                          torch.empty((Bn, L, d), **f32), torch.empty((Bn, L, d), **f32),
-                          torch.empty((Bn, L, 2 * d), **f32), torch.empty((Bn, L, 2 * d), **f32),
-                          torch.empty(need, dtype=torch.uint8, device=x.device),
-                          torch.empty((Bn, L, d), **f32), torch.empty((Bn, L, d), **f32))
-        return self._bufs[1:]
+            self._bufs[key] = (ws, [torch.empty((Bn, L, d), **f32) for _ in range(4)],
+                               torch.empty((Bn, L, 2 * d), **f32), torch.empty((Bn, L, 2 * d), **f32))
+        return (chunks,) + self._bufs[key]
 
     def _ring(self, x, layers, phase, half, c0, ws, ping, valid_len):
         d = x.shape[2]
@@ -52,34 +71,50 @@ class GsitStack:
             B.im_layer_fwd(cur, w, self.seg_len, self.heads, valid_len, phase, ln_eps=self.ln_eps, out=dst, workspace=ws)
             cur = dst
 
-    def forward(self, x, valid_len=None):
-        """x float32 [B, L, d] -> float32 [B, L, 2d].  The result lives in a buffer owned by this object."""
-        ws, t0, t1, c0, c1, ws_b, u0, u1 = self._buffers(x, valid_len)
-        if self.concurrent_rings and self.fwd and self.bwd:
-            if self._side is None:
-                self._side = (torch.cuda.Stream(device=x.device), torch.cuda.Event(), torch.cuda.Event())
-            side, fork, join = self._side
-            main = torch.cuda.current_stream(x.device)
-            fork.record(main)
-            side.wait_event(fork)
-            with torch.cuda.stream(side):
-                self._ring(x, self.bwd, B.PHASE_INTER_BWD, 1, c0, ws_b, [u0, u1], valid_len)
-                join.record(side)
-            x.record_stream(side)
-            if valid_len is not None:
-                valid_len.record_stream(side)
-            self._ring(x, self.fwd, B.PHASE_INTER_FWD, 0, c0, ws, [t0, t1], valid_len)
-            main.wait_event(join)
-        else:
-            self._ring(x, self.fwd, B.PHASE_INTER_FWD, 0, c0, ws, [t0, t1], valid_len)
-            self._ring(x, self.bwd, B.PHASE_INTER_BWD, 1, c0, ws, [t0, t1], valid_len)
+    def _intra(self, c0, c1, ws, valid_len):
         cur, ping = c0, [c1, c0]
         for i, w in enumerate(self.intra):
             dst = ping[i % 2]
             B.im_layer_fwd(cur, w, self.seg_len, self.intra_heads, valid_len, B.PHASE_INTRA, ln_eps=self.ln_eps,
                            out=dst, workspace=ws)
             cur = dst
-        return cur
+        return len(self.intra) % 2  # 1: the result is in c1, 0: in c0
+
+    def forward(self, x, valid_len=None):
+        """x float32 [B, L, d] -> float32 [B, L, 2d].  The result lives in a buffer owned by this object."""
+        chunks, ws, t, c0, c1 = self._buffers(x, valid_len)
+        if len(chunks) == 1 and not (self.concurrent_rings and self.fwd and self.bwd):
+            self._ring(x, self.fwd, B.PHASE_INTER_FWD, 0, c0, ws[0][0], t[0:2], valid_len)
+            self._ring(x, self.bwd, B.PHASE_INTER_BWD, 1, c0, ws[0][0], t[0:2], valid_len)
+            return c1 if self._intra(c0, c1, ws[0][0], valid_len) else c0
+        nch = len(chunks)
+        if self._lanes is None or len(self._lanes[0]) != 2 * nch:
+            dev = x.device
+            self._lanes = ([torch.cuda.Stream(device=dev) for _ in range(2 * nch)], torch.cuda.Event(),
+                           [torch.cuda.Event() for _ in range(2 * nch)])
+        streams, fork, done = self._lanes
+        main = torch.cuda.current_stream(x.device)
+        fork.record(main)
+        for c, sl in enumerate(chunks):
+            vl = None if valid_len is None else valid_len[sl]
+            s_f, s_b = streams[2 * c], streams[2 * c + 1]
+            s_f.wait_event(fork)
+            s_b.wait_event(fork)
+            with torch.cuda.stream(s_b):
+                self._ring(x[sl], self.bwd, B.PHASE_INTER_BWD, 1, c0[sl], ws[c][1], [t[2][sl], t[3][sl]], vl)
+                done[2 * c + 1].record(s_b)
+            with torch.cuda.stream(s_f):
+                self._ring(x[sl], self.fwd, B.PHASE_INTER_FWD, 0, c0[sl], ws[c][0], [t[0][sl], t[1][sl]], vl)
+                s_f.wait_event(done[2 * c + 1])  # both rings of this chunk are complete
+                which = self._intra(c0[sl], c1[sl], ws[c][0], vl)
+                done[2 * c].record(s_f)
+        for c in range(nch):
+            main.wait_event(done[2 * c])
+        for st in streams:
+            x.record_stream(st)
+            if valid_len is not None:
+                valid_len.record_stream(st)
+        return c1 if which else c0
 
     def read_out(self, c, valid_len=None):
         """X_m = f(|| Split(c)[-1]): last real step of each modality of the stack output c [B, L, 2d], through the linear

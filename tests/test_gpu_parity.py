@@ -263,15 +263,16 @@ def test_stack_rings_on_two_streams_match_serial_issue(g):
     wl = inp["workload"]
     n_f, n_b, n_i, ih = wl.stack
     vl = torch.from_numpy(inp["valid_len"]).cuda()
-    mk = lambda conc: g.GsitStack([weights_to_dev(w, "bf16") for w in inp["fwd_layers"]],
-                                  [weights_to_dev(w, "bf16") for w in inp["bwd_layers"]],
-                                  [weights_to_dev(w, "bf16") for w in inp["intra_layers"]], wl.seg_len, wl.heads, ih,
-                                  concurrent_rings=conc)
+    mk = lambda conc, chunks=1: g.GsitStack([weights_to_dev(w, "bf16") for w in inp["fwd_layers"]],
+                                            [weights_to_dev(w, "bf16") for w in inp["bwd_layers"]],
+                                            [weights_to_dev(w, "bf16") for w in inp["intra_layers"]], wl.seg_len, wl.heads,
+                                            ih, concurrent_rings=conc, batch_chunks=chunks)
     x = to_dev(inp["x"])
     a = mk(True).forward(x, vl).clone()
     b = mk(False).forward(x, vl).clone()
+    c = mk(True, 4).forward(x, vl).clone()  # the batch cut into groups of samples (6 -> 2, 2, 1, 1), each on its own streams
     torch.cuda.synchronize()
-    assert torch.equal(a, b)
+    assert torch.equal(a, b) and torch.equal(a, c)
     assert g.last_device_status() == (0, 0)
 
 
