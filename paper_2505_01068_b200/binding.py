@@ -227,7 +227,7 @@ def im_layer_fwd_static(x, weights: dict, seg_len, heads, valid_len=None, phase=
         out = torch.empty((B, L, d), dtype=torch.float32, device=x.device)
     assert out.stride(2) == 1 and out.stride(0) == L * out.stride(1)
     _check(load().gsit_im_layer_fwd_static(ctypes.byref(shape), ctypes.byref(lw), _ptr(x), x.stride(1), _ptr(out),
-                                           out.stride(1), _stream()), "gsit_im_layer_fwd_static", "gsit_stack_head_fwd")
+                                           out.stride(1), _stream()), "gsit_im_layer_fwd_static")
     return out
 
 
