@@ -271,8 +271,11 @@ def test_stack_rings_on_two_streams_match_serial_issue(g):
     a = mk(True).forward(x, vl).clone()
     b = mk(False).forward(x, vl).clone()
     c = mk(True, 4).forward(x, vl).clone()  # the batch cut into groups of samples (6 -> 2, 2, 1, 1), each on its own streams
+    st = mk(True)
+    st.intra_halves = False                 # intra encoder on the whole batch instead of one half per stream
+    d = st.forward(x, vl).clone()
     torch.cuda.synchronize()
-    assert torch.equal(a, b) and torch.equal(a, c)
+    assert torch.equal(a, b) and torch.equal(a, c) and torch.equal(a, d)
     assert g.last_device_status() == (0, 0)
 
 
