@@ -61,3 +61,22 @@ def test_single_process_and_slices_cover_every_batch():
         for world in (1, 2, 3, 8):
             idx = [i for r in range(world) for i in range(batch)[shard.batch_slice(batch, world, r)]]
             assert idx == list(range(batch))
+
+
+def test_stack_chunks_tile_the_batch():
+    """Host logic of the stack's concurrent issue: the groups of samples cover the batch once, in order, balanced, and
+    collapse to one group when everything is issued on the caller's stream."""
+    from paper_2505_01068_b200.stack import GsitStack
+
+    layer = [{}]
+    for batch in (1, 2, 5, 64):
+        for chunks in (1, 2, 3, 8):
+            st = GsitStack(layer, layer, layer, (4, 4, 4), 2, 2, batch_chunks=chunks)
+            sl = st._chunks(batch)
+            assert len(sl) == min(chunks, batch)
+            assert sl[0].start == 0 and sl[-1].stop == batch
+            assert all(a.stop == b.start for a, b in zip(sl, sl[1:]))
+            sizes = [s.stop - s.start for s in sl]
+            assert max(sizes) - min(sizes) <= 1 and min(sizes) >= 1
+            st.concurrent_rings = False
+            assert st._chunks(batch) == [slice(0, batch)]
