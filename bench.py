@@ -229,6 +229,8 @@ def run_gpu(args):
     xbufs = [x_host.cuda() for _ in range(nbuf)]
     # per layer: LN1+QKV, IM attention, out-proj+LN2+MLP (fused kernels); each intra layer once per half of the batch
     launches_per_step = 3 * (n_f + n_b) + 3 * n_i * (2 if (stack.intra_halves and B >= 2) else 1)
+    if stack.packed:
+        launches_per_step += 3   # row plan, gather of the real rows, scatter of the result
 
     for i in range(max(1, min(args.warmup, 2))):           # eager warm-up (module load, attributes, buffers)
         stack.forward(xbufs[i % nbuf], vl)
@@ -368,7 +370,7 @@ def run_gpu(args):
                    "valid_tokens_per_step": tokens, "padded_tokens_per_step": B * wl.L,
                    "l2": f"inputs rotate over {nbuf} device copies ({nbuf * x_host.numel() * 4 >> 20} MiB > 126 MiB L2); "
                          "the step's scratch alone is larger than L2", "launch": "one CUDA graph per input buffer; inside it the forward and backward rings on two streams, then the "
-                             "intra encoder on the two halves of the batch on the same two streams"},
+                             "intra encoder on the two halves of the batch on the same two streams; packed row layout (real rows only)"},
         "clocks": clocks.summary(),
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(x_host.numel() * 4),
                 "d2h_bytes_per_step": int(y_host.numel() * 4) ,

@@ -75,6 +75,15 @@ typedef struct gsit_shape {
   int32_t phase;            /* gsit_phase */
   uint32_t custom_mask;     /* used when phase == GSIT_PHASE_CUSTOM */
   float scale;              /* score scale; <= 0 selects 1/sqrt(head_dim) */
+  /* Packed row layout (optional; NULL selects the padded [B, L] layout described with each call).  The paper's
+   * Decomposition drops padded positions from the computation; in the packed layout they do not exist in memory
+   * either: activations are [packed_capacity, d] matrices of real rows, segment s of sample b at rows
+   * row_start[3 b + s] .. + valid_len[b][s] - 1.  row_start is a DEVICE int32 array of 3 B + 1 entries written by
+   * gsit_plan_rows (entry 3 B = the row after the last one); valid_len must be given.  Accepted by
+   * gsit_im_attention_fwd (bf16, head_dim 8 / 16 / 32) and gsit_im_layer_fwd (bf16, d_model 64 or 128); other
+   * calls and shapes answer GSIT_ERR_UNSUPPORTED. */
+  const int32_t* row_start;
+  int32_t packed_capacity;  /* rows of the packed matrices (>= the plan's last entry rounded up to 128) */
 } gsit_shape;
 
 /* Weights of one IM encoder layer (HOST struct of DEVICE pointers).  Matrices are [out_features,
@@ -122,6 +131,25 @@ gsit_status gsit_im_attention_fwd(const gsit_shape* shape, const void* q, const 
 gsit_status gsit_im_layer_fwd(const gsit_shape* shape, const gsit_layer_weights* weights, const float* x,
                               int64_t x_row_stride, float* y, int64_t y_row_stride, void* workspace,
                               size_t workspace_bytes, gsit_stream stream);
+
+/* Packed row layout, the three helpers (Section "Inner Decomposition for Efficiency": padded positions take no part in
+ * the computation; here they take no memory either).  All run on the device, asynchronously on `stream`, and need no
+ * host knowledge of the lengths, so a captured sequence of calls stays valid when valid_len changes.
+ *
+ * gsit_plan_rows: row_start[3 b + s] = running sum of the (clamped) valid lengths in the order (b, s), row_start[3 B] =
+ *   their total.  If 0 < split_sample < B, the first row of sample split_sample is rounded up to a multiple of 128, so that
+ *   the samples before and after it can be processed by separate calls (shape->batch and the valid_len / row_start
+ *   pointers advanced) whose 128-row tiles do not touch each other's rows.
+ *   shape: batch, seg_len, valid_len (required) are read.  row_start: DEVICE int32 [3 B + 1].
+ * gsit_pack_rows: x_packed[row_start[3 b + s] + i, :] = x[b, seg_off[s] + i, :] for i < valid_len[b][s].
+ * gsit_unpack_rows: the inverse; padded positions of y are written as +0.
+ *   x / y float [B, L, cols] with the given row strides (elements); the packed matrices are float [capacity, cols].
+ * A capacity of B * L + 128 rows always suffices. */
+gsit_status gsit_plan_rows(const gsit_shape* shape, int32_t split_sample, int32_t* row_start, gsit_stream stream);
+gsit_status gsit_pack_rows(const gsit_shape* shape, const float* x, int64_t x_row_stride, float* x_packed,
+                           int64_t packed_row_stride, int32_t cols, gsit_stream stream);
+gsit_status gsit_unpack_rows(const gsit_shape* shape, const float* y_packed, int64_t packed_row_stride, float* y,
+                             int64_t y_row_stride, int32_t cols, gsit_stream stream);
 
 /* Read-out of the fusion stack (Eq. "All-Modal-In-One fusion": X_m = f(|| Split(a(G_intra))[-1])): the encoder output is
  * split by the original modality lengths, the last time step of each modality is taken (with right padding inside a

@@ -29,7 +29,8 @@ class GsitError(RuntimeError):
 class Shape(ctypes.Structure):
     _fields_ = [("batch", ctypes.c_int32), ("seg_len", ctypes.c_int32 * 3), ("d_model", ctypes.c_int32),
                 ("heads", ctypes.c_int32), ("valid_len", ctypes.c_void_p), ("dtype", ctypes.c_int32),
-                ("phase", ctypes.c_int32), ("custom_mask", ctypes.c_uint32), ("scale", ctypes.c_float)]
+                ("phase", ctypes.c_int32), ("custom_mask", ctypes.c_uint32), ("scale", ctypes.c_float),
+                ("row_start", ctypes.c_void_p), ("packed_capacity", ctypes.c_int32)]
 
 
 class LayerWeights(ctypes.Structure):
@@ -40,7 +41,8 @@ class LayerWeights(ctypes.Structure):
 
 EXPORTS = ("gsit_im_qkv_proj", "gsit_im_attention_fwd", "gsit_im_layer_fwd", "gsit_workspace_bytes",
            "gsit_last_device_status", "gsit_status_string", "gsit_version", "gsit_trace_enable", "gsit_trace_read",
-           "gsit_trace_launches", "gsit_trace_reset", "gsit_tune_attention", "gsit_im_layer_fwd_static", "gsit_stack_head_fwd")
+           "gsit_trace_launches", "gsit_trace_reset", "gsit_tune_attention", "gsit_im_layer_fwd_static", "gsit_stack_head_fwd",
+           "gsit_plan_rows", "gsit_pack_rows", "gsit_unpack_rows")
 STATIC_SCRATCH_BYTES = 4 << 20
 KERNEL_ATTENTION, KERNEL_LINEAR, KERNEL_LAYERNORM = 0, 1, 2
 
@@ -66,6 +68,11 @@ def load():
     lib.gsit_im_layer_fwd_static.restype = ctypes.c_int
     lib.gsit_stack_head_fwd.argtypes = [sp, vp, i64, ctypes.c_int32, vp, vp, vp, ctypes.c_int32, vp]
     lib.gsit_stack_head_fwd.restype = ctypes.c_int
+    lib.gsit_plan_rows.argtypes = [sp, ctypes.c_int32, vp, vp]
+    lib.gsit_plan_rows.restype = ctypes.c_int
+    for fn in (lib.gsit_pack_rows, lib.gsit_unpack_rows):
+        fn.argtypes = [sp, vp, i64, vp, i64, ctypes.c_int32, vp]
+        fn.restype = ctypes.c_int
     lib.gsit_workspace_bytes.argtypes = [sp, ctypes.c_int, ctypes.c_int32]
     lib.gsit_workspace_bytes.restype = sz
     lib.gsit_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
@@ -103,12 +110,18 @@ def _dtype_code(t: torch.dtype) -> int:
     raise TypeError(f"unsupported dtype {t}")
 
 
-def make_shape(batch, seg_len, d_model, heads, valid_len, dtype_code, phase, custom_mask=0, scale=0.0) -> Shape:
+def make_shape(batch, seg_len, d_model, heads, valid_len, dtype_code, phase, custom_mask=0, scale=0.0,
+               row_start=None, capacity=0) -> Shape:
+    """row_start (int32 device tensor of >= 3 * batch + 1 entries, from plan_rows) selects the packed row layout with
+    `capacity` rows."""
     if valid_len is not None:
         assert valid_len.is_cuda and valid_len.dtype == torch.int32 and valid_len.is_contiguous()
         assert tuple(valid_len.shape) == (batch, 3)
+    if row_start is not None:
+        assert row_start.is_cuda and row_start.dtype == torch.int32 and row_start.is_contiguous()
+        assert row_start.numel() >= 3 * batch + 1 and valid_len is not None and capacity >= 1
     return Shape(int(batch), (ctypes.c_int32 * 3)(*[int(s) for s in seg_len]), int(d_model), int(heads),
-                 _ptr(valid_len), int(dtype_code), int(phase), int(custom_mask), float(scale))
+                 _ptr(valid_len), int(dtype_code), int(phase), int(custom_mask), float(scale), _ptr(row_start), int(capacity))
 
 
 def _check(code: int, what: str):
@@ -183,6 +196,43 @@ def im_attention_fwd(q, k, v, seg_len, valid_len=None, phase=PHASE_INTER_FWD, cu
     return (out, lse) if want_lse else out
 
 
+def plan_rows(valid_len, seg_len, split_sample=0, out=None):
+    """Packed row layout: int32 device tensor of 3 B + 1 entries, entry 3 b + s = first packed row of segment s of sample
+    b, entry 3 B = rows in use.  split_sample > 0 starts that sample on a multiple of 128 rows.  Runs on the device."""
+    Bn = valid_len.shape[0]
+    shape = make_shape(Bn, seg_len, 16, 1, valid_len, DTYPE_F32, PHASE_INTRA)
+    if out is None:
+        out = torch.empty(3 * Bn + 1, dtype=torch.int32, device=valid_len.device)
+    assert out.is_cuda and out.dtype == torch.int32 and out.is_contiguous() and out.numel() >= 3 * Bn + 1
+    _check(load().gsit_plan_rows(ctypes.byref(shape), int(split_sample), _ptr(out), _stream()), "gsit_plan_rows")
+    return out
+
+
+def _move_rows(fn_name, padded, packed, seg_len, valid_len, row_start):
+    Bn, L, cols = padded.shape
+    for t in (padded, packed):
+        assert t.is_cuda and t.dtype == torch.float32 and t.stride(-1) == 1
+    assert padded.stride(0) == L * padded.stride(1) and packed.dim() == 2 and packed.shape[1] == cols
+    shape = make_shape(Bn, seg_len, 16, 1, valid_len, DTYPE_F32, PHASE_INTRA, row_start=row_start, capacity=packed.shape[0])
+    fn = getattr(load(), fn_name)
+    if fn_name == "gsit_pack_rows":
+        _check(fn(ctypes.byref(shape), _ptr(padded), padded.stride(1), _ptr(packed), packed.stride(0), cols, _stream()), fn_name)
+    else:
+        _check(fn(ctypes.byref(shape), _ptr(packed), packed.stride(0), _ptr(padded), padded.stride(1), cols, _stream()), fn_name)
+
+
+def pack_rows(x, x_packed, seg_len, valid_len, row_start):
+    """x float32 [B, L, cols] -> the real rows, in x_packed float32 [capacity, cols] at the rows the plan gives."""
+    _move_rows("gsit_pack_rows", x, x_packed, seg_len, valid_len, row_start)
+    return x_packed
+
+
+def unpack_rows(y_packed, y, seg_len, valid_len, row_start):
+    """The inverse of pack_rows; padded positions of y float32 [B, L, cols] become +0."""
+    _move_rows("gsit_unpack_rows", y, y_packed, seg_len, valid_len, row_start)
+    return y
+
+
 _W_KEYS = ("ln1_g", "ln1_b", "w_qkv", "b_qkv", "w_o", "b_o", "ln2_g", "ln2_b", "w_1", "b_1", "w_2", "b_2")
 
 
@@ -196,13 +246,26 @@ def make_layer_weights(w: dict, ln_eps: float = 1e-5) -> LayerWeights:
 
 
 def im_layer_fwd(x, weights: dict, seg_len, heads, valid_len=None, phase=PHASE_INTER_FWD, custom_mask=0, scale=0.0,
-                 ln_eps=1e-5, out=None, workspace=None):
-    """x float32 [B, L, d] (row stride free) -> y float32 [B, L, d]; weights in bf16 or float32 select the path."""
+                 ln_eps=1e-5, out=None, workspace=None, row_start=None):
+    """x float32 [B, L, d] (row stride free) -> y float32 [B, L, d]; weights in bf16 or float32 select the path.
+    With row_start (from plan_rows) x and out are packed matrices [capacity, d] (row stride free) and the batch size is
+    that of valid_len."""
+    code = _dtype_code(weights["w_qkv"].dtype)
+    lw = make_layer_weights(weights, ln_eps)
+    if row_start is not None:
+        cap, d = x.shape
+        assert x.is_cuda and x.dtype == torch.float32 and x.stride(1) == 1 and out is not None and out.shape[0] == cap
+        assert out.stride(1) == 1
+        shape = make_shape(valid_len.shape[0], seg_len, d, heads, valid_len, code, phase, custom_mask, scale, row_start, cap)
+        need = workspace_bytes(shape, CALL_LAYER, lw.d_ff)
+        if workspace is None:
+            workspace = torch.empty(need, dtype=torch.uint8, device=x.device)
+        _check(load().gsit_im_layer_fwd(ctypes.byref(shape), ctypes.byref(lw), _ptr(x), x.stride(0), _ptr(out),
+                                        out.stride(0), _ptr(workspace), workspace.numel(), _stream()), "gsit_im_layer_fwd")
+        return out
     B, L, d = x.shape
     assert x.is_cuda and x.dtype == torch.float32 and x.stride(2) == 1 and x.stride(0) == L * x.stride(1)
-    code = _dtype_code(weights["w_qkv"].dtype)
     shape = make_shape(B, seg_len, d, heads, valid_len, code, phase, custom_mask, scale)
-    lw = make_layer_weights(weights, ln_eps)
     if out is None:
         out = torch.empty((B, L, d), dtype=torch.float32, device=x.device)
     assert out.stride(2) == 1 and out.stride(0) == L * out.stride(1)

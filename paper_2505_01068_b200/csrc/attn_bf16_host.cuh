@@ -8,7 +8,7 @@ template <typename C>
 cudaError_t launch_one(const Geometry& g, const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
                        int64_t row_stride, __nv_bfloat16* out, float* lse, float scale, cudaStream_t st) {
   constexpr int CW = C::CW;
-  const int64_t rows = (int64_t)g.batch * g.L;
+  const int64_t rows = matrix_rows(g);
   alignas(64) CUtensorMap tmQ, tmK, tmV;
   if (!make_map(&tmQ, q, rows, g.d, row_stride, CW, C::QT) || !make_map(&tmK, k, rows, g.d, row_stride, CW, KT) ||
       !make_map(&tmV, v, rows, g.d, row_stride, CW, KT))

@@ -39,26 +39,28 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     if (tile >= nts) { tile -= nts; s = (seg_order >> (2 * rank + 2)) & 3; }
   }
   const int q0 = tile * QT;
-  const int rows_in_tile = min(QT, g.seg_len[s] - q0);
   const int cs = blockIdx.y;
-  const int q_real_all = max(0, min(rows_in_tile, valid_rows(g, b, s) - q0));
+  const int q_real_all = max(0, min(min(QT, g.seg_len[s] - q0), valid_rows(g, b, s) - q0));
+  // rows of the tile this CTA writes: in the padded layout all that belong to the segment (padding as +0); in the packed
+  // layout only the real ones exist -- what follows them in memory is another segment
+  const bool packed = g.row_start != nullptr;
+  const int rows_in_tile = packed ? q_real_all : min(QT, g.seg_len[s] - q0);
   const int kn0 = ((g.allowed >> (3 * s + 0)) & 1u) ? valid_rows(g, b, 0) : 0;
   const int kn1 = ((g.allowed >> (3 * s + 1)) & 1u) ? valid_rows(g, b, 1) : 0;
   const int kn2 = ((g.allowed >> (3 * s + 2)) & 1u) ? valid_rows(g, b, 2) : 0;
   const int nk0 = (kn0 + KT - 1) / KT, nk1 = (kn1 + KT - 1) / KT, nk2 = (kn2 + KT - 1) / KT;
   const int T = (q_real_all > 0) ? nk0 + nk1 + nk2 : 0;  // key tiles this CTA walks
   const int q_real = (T > 0) ? q_real_all : 0;           // rows that receive a computed result
-  const int64_t grow0 = (int64_t)b * g.L + g.seg_off[s] + q0;  // first global row of the tile
+  const int64_t grow0 = (int64_t)seg_row0(g, b, s) + q0;  // first row of the tile in the activation matrices
   const int xcol = cs * CW;
-  const int off1 = g.seg_off[1], off2 = g.seg_off[2];
+  const int kbase0 = seg_row0(g, b, 0), kbase1 = seg_row0(g, b, 1), kbase2 = seg_row0(g, b, 2);
 
   auto locate = [&](int i, int& krem, int& yrow) {
     int t = i, r = 0;
     if (t >= nk0) { t -= nk0; r = 1; if (t >= nk1) { t -= nk1; r = 2; } }
     const int kn = (r == 0) ? kn0 : (r == 1) ? kn1 : kn2;
-    const int off = (r == 0) ? 0 : (r == 1) ? off1 : off2;
     krem = kn - t * KT;
-    yrow = b * g.L + off + t * KT;
+    yrow = ((r == 0) ? kbase0 : (r == 1) ? kbase1 : kbase2) + t * KT;
   };
   auto issue = [&](int i) {  // one thread: TMA loads of key tile i into its stage
     int krem, yrow;

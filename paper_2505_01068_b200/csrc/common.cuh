@@ -16,6 +16,10 @@ struct Geometry {
   uint32_t allowed;          // bit (3*s + r): query segment s may attend key segment r
   const int32_t* valid_len;  // device [B][3] or nullptr
   unsigned int* status;      // device status word (GSIT_DEVFLAG_* bits), one per device
+  // Packed row layout (nullptr = padded [B, L] layout): device int32 [3 B + 1]; entry 3 b + s is the first row of
+  // segment s of sample b in a [capacity, d] matrix that holds real rows only, entry 3 B is the row after the last one.
+  const int32_t* row_start;
+  int capacity;              // rows of the packed matrices (host value, for the tensor maps)
 };
 
 __device__ __forceinline__ void raise_flag(const Geometry& g, unsigned int f) { atomicOr(g.status, f); }
@@ -30,6 +34,17 @@ __device__ __forceinline__ int valid_rows(const Geometry& g, int b, int s) {
   }
   return n;
 }
+
+// First row of segment s of sample b in the activation matrices, and the range of rows that belongs to this problem.
+__device__ __forceinline__ int seg_row0(const Geometry& g, int b, int s) {
+  return (g.row_start != nullptr) ? g.row_start[3 * b + s] : b * g.L + g.seg_off[s];
+}
+__device__ __forceinline__ int rows_begin(const Geometry& g) { return (g.row_start != nullptr) ? g.row_start[0] : 0; }
+__device__ __forceinline__ int rows_end(const Geometry& g) {
+  return (g.row_start != nullptr) ? g.row_start[3 * g.batch] : g.batch * g.L;
+}
+// Rows of the activation matrices as the host knows them (bounds of the tensor maps).
+inline int64_t matrix_rows(const Geometry& g) { return (g.row_start != nullptr) ? (int64_t)g.capacity : (int64_t)g.batch * g.L; }
 
 __device__ __forceinline__ int segment_of(const Geometry& g, int p) {
   return (p >= g.seg_off[2]) ? 2 : (p >= g.seg_off[1]) ? 1 : 0;
@@ -118,5 +133,10 @@ cudaError_t launch_layernorm(const Geometry& g, const float* x, int64_t ldx, con
 // Stack read-out: last real step of each segment of c [B, L, dc] (row stride ldc), concatenated, times w^T + bias.
 cudaError_t launch_stack_head(const Geometry& g, int dtype, const float* c, int64_t ldc, int dc, const void* w,
                               const float* bias, float* out, int n_out, cudaStream_t st);
+
+// packed row layout (rows.cu)
+cudaError_t launch_plan_rows(const Geometry& g, int split_sample, int32_t* row_start, cudaStream_t st);
+cudaError_t launch_move_rows(const Geometry& g, bool pack, const float* src, int64_t src_stride, float* dst, int64_t dst_stride,
+                             int cols, cudaStream_t st);
 
 }  // namespace gsit

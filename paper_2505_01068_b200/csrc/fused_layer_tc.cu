@@ -86,8 +86,8 @@ ln_qkv_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
   uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t bars = base + OFF_BAR;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int rows = g.batch * g.L;
-  const int ntiles = (rows + TM - 1) / TM;
+  const int row_base = rows_begin(g), rows = rows_end(g);  // this problem's rows of the activation matrices
+  const int ntiles = (rows - row_base + TM - 1) / TM;
 
   float* prm = reinterpret_cast<float*>(base_ptr + OFF_P);
   stage_vector(prm, gamma, TD, 1.f, tid, T_THREADS);
@@ -125,8 +125,8 @@ ln_qkv_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
       if (i >= 2) t_mbar_wait(g, bars + B_XFREE + 8 * xb, ((i >> 1) - 1) & 1);  // the row warps hold that tile in registers
       if (t_elect()) {
         t_mbar_expect_tx(bars + B_XFULL + 8 * xb, 2 * XBOX);
-        t_tma_2d(base + OFF_X + xb * 2 * XBOX, &tmX, 0, t * TM, bars + B_XFULL + 8 * xb);
-        t_tma_2d(base + OFF_X + xb * 2 * XBOX + XBOX, &tmX, 32, t * TM, bars + B_XFULL + 8 * xb);
+        t_tma_2d(base + OFF_X + xb * 2 * XBOX, &tmX, 0, row_base + t * TM, bars + B_XFULL + 8 * xb);
+        t_tma_2d(base + OFF_X + xb * 2 * XBOX + XBOX, &tmX, 32, row_base + t * TM, bars + B_XFULL + 8 * xb);
       }
       __syncwarp();
     }
@@ -153,9 +153,9 @@ ln_qkv_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
     const uint32_t tl = tmem + ((uint32_t)((warp & 3) << 5) << 16);
     const uint32_t s_gamma = base + OFF_P, s_beta = s_gamma + TD * 4, s_bias = s_beta + TD * 4;
     int i = 0;
-    bool real = row_real32(g, (int)blockIdx.x * TM + r, rows);
+    bool real = row_real32(g, row_base + (int)blockIdx.x * TM + r, rows);
     for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
-      const int row0 = t * TM, xb = i & 1;
+      const int row0 = row_base + t * TM, xb = i & 1;
       t_mbar_wait(g, bars + B_XFULL + 8 * xb, (i >> 1) & 1);
       float v[TD];
       if (real) {
@@ -171,7 +171,7 @@ ln_qkv_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
       t_fence_async();
       __syncwarp();
       if (lane == 0) t_mbar_arrive(bars + B_HREADY);
-      const bool real_next = row_real32(g, (t + (int)gridDim.x) * TM + r, rows);  // overlaps the MMA
+      const bool real_next = row_real32(g, row_base + (t + (int)gridDim.x) * TM + r, rows);  // overlaps the MMA
 
       t_mbar_wait(g, bars + B_ACCFULL, i & 1);
       t_fence_after();
@@ -252,8 +252,8 @@ proj_mlp_tc_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_const
   uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t bars = base + OFF_BAR;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int rows = g.batch * g.L;
-  const int ntiles = (rows + TM - 1) / TM;
+  const int row_base = rows_begin(g), rows = rows_end(g);  // this problem's rows of the activation matrices
+  const int ntiles = (rows - row_base + TM - 1) / TM;
   const int nh = d_ff / 64;  // k-blocks of hidden units
 
   float* prm = reinterpret_cast<float*>(base_ptr + OFF_P);
@@ -296,7 +296,7 @@ proj_mlp_tc_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_const
     __syncwarp();
     int i = 0;
     for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
-      const int row0 = t * TM;
+      const int row0 = row_base + t * TM;
       const int b = i & 1;
       if (i >= 2) t_mbar_wait(g, bars + B_ATTFREE + 8 * b, ((i >> 1) - 1) & 1);
       if (t_elect()) {
@@ -361,9 +361,9 @@ proj_mlp_tc_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_const
     const uint32_t s_bo = base + OFF_P, s_gamma = s_bo + TD * 4, s_beta = s_gamma + TD * 4, s_b2 = s_beta + TD * 4,
                    s_b1 = s_b2 + TD * 4;
     int i = 0;
-    bool real = row_real32(g, (int)blockIdx.x * TM + r, rows);
+    bool real = row_real32(g, row_base + (int)blockIdx.x * TM + r, rows);
     for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
-      const int row0 = t * TM;
+      const int row0 = row_base + t * TM;
       // ---- y1 = x + att W_o^T + b_o (registers) ----
       t_mbar_wait(g, bars + B_XFULL, i & 1);
       float v[TD];
@@ -397,7 +397,7 @@ proj_mlp_tc_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_const
       t_fence_before();
       __syncwarp();
       if (lane == 0) t_mbar_arrive(bars + B_HREADY);
-      const bool real_next = row_real32(g, (t + (int)gridDim.x) * TM + r, rows);  // overlaps the MMA
+      const bool real_next = row_real32(g, row_base + (t + (int)gridDim.x) * TM + r, rows);  // overlaps the MMA
       // ---- f = relu(h W_1^T + b_1) -> A operand of the second MLP product ----
       t_mbar_wait(g, bars + B_ACCF, i & 1);
       t_fence_after();
@@ -473,7 +473,7 @@ bool fused_layer_tc_supported(const Geometry& g, int d_ff) { return g.d == TD &&
 cudaError_t launch_ln_qkv_tc(const Geometry& g, const float* x, int64_t ldx, const float* gamma, const float* beta, float eps,
                              const __nv_bfloat16* w_qkv, const float* b_qkv, __nv_bfloat16* qkv, cudaStream_t st) {
   if (g.d != TD) return cudaErrorNotSupported;
-  const int64_t rows = (int64_t)g.batch * g.L;
+  const int64_t rows = matrix_rows(g);  // bounds of the tensor maps; the kernel takes its own row range from the geometry
   const int ntiles = (int)((rows + TM - 1) / TM), nsm = t_sm_count();
   if (nsm == 0) return cudaErrorUnknown;
   alignas(64) CUtensorMap tmW, tmX, tmOut;
@@ -495,7 +495,7 @@ cudaError_t launch_proj_mlp_tc(const Geometry& g, const __nv_bfloat16* att, cons
                                const __nv_bfloat16* w_1, const float* b_1, const __nv_bfloat16* w_2, const float* b_2, int d_ff,
                                float* y, int64_t ldy, cudaStream_t st) {
   if (!fused_layer_tc_supported(g, d_ff)) return cudaErrorNotSupported;
-  const int64_t rows = (int64_t)g.batch * g.L;
+  const int64_t rows = matrix_rows(g);  // bounds of the tensor maps; the kernel takes its own row range from the geometry
   const int ntiles = (int)((rows + TM - 1) / TM), nsm = t_sm_count();
   if (nsm == 0) return cudaErrorUnknown;
   alignas(64) CUtensorMap tmAtt, tmX, tmWo, tmW1, tmW2, tmY;

@@ -78,8 +78,8 @@ ln_qkv_tc128_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t bars = base + OFF_BAR;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int rows = g.batch * g.L;
-  const int ntiles = (rows + TM - 1) / TM;
+  const int row_base = rows_begin(g), rows = rows_end(g);  // this problem's rows of the activation matrices
+  const int ntiles = (rows - row_base + TM - 1) / TM;
 
   float* prm = reinterpret_cast<float*>(base_ptr + OFF_P);
   stage_vector(prm, gamma, D2, 1.f, tid, T_THREADS);
@@ -120,7 +120,7 @@ ln_qkv_tc128_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       if (i > 0) t_mbar_wait(g, bars + B_XFREE, (i - 1) & 1);
       if (t_elect()) {
         t_mbar_expect_tx(bars + B_XFULL, 4 * XBOX);
-        for (int j = 0; j < 4; ++j) t_tma_2d(base + OFF_X + j * XBOX, &tmX, 32 * j, t * TM, bars + B_XFULL);
+        for (int j = 0; j < 4; ++j) t_tma_2d(base + OFF_X + j * XBOX, &tmX, 32 * j, row_base + t * TM, bars + B_XFULL);
       }
       __syncwarp();
     }
@@ -153,9 +153,9 @@ ln_qkv_tc128_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     const uint32_t tl = tmem + ((uint32_t)((warp & 3) << 5) << 16);
     const uint32_t s_gamma = base + OFF_P, s_beta = s_gamma + D2 * 4, s_bias = s_beta + D2 * 4;
     int i = 0;
-    bool real = row_real32(g, (int)blockIdx.x * TM + r, rows);
+    bool real = row_real32(g, row_base + (int)blockIdx.x * TM + r, rows);
     for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
-      const int row0 = t * TM;
+      const int row0 = row_base + t * TM;
       t_mbar_wait(g, bars + B_XFULL, i & 1);
       float v[D2];
       if (real) {
@@ -169,7 +169,7 @@ ln_qkv_tc128_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       t_fence_async();
       __syncwarp();
       if (lane == 0) t_mbar_arrive(bars + B_HREADY);
-      const bool real_next = row_real32(g, (t + (int)gridDim.x) * TM + r, rows);  // overlaps the MMA
+      const bool real_next = row_real32(g, row_base + (t + (int)gridDim.x) * TM + r, rows);  // overlaps the MMA
 
       t_mbar_wait(g, bars + B_ACCFULL, i & 1);
       t_fence_after();
@@ -258,8 +258,8 @@ proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_co
   uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t bars = base + OFF_BAR;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int rows = g.batch * g.L;
-  const int ntiles = (rows + TM - 1) / TM;
+  const int row_base = rows_begin(g), rows = rows_end(g);  // this problem's rows of the activation matrices
+  const int ntiles = (rows - row_base + TM - 1) / TM;
   const int nc = d_ff / 64;  // chunks of 64 hidden units
 
   float* prm = reinterpret_cast<float*>(base_ptr + OFF_P);
@@ -306,7 +306,7 @@ proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_co
     __syncwarp();
     int i = 0, n = 0;  // tiles, weight chunks requested so far
     for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
-      const int row0 = t * TM;
+      const int row0 = row_base + t * TM;
       // the attention buffer also holds the LN2 rows of the previous tile until its last first-MLP product is done
       if (i > 0) t_mbar_wait(g, bars + B_ATTFREE, (i - 1) & 1);
       if (t_elect()) {
@@ -396,9 +396,9 @@ proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_co
     const uint32_t s_bo = base + OFF_P, s_gamma = s_bo + D2 * 4, s_beta = s_gamma + D2 * 4, s_b2 = s_beta + D2 * 4,
                    s_b1 = s_b2 + D2 * 4;
     int i = 0, n = 0;
-    bool real = row_real32(g, (int)blockIdx.x * TM + r, rows);
+    bool real = row_real32(g, row_base + (int)blockIdx.x * TM + r, rows);
     for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
-      const int row0 = t * TM;
+      const int row0 = row_base + t * TM;
       // ---- y1 = x + att W_o^T + b_o (registers) ----
       t_mbar_wait(g, bars + B_XFULL, i & 1);
       float v[D2];
@@ -432,7 +432,7 @@ proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_co
       t_fence_before();
       __syncwarp();
       if (lane == 0) t_mbar_arrive(bars + B_HREADY);
-      const bool real_next = row_real32(g, (t + (int)gridDim.x) * TM + r, rows);
+      const bool real_next = row_real32(g, row_base + (t + (int)gridDim.x) * TM + r, rows);
       // ---- hidden chunks: f = relu(h W_1c^T + b_1c) -> A operand of the second product ----
 #pragma unroll 1
       for (int c = 0; c < nc; ++c, ++n) {
@@ -499,7 +499,7 @@ bool fused_layer_tc128_supported(const Geometry& g, int d_ff) { return g.d == D2
 cudaError_t launch_ln_qkv_tc128(const Geometry& g, const float* x, int64_t ldx, const float* gamma, const float* beta, float eps,
                                 const __nv_bfloat16* w_qkv, const float* b_qkv, __nv_bfloat16* qkv, cudaStream_t st) {
   if (g.d != D2) return cudaErrorNotSupported;
-  const int64_t rows = (int64_t)g.batch * g.L;
+  const int64_t rows = matrix_rows(g);  // bounds of the tensor maps; the kernel takes its own row range from the geometry
   const int ntiles = (int)((rows + TM - 1) / TM), nsm = t_sm_count();
   if (nsm == 0) return cudaErrorUnknown;
   alignas(64) CUtensorMap tmW, tmX, tmOut;
@@ -521,7 +521,7 @@ cudaError_t launch_proj_mlp_tc128(const Geometry& g, const __nv_bfloat16* att, c
                                   const __nv_bfloat16* w_1, const float* b_1, const __nv_bfloat16* w_2, const float* b_2, int d_ff,
                                   float* y, int64_t ldy, cudaStream_t st) {
   if (!fused_layer_tc128_supported(g, d_ff)) return cudaErrorNotSupported;
-  const int64_t rows = (int64_t)g.batch * g.L;
+  const int64_t rows = matrix_rows(g);  // bounds of the tensor maps; the kernel takes its own row range from the geometry
   const int ntiles = (int)((rows + TM - 1) / TM), nsm = t_sm_count();
   if (nsm == 0) return cudaErrorUnknown;
   alignas(64) CUtensorMap tmAtt, tmX, tmWo, tmW1, tmW2;

@@ -98,6 +98,7 @@ __device__ __forceinline__ void stage_vector(float* dst, const float* src, int n
 // Row validity with 32-bit arithmetic (the library limits B * L to 2^29).
 __device__ __forceinline__ bool row_real32(const Geometry& g, int row, int rows) {
   if (row >= rows) return false;
+  if (g.row_start != nullptr) return true;  // packed layout: every row below the end is taken as real
   const int b = row / g.L, p = row - b * g.L;
   const int sgm = segment_of(g, p);
   return (p - g.seg_off[sgm]) < valid_rows(g, b, sgm);

@@ -71,6 +71,13 @@ gsit_status make_geometry(const gsit_shape* s, Geometry* g) {
   g->allowed = bits;
   g->valid_len = s->valid_len;
   g->status = nullptr;
+  g->row_start = s->row_start;
+  g->capacity = 0;
+  if (s->row_start != nullptr) {  // packed row layout
+    if (s->valid_len == nullptr || s->packed_capacity < 1) return GSIT_ERR_INVALID_ARG;
+    if ((int64_t)s->packed_capacity > 0x7fffffffLL / 4) return GSIT_ERR_UNSUPPORTED;
+    g->capacity = s->packed_capacity;
+  }
   if (s->dtype == GSIT_BF16) {
     if (g->d % 16 != 0) return GSIT_ERR_UNSUPPORTED;
     if (g->hd != 8 && g->hd != 16 && g->hd != 32 && g->hd != 64) return GSIT_ERR_UNSUPPORTED;
@@ -94,7 +101,8 @@ struct LayerScratch {
   size_t h, qkv, att, y1, f, total;
 };
 LayerScratch layer_scratch(const Geometry& g, int dtype, int d_ff) {
-  const size_t rows = (size_t)g.batch * g.L, es = (dtype == GSIT_BF16) ? 2 : 4;
+  // packed layout: every call addresses the packed matrices by absolute row, whatever part of the batch it covers
+  const size_t rows = (size_t)matrix_rows(g), es = (dtype == GSIT_BF16) ? 2 : 4;
   LayerScratch s;
   size_t off = 0;
   s.h = off;   off += align_up(rows * g.d * es, 256);       // LN1(x), later LN2(y1)
@@ -170,6 +178,7 @@ gsit_status gsit_im_qkv_proj(const gsit_shape* shape, const void* x, int64_t x_r
   Geometry g;
   gsit_status st = make_geometry(shape, &g);
   if (st != GSIT_OK) return st;
+  if (g.row_start != nullptr) return GSIT_ERR_UNSUPPORTED;  // the packed layout reaches this projection through the layer call
   if (!x || !w_qkv || !qkv || x_row_stride < g.d) return GSIT_ERR_INVALID_ARG;
   if (!aligned16(x) || !aligned16(w_qkv) || !aligned16(qkv)) return GSIT_ERR_INVALID_ARG;
   if (shape->dtype == GSIT_BF16 && x_row_stride % 8 != 0) return GSIT_ERR_INVALID_ARG;
@@ -192,6 +201,7 @@ gsit_status gsit_im_attention_fwd(const gsit_shape* shape, const void* q, const 
   if (!q || !k || !v || !out || row_stride < g.d) return GSIT_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return GSIT_ERR_INVALID_ARG;
   if (shape->dtype == GSIT_BF16 && row_stride % 8 != 0) return GSIT_ERR_INVALID_ARG;
+  if (g.row_start != nullptr && (shape->dtype != GSIT_BF16 || g.hd > 32)) return GSIT_ERR_UNSUPPORTED;
   if (from_cuda(status_ptr(&g.status)) != GSIT_OK) return GSIT_ERR_CUDA;
   return run_attention(g, shape->dtype, q, k, v, row_stride, out, lse, pick_scale(shape, g),
                        static_cast<cudaStream_t>(stream));
@@ -223,12 +233,15 @@ gsit_status gsit_im_layer_fwd(const gsit_shape* shape, const gsit_layer_weights*
   const int bf = (dtype == GSIT_BF16);
   const int es = bf ? 2 : 4;
   const int M = g.batch * g.L, d = g.d;
+  if (g.row_start != nullptr &&
+      !(bf && g.hd <= 32 && (fused_layer_tc_supported(g, w->d_ff) || fused_layer_tc128_supported(g, w->d_ff))))
+    return GSIT_ERR_UNSUPPORTED;  // the packed layout is implemented by the tcgen05 fused halves and the mma.sync attention
 
-  if (bf && fused_layer_supported(g, w->d_ff) && g_attn_variant != 8) {
+  if (bf && fused_layer_supported(g, w->d_ff) && (g_attn_variant != 8 || g.row_start != nullptr)) {
     // three launches: LN1 + shared projection, IM attention, out-projection + residual + LN2 + MLP + residual
     // d_model 64 and 128 run both halves on tcgen05 (tuning knob 9 keeps the mma.sync kernels)
-    const bool tc = fused_layer_tc_supported(g, w->d_ff) && g_attn_variant != 9;
-    const bool tc128 = fused_layer_tc128_supported(g, w->d_ff) && g_attn_variant != 9;
+    const bool tc = fused_layer_tc_supported(g, w->d_ff) && (g_attn_variant != 9 || g.row_start != nullptr);
+    const bool tc128 = fused_layer_tc128_supported(g, w->d_ff) && (g_attn_variant != 9 || g.row_start != nullptr);
     {
       TraceScope t(GSIT_KERNEL_LINEAR, cs);
       st = from_cuda(tc ? launch_ln_qkv_tc(g, x, x_row_stride, w->ln1_gamma, w->ln1_beta, eps,
@@ -291,11 +304,49 @@ gsit_status gsit_im_layer_fwd(const gsit_shape* shape, const gsit_layer_weights*
   return run_linear(g, dtype, a, cs);
 }
 
+gsit_status gsit_plan_rows(const gsit_shape* shape, int32_t split_sample, int32_t* row_start, gsit_stream stream) {
+  if (shape == nullptr || row_start == nullptr || shape->valid_len == nullptr) return GSIT_ERR_INVALID_ARG;
+  gsit_shape sh = *shape;  // only batch, seg_len and valid_len matter here: make the rest valid
+  sh.d_model = 16; sh.heads = 1; sh.phase = GSIT_PHASE_INTRA; sh.dtype = GSIT_F32; sh.row_start = nullptr; sh.packed_capacity = 0;
+  Geometry g;
+  gsit_status st = make_geometry(&sh, &g);
+  if (st != GSIT_OK) return st;
+  if (split_sample < 0) return GSIT_ERR_INVALID_ARG;
+  if (from_cuda(status_ptr(&g.status)) != GSIT_OK) return GSIT_ERR_CUDA;
+  return from_cuda(launch_plan_rows(g, split_sample, row_start, static_cast<cudaStream_t>(stream)));
+}
+
+static gsit_status move_rows(const gsit_shape* shape, bool pack, const float* src, int64_t src_stride, float* dst,
+                             int64_t dst_stride, int32_t cols, gsit_stream stream) {
+  if (shape == nullptr || shape->row_start == nullptr || !src || !dst) return GSIT_ERR_INVALID_ARG;
+  if (cols < 4 || cols % 4 != 0 || src_stride < cols || dst_stride < cols || src_stride % 4 != 0 || dst_stride % 4 != 0)
+    return GSIT_ERR_INVALID_ARG;
+  if (!aligned16(src) || !aligned16(dst)) return GSIT_ERR_INVALID_ARG;
+  gsit_shape sh = *shape;
+  sh.d_model = 16; sh.heads = 1; sh.phase = GSIT_PHASE_INTRA; sh.dtype = GSIT_F32;
+  Geometry g;
+  gsit_status st = make_geometry(&sh, &g);
+  if (st != GSIT_OK) return st;
+  if (from_cuda(status_ptr(&g.status)) != GSIT_OK) return GSIT_ERR_CUDA;
+  return from_cuda(launch_move_rows(g, pack, src, src_stride, dst, dst_stride, cols, static_cast<cudaStream_t>(stream)));
+}
+
+gsit_status gsit_pack_rows(const gsit_shape* shape, const float* x, int64_t x_row_stride, float* x_packed,
+                           int64_t packed_row_stride, int32_t cols, gsit_stream stream) {
+  return move_rows(shape, true, x, x_row_stride, x_packed, packed_row_stride, cols, stream);
+}
+
+gsit_status gsit_unpack_rows(const gsit_shape* shape, const float* y_packed, int64_t packed_row_stride, float* y,
+                             int64_t y_row_stride, int32_t cols, gsit_stream stream) {
+  return move_rows(shape, false, y_packed, packed_row_stride, y, y_row_stride, cols, stream);
+}
+
 gsit_status gsit_stack_head_fwd(const gsit_shape* shape, const float* c, int64_t c_row_stride, int32_t d_c, const void* w_f,
                                 const float* b_f, float* out, int32_t out_features, gsit_stream stream) {
   if (shape == nullptr || !c || !w_f || !out || d_c < 1 || out_features < 1 || c_row_stride < d_c) return GSIT_ERR_INVALID_ARG;
   gsit_shape sh = *shape;  // only batch, seg_len, valid_len and dtype matter here: make the rest valid
   sh.d_model = 16; sh.heads = 1; sh.phase = GSIT_PHASE_INTRA;
+  sh.row_start = nullptr; sh.packed_capacity = 0;  // c is in the padded layout
   Geometry g;
   gsit_status st = make_geometry(&sh, &g);
   if (st != GSIT_OK) return st;

@@ -1,0 +1,90 @@
+// Packed row layout: the plan (where each segment of each sample starts among the real rows), and the copies between
+// the padded [B, L, cols] layout and the packed [rows, cols] one.  Section "Inner Decomposition for Efficiency" drops
+// padded positions from the computation; packed, they are not stored either, so the row-wise parts of the layer
+// (LayerNorm, projections, MLP) do no work for them at all.
+#include "common.cuh"
+
+namespace gsit {
+namespace {
+
+// One CTA; thread i owns the pairs (b, s) = i, i + 1024, ...; an exclusive scan in (b, s) order.
+__global__ void __launch_bounds__(1024) plan_rows_kernel(const Geometry g, const int split_sample, int32_t* __restrict__ row_start) {
+  __shared__ int part[1024];
+  __shared__ int split_sum;
+  const int n = 3 * g.batch, tid = threadIdx.x;
+  const int per = (n + 1023) / 1024;                 // consecutive entries per thread
+  const int lo = min(n, tid * per), hi = min(n, lo + per);
+  int sum = 0;
+  for (int e = lo; e < hi; ++e) sum += valid_rows(g, e / 3, e % 3);
+  part[tid] = sum;
+  __syncthreads();
+  for (int off = 1; off < 1024; off <<= 1) {         // inclusive scan of the per-thread sums
+    const int v = (tid >= off) ? part[tid - off] : 0;
+    __syncthreads();
+    part[tid] += v;
+    __syncthreads();
+  }
+  int run = part[tid] - sum;                          // exclusive prefix of this thread's first entry
+  // rows before the split sample, to find the padding that aligns it
+  if (tid == 0) split_sum = -1;
+  __syncthreads();
+  const int split_e = 3 * split_sample;
+  {
+    int r2 = run;
+    for (int e = lo; e < hi; ++e) {
+      if (e == split_e) split_sum = r2;
+      r2 += valid_rows(g, e / 3, e % 3);
+    }
+  }
+  __syncthreads();
+  const int pad = (split_sample > 0 && split_sample < g.batch && split_sum >= 0) ? ((split_sum + 127) / 128 * 128 - split_sum) : 0;
+  for (int e = lo; e < hi; ++e) {
+    row_start[e] = run + ((pad > 0 && e >= split_e) ? pad : 0);
+    run += valid_rows(g, e / 3, e % 3);
+  }
+  if (tid == 1023) row_start[n] = part[1023] + pad;
+}
+
+// One warp per (sample, position); lanes stride over 16-byte chunks of the row.
+template <bool PACK>
+__global__ void __launch_bounds__(256) move_rows_kernel(const Geometry g, const float* __restrict__ src, const int64_t src_stride,
+                                                        float* __restrict__ dst, const int64_t dst_stride, const int cols) {
+  const int64_t w = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (w >= (int64_t)g.batch * g.L) return;
+  const int b = (int)(w / g.L), p = (int)(w - (int64_t)b * g.L), lane = threadIdx.x & 31;
+  const int s = segment_of(g, p), i = p - g.seg_off[s];
+  const bool real = i < valid_rows(g, b, s);
+  const int64_t packed = real ? (int64_t)g.row_start[3 * b + s] + i : 0;
+  if (PACK) {
+    if (!real) return;
+    const float4* a = reinterpret_cast<const float4*>(src + w * src_stride);
+    float4* o = reinterpret_cast<float4*>(dst + packed * dst_stride);
+    for (int c = lane; c < cols / 4; c += 32) o[c] = a[c];
+  } else {
+    float4* o = reinterpret_cast<float4*>(dst + w * dst_stride);
+    if (real) {
+      const float4* a = reinterpret_cast<const float4*>(src + packed * src_stride);
+      for (int c = lane; c < cols / 4; c += 32) o[c] = a[c];
+    } else {
+      for (int c = lane; c < cols / 4; c += 32) o[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_plan_rows(const Geometry& g, int split_sample, int32_t* row_start, cudaStream_t st) {
+  plan_rows_kernel<<<1, 1024, 0, st>>>(g, split_sample, row_start);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_move_rows(const Geometry& g, bool pack, const float* src, int64_t src_stride, float* dst, int64_t dst_stride,
+                             int cols, cudaStream_t st) {
+  const int64_t warps = (int64_t)g.batch * g.L;
+  const unsigned blocks = (unsigned)((warps + 7) / 8);
+  if (pack) move_rows_kernel<true><<<blocks, 256, 0, st>>>(g, src, src_stride, dst, dst_stride, cols);
+  else move_rows_kernel<false><<<blocks, 256, 0, st>>>(g, src, src_stride, dst, dst_stride, cols);
+  return cudaGetLastError();
+}
+
+}  // namespace gsit

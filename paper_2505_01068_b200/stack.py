@@ -16,7 +16,8 @@ from . import binding as B
 
 class GsitStack:
     def __init__(self, fwd_layers, bwd_layers, intra_layers, seg_len, heads, intra_heads, ln_eps=1e-5, head=None,
-                 concurrent_rings=True, batch_chunks=1, intra_halves=True):
+                 concurrent_rings=True, batch_chunks=1, intra_halves=True,
+                 packed=True):
         """head: optional (w_f, b_f) of the read-out X_m = f(|| Split(.)[-1]); see read_out().
         concurrent_rings: issue independent work on several streams (False: every launch on the caller's stream, whole
         batch per launch).  batch_chunks: with concurrent issue, the batch is cut into this many groups of samples, each
@@ -24,11 +25,17 @@ class GsitStack:
         one chunk is fastest: the persistent fused kernels pay their per-CTA set-up once per launch.)
         intra_halves: with concurrent issue, the intra encoder runs on the two halves of the batch on the two streams, so
         that the attention of one half overlaps the fused layer halves of the other (0.934 -> 0.914 ms at that shape;
-        three or four parts are slower again)."""
+        three or four parts are slower again).
+        packed: when valid lengths are given (and the layers are bf16 at widths the tcgen05 fused kernels cover), the
+        stack works on the packed row layout: the real rows are gathered once, every layer runs on them only, and the
+        result is scattered back with +0 in the padded positions.  The row-wise parts of the layers then do no work
+        for padding (24 % of the rows at the benchmark's lengths).  The plan of where each segment starts is made on the
+        device, so a captured forward stays valid when the lengths change."""
         self.head = head
         self.concurrent_rings = concurrent_rings
         self.batch_chunks = max(1, int(batch_chunks))
         self.intra_halves = bool(intra_halves)
+        self.packed = bool(packed)
         self.fwd, self.bwd, self.intra = list(fwd_layers), list(bwd_layers), list(intra_layers)
         self.seg_len, self.heads, self.intra_heads, self.ln_eps = tuple(seg_len), heads, intra_heads, ln_eps
         self._bufs = None
@@ -85,8 +92,107 @@ class GsitStack:
             cur = dst
         return len(self.intra) % 2  # 1: the result is in c1, 0: in c0
 
+    def _packed_buffers(self, x, valid_len):
+        Bn, L, d = x.shape
+        key = ("packed", Bn, L, d, x.device)
+        if self._bufs is None:
+            self._bufs = {}
+        if key not in self._bufs:
+            cap = Bn * L + 128  # always enough: the real rows plus the alignment of the second half's first row
+            code = B._dtype_code(self.fwd[0]["w_qkv"].dtype)
+            plan = torch.zeros(3 * Bn + 1, dtype=torch.int32, device=x.device)
+            sh1 = B.make_shape(Bn, self.seg_len, d, self.heads, valid_len, code, B.PHASE_INTER_FWD, row_start=plan, capacity=cap)
+            need = B.workspace_bytes(sh1, B.CALL_LAYER, self.fwd[0]["w_1"].shape[0])
+            if self.intra:
+                sh2 = B.make_shape(Bn, self.seg_len, 2 * d, self.intra_heads, valid_len, code, B.PHASE_INTRA, row_start=plan,
+                                   capacity=cap)
+                need = max(need, B.workspace_bytes(sh2, B.CALL_LAYER, self.intra[0]["w_1"].shape[0]))
+            f32 = dict(dtype=torch.float32, device=x.device)
+            self._bufs[key] = (cap, plan, [torch.empty(need, dtype=torch.uint8, device=x.device) for _ in range(2)],
+                               [torch.zeros((cap, d), **f32) for _ in range(5)],
+                               torch.zeros((cap, 2 * d), **f32), torch.zeros((cap, 2 * d), **f32),
+                               torch.empty((Bn, L, 2 * d), **f32))
+        return self._bufs[key]
+
+    def _forward_packed(self, x, valid_len):
+        cap, plan, ws, t, c0, c1, y = self._packed_buffers(x, valid_len)
+        Bn, L, d = x.shape
+        conc = self.concurrent_rings and self.fwd and self.bwd
+        halves = conc and self.intra_halves and self.intra and Bn >= 2
+        mid = Bn // 2
+        B.plan_rows(valid_len, self.seg_len, mid if halves else 0, out=plan)
+        xp = B.pack_rows(x, t[4], self.seg_len, valid_len, plan)
+
+        def ring(layers, phase, half, w_s, ping):
+            cur = xp
+            for i, w in enumerate(layers):
+                dst = c0[:, half * d:(half + 1) * d] if i == len(layers) - 1 else ping[i % 2]
+                B.im_layer_fwd(cur, w, self.seg_len, self.heads, valid_len, phase, ln_eps=self.ln_eps, out=dst, workspace=w_s,
+                               row_start=plan)
+                cur = dst
+
+        def intra(lo, hi, w_s):  # samples lo .. hi - 1: their rows of the packed matrices are addressed through the plan
+            cur, ping = c0, [c1, c0]
+            for i, w in enumerate(self.intra):
+                dst = ping[i % 2]
+                B.im_layer_fwd(cur, w, self.seg_len, self.intra_heads, valid_len[lo:hi], B.PHASE_INTRA, ln_eps=self.ln_eps,
+                               out=dst, workspace=w_s, row_start=plan[3 * lo:])
+                cur = dst
+            return cur
+
+        if not conc:
+            ring(self.fwd, B.PHASE_INTER_FWD, 0, ws[0], t[0:2])
+            ring(self.bwd, B.PHASE_INTER_BWD, 1, ws[0], t[0:2])
+            res = intra(0, Bn, ws[0]) if self.intra else c0
+        else:
+            if self._lanes is None:
+                dev = x.device
+                self._lanes = ([torch.cuda.Stream(device=dev) for _ in range(2)], torch.cuda.Event(),
+                               [torch.cuda.Event() for _ in range(2)])
+                self._ring_done = [torch.cuda.Event()]
+            streams, fork, done = self._lanes
+            s_f, s_b = streams[0], streams[1]
+            main = torch.cuda.current_stream(x.device)
+            fork.record(main)
+            s_f.wait_event(fork)
+            s_b.wait_event(fork)
+            with torch.cuda.stream(s_b):
+                ring(self.bwd, B.PHASE_INTER_BWD, 1, ws[1], t[2:4])
+                done[1].record(s_b)
+            with torch.cuda.stream(s_f):
+                ring(self.fwd, B.PHASE_INTER_FWD, 0, ws[0], t[0:2])
+                res = c0
+                if halves:
+                    ring_f = self._ring_done[0]
+                    ring_f.record(s_f)
+                    s_f.wait_event(done[1])
+                    res = intra(0, mid, ws[0])
+                    with torch.cuda.stream(s_b):
+                        s_b.wait_event(ring_f)
+                        intra(mid, Bn, ws[1])
+                        done[1].record(s_b)
+                    s_f.wait_event(done[1])
+                else:
+                    s_f.wait_event(done[1])
+                    if self.intra:
+                        res = intra(0, Bn, ws[0])
+                done[0].record(s_f)
+            main.wait_event(done[0])
+            for st in streams:
+                x.record_stream(st)
+                valid_len.record_stream(st)
+        B.unpack_rows(res, y, self.seg_len, valid_len, plan)
+        return y
+
     def forward(self, x, valid_len=None):
         """x float32 [B, L, d] -> float32 [B, L, 2d].  The result lives in a buffer owned by this object."""
+        if self.packed and valid_len is not None and self.batch_chunks == 1:
+            try:
+                return self._forward_packed(x, valid_len)
+            except B.GsitError as e:
+                if e.code != 2:  # anything but "this shape is not covered": a real error
+                    raise
+                self.packed = False
         chunks, ws, t, c0, c1 = self._buffers(x, valid_len)
         if len(chunks) == 1 and not (self.concurrent_rings and self.fwd and self.bwd):
             self._ring(x, self.fwd, B.PHASE_INTER_FWD, 0, c0, ws[0][0], t[0:2], valid_len)

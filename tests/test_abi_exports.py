@@ -29,7 +29,8 @@ def test_status_strings_and_shape_struct_layout():
 
     assert g.version() >= 100
     assert g.status_string(0) == "ok" and "workspace" in g.status_string(3)
-    assert ctypes.sizeof(g.binding.Shape) == 48 and g.binding.Shape.valid_len.offset == 24
+    assert ctypes.sizeof(g.binding.Shape) == 64 and g.binding.Shape.valid_len.offset == 24
+    assert g.binding.Shape.row_start.offset == 48 and g.binding.Shape.packed_capacity.offset == 56
     assert ctypes.sizeof(g.binding.LayerWeights) == 12 * 8 + 8
 
 

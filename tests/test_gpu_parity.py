@@ -308,3 +308,92 @@ def test_host_pipeline_delivers_every_step(g):
     err = np.abs(y_host[0].numpy().astype(np.float64) - ref)
     assert err.max() <= 10 * 2e-2 and err.mean() <= 10 * 2e-3, (err.max(), err.mean())
     assert g.last_device_status() == (0, 0)
+
+
+def _real_mask(seg_len, valid, B):
+    L = sum(seg_len)
+    off = np.cumsum([0] + list(seg_len))
+    real = np.zeros((B, L), dtype=bool)
+    for b in range(B):
+        for s in range(3):
+            real[b, off[s]:off[s] + valid[b, s]] = True
+    return real
+
+
+def test_packed_rows_plan_pack_unpack(g):
+    """Packed row layout: the device-made plan is the running sum of the valid lengths (with the requested sample
+    starting on a multiple of 128 rows), packing gathers exactly the real rows, unpacking restores them and writes +0
+    in the padded positions."""
+    seg = (50, 300, 270)
+    valid = np.array([[50, 300, 270], [25, 0, 200], [0, 0, 0], [1, 151, 7], [50, 299, 1]], dtype=np.int32)
+    B, L, cols = valid.shape[0], sum(seg), 64
+    vl = torch.from_numpy(valid).cuda()
+    rng = np.random.default_rng(3)
+    x = rng.standard_normal((B, L, cols), dtype=np.float32)
+    real = _real_mask(seg, valid, B)
+    for split in (0, 2, 4):
+        plan = g.plan_rows(vl, seg, split).cpu().numpy()
+        run, want = 0, []
+        for b in range(B):
+            if split and b == split:
+                run = (run + 127) // 128 * 128
+            for s in range(3):
+                want.append(run)
+                run += int(valid[b, s])
+        want.append(run)
+        assert np.array_equal(plan, np.array(want, dtype=np.int32)), split
+        plan_d = torch.from_numpy(plan).cuda()
+        xp = torch.full((B * L + 128, cols), float("nan"), device="cuda")
+        g.pack_rows(to_dev(x), xp, seg, vl, plan_d)
+        xp_h = xp.cpu().numpy()
+        for b in range(B):
+            off = 0
+            for s in range(3):
+                n = valid[b, s]
+                assert np.array_equal(xp_h[plan[3 * b + s]:plan[3 * b + s] + n], x[b, off:off + n])
+                off += seg[s]
+        back = torch.full((B, L, cols), 7.0, device="cuda")
+        g.unpack_rows(xp, back, seg, vl, plan_d)
+        bk = back.cpu().numpy()
+        assert np.array_equal(bk[real], x[real]) and np.all(bk[~real] == 0.0) and not np.signbit(bk[~real]).any()
+    assert g.last_device_status() == (0, 0)
+
+
+def test_packed_layout_gives_the_same_bits_as_the_padded_one(g):
+    """Layers and the whole stack on the packed rows against the same calls on the padded layout: samples and rows are
+    independent and the arithmetic per row is the same, so the results are equal bit for bit (and the padded layout is
+    held to the oracle above)."""
+    inp = wk.make_inputs(4, batch=5)
+    wl = inp["workload"]
+    n_f, n_b, n_i, ih = wl.stack
+    valid = inp["valid_len"].copy()
+    valid[1] = [0, valid[1, 1], 0]          # a sample with two empty modalities
+    valid[3] = [0, 0, 0]                     # and an empty sample
+    vl = torch.from_numpy(valid).cuda()
+    B, L, d = inp["x"].shape
+    cap = B * L + 128
+    x = to_dev(wk.fill_padding(inp["x"], wl.seg_len, valid, np.nan))
+    plan = g.plan_rows(vl, wl.seg_len)
+    for w, heads, ph, width in ((inp["fwd_layers"][0], wl.heads, g.PHASE_INTER_FWD, d), (inp["bwd_layers"][1], wl.heads, g.PHASE_INTER_BWD, d),
+                                (inp["intra_layers"][0], ih, g.PHASE_INTRA, 2 * d)):
+        xin = x if width == d else torch.cat([x, x.flip(2)], dim=2).contiguous()
+        wd = weights_to_dev(w, "bf16")
+        want = g.im_layer_fwd(xin, wd, wl.seg_len, heads, vl, ph)
+        xp = torch.zeros((cap, width), device="cuda")
+        g.pack_rows(xin, xp, wl.seg_len, vl, plan)
+        yp = torch.full((cap, width), float("nan"), device="cuda")
+        g.im_layer_fwd(xp, wd, wl.seg_len, heads, vl, ph, out=yp, row_start=plan)
+        got = torch.full_like(want, 3.0)
+        g.unpack_rows(yp, got, wl.seg_len, vl, plan)
+        torch.cuda.synchronize()
+        assert torch.equal(got, want), (ph, width)
+    mk = lambda **kw: g.GsitStack([weights_to_dev(w, "bf16") for w in inp["fwd_layers"]],
+                                  [weights_to_dev(w, "bf16") for w in inp["bwd_layers"]],
+                                  [weights_to_dev(w, "bf16") for w in inp["intra_layers"]], wl.seg_len, wl.heads, ih, **kw)
+    a = mk(packed=False).forward(x, vl).clone()
+    for kw in (dict(), dict(intra_halves=False), dict(concurrent_rings=False)):
+        st = mk(**kw)
+        b = st.forward(x, vl).clone()
+        torch.cuda.synchronize()
+        assert st.packed and torch.equal(a, b), kw
+    assert g.last_device_status() == (0, 0)
