@@ -311,6 +311,30 @@ def run_gpu(args):
                            "t_hbm_us": t_hbm * 1e6, "t_exp_us": t_exp * 1e6, "d_model": d, "heads": heads,
                            "buffer_sets": nsets, "in_step_us": (cross_s if name == "cross" else intra_s) * 1e6}
 
+    # ---- the same stack at the paper's length statistics (second workload family: about a quarter of the positions
+    # are real), packed row layout against the padded one: context, not part of `value` ----
+    stats_lengths = {}
+    if not args.no_scaled:
+        v6 = wk.draw_valid_len(np.random.default_rng(wk.WORKLOADS[6].seed), wk.WORKLOADS[6], B)
+        vl6 = torch.from_numpy(v6).cuda()
+        for name, packed in (("padded_layout", False), ("packed_layout", True)):
+            st6 = g.GsitStack(stack.fwd, stack.bwd, stack.intra, wl.seg_len, wl.heads, ih, packed=packed)
+            st6.forward(xbufs[0], vl6)
+            torch.cuda.synchronize()
+            gs6 = []
+            for i in range(nbuf):
+                gr = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(gr):
+                    st6.forward(xbufs[i], vl6)
+                gs6.append(gr)
+            _time_graph_replays(torch, gs6, nbuf, dist, 1)
+            ms6 = _time_graph_replays(torch, gs6, 50, dist, 1) / 50
+            stats_lengths[name] = {"ms_per_step": ms6, "tokens_per_s": float(v6.sum()) / (ms6 * 1e-3)}
+            del gs6, st6
+        stats_lengths["valid_tokens_per_step"] = int(v6.sum())
+        stats_lengths["real_fraction"] = float(v6.sum()) / (B * wl.L)
+        torch.cuda.empty_cache()
+
     # ---- the scaled shape (head_dim 64, tcgen05 kernel), attention alone: context for the tensor-bound case ----
     scaled = {}
     if not args.no_scaled:
@@ -389,6 +413,7 @@ def run_gpu(args):
                          "sample": f"{sub} of {B} samples, one step (valid tokens {ref_tokens}) in {cpu_s:.2f} s"},
         "attention": attention,
         "scaled_attention_hd64": scaled,
+        "length_statistics_workload": stats_lengths,
         "step_kernel_ms": {"attention": float(att.sum()) / trace_steps, "linear": lin_ms / trace_steps,
                            "layernorm": ln_ms / trace_steps, "launches": {"attention": per_step, "linear": lin_n // trace_steps,
                                                                           "layernorm": ln_n // trace_steps}},
