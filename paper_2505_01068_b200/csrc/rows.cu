@@ -45,29 +45,26 @@ __global__ void __launch_bounds__(1024) plan_rows_kernel(const Geometry g, const
   if (tid == 1023) row_start[n] = part[1023] + pad;
 }
 
-// One warp per (sample, position); lanes stride over 16-byte chunks of the row.
+// One thread per 16-byte chunk of a padded-layout row: a warp covers whole rows (or several short ones), so both sides of
+// the copy are coalesced.  All index arithmetic is 32-bit (the library limits B * L to 2^29 rows).
 template <bool PACK>
 __global__ void __launch_bounds__(256) move_rows_kernel(const Geometry g, const float* __restrict__ src, const int64_t src_stride,
-                                                        float* __restrict__ dst, const int64_t dst_stride, const int cols) {
-  const int64_t w = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
-  if (w >= (int64_t)g.batch * g.L) return;
-  const int b = (int)(w / g.L), p = (int)(w - (int64_t)b * g.L), lane = threadIdx.x & 31;
+                                                        float* __restrict__ dst, const int64_t dst_stride, const int cpr /* chunks per row */,
+                                                        const unsigned total /* chunks in all */) {
+  const unsigned idx = blockIdx.x * 256u + threadIdx.x;
+  if (idx >= total) return;
+  const unsigned w = idx / (unsigned)cpr, c = idx - w * (unsigned)cpr;  // padded-layout row, chunk in the row
+  const int b = (int)(w / (unsigned)g.L), p = (int)(w - (unsigned)b * (unsigned)g.L);
   const int s = segment_of(g, p), i = p - g.seg_off[s];
   const bool real = i < valid_rows(g, b, s);
-  const int64_t packed = real ? (int64_t)g.row_start[3 * b + s] + i : 0;
   if (PACK) {
     if (!real) return;
-    const float4* a = reinterpret_cast<const float4*>(src + w * src_stride);
-    float4* o = reinterpret_cast<float4*>(dst + packed * dst_stride);
-    for (int c = lane; c < cols / 4; c += 32) o[c] = a[c];
+    const int64_t packed = (int64_t)g.row_start[3 * b + s] + i;
+    reinterpret_cast<float4*>(dst + packed * dst_stride)[c] = reinterpret_cast<const float4*>(src + (int64_t)w * src_stride)[c];
   } else {
-    float4* o = reinterpret_cast<float4*>(dst + w * dst_stride);
-    if (real) {
-      const float4* a = reinterpret_cast<const float4*>(src + packed * src_stride);
-      for (int c = lane; c < cols / 4; c += 32) o[c] = a[c];
-    } else {
-      for (int c = lane; c < cols / 4; c += 32) o[c] = make_float4(0.f, 0.f, 0.f, 0.f);
-    }
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (real) v = reinterpret_cast<const float4*>(src + ((int64_t)g.row_start[3 * b + s] + i) * src_stride)[c];
+    reinterpret_cast<float4*>(dst + (int64_t)w * dst_stride)[c] = v;
   }
 }
 
@@ -80,10 +77,12 @@ cudaError_t launch_plan_rows(const Geometry& g, int split_sample, int32_t* row_s
 
 cudaError_t launch_move_rows(const Geometry& g, bool pack, const float* src, int64_t src_stride, float* dst, int64_t dst_stride,
                              int cols, cudaStream_t st) {
-  const int64_t warps = (int64_t)g.batch * g.L;
-  const unsigned blocks = (unsigned)((warps + 7) / 8);
-  if (pack) move_rows_kernel<true><<<blocks, 256, 0, st>>>(g, src, src_stride, dst, dst_stride, cols);
-  else move_rows_kernel<false><<<blocks, 256, 0, st>>>(g, src, src_stride, dst, dst_stride, cols);
+  const int cpr = cols / 4;
+  const int64_t total = (int64_t)g.batch * g.L * cpr;
+  if (total > 0xffffffffLL) return cudaErrorNotSupported;
+  const unsigned blocks = (unsigned)((total + 255) / 256);
+  if (pack) move_rows_kernel<true><<<blocks, 256, 0, st>>>(g, src, src_stride, dst, dst_stride, cpr, (unsigned)total);
+  else move_rows_kernel<false><<<blocks, 256, 0, st>>>(g, src, src_stride, dst, dst_stride, cpr, (unsigned)total);
   return cudaGetLastError();
 }
 
