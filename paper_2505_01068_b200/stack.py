@@ -114,8 +114,10 @@ class GsitStack:
                                torch.empty((Bn, L, 2 * d), **f32))
         return self._bufs[key]
 
-    def _forward_packed(self, x, valid_len):
+    def _forward_packed(self, x, valid_len, out=None):
         cap, plan, ws, t, c0, c1, y = self._packed_buffers(x, valid_len)
+        if out is not None:
+            y = out
         Bn, L, d = x.shape
         conc = self.concurrent_rings and self.fwd and self.bwd
         halves = conc and self.intra_halves and self.intra and Bn >= 2
@@ -184,11 +186,21 @@ class GsitStack:
         B.unpack_rows(res, y, self.seg_len, valid_len, plan)
         return y
 
-    def forward(self, x, valid_len=None):
-        """x float32 [B, L, d] -> float32 [B, L, 2d].  The result lives in a buffer owned by this object."""
+    def forward(self, x, valid_len=None, out=None):
+        """x float32 [B, L, d] -> float32 [B, L, 2d].  The result lives in a buffer owned by this object, or in `out`
+        (float32 [B, L, 2d], contiguous) when one is given."""
+        if out is not None:
+            assert out.shape == (x.shape[0], x.shape[1], 2 * x.shape[2]) and out.dtype == torch.float32 and out.is_contiguous()
+        res = self._forward(x, valid_len, out)
+        if out is not None and res.data_ptr() != out.data_ptr():
+            out.copy_(res)
+            res = out
+        return res
+
+    def _forward(self, x, valid_len, out):
         if self.packed and valid_len is not None and self.batch_chunks == 1:
             try:
-                return self._forward_packed(x, valid_len)
+                return self._forward_packed(x, valid_len, out)
             except B.GsitError as e:
                 if e.code != 2:  # anything but "this shape is not covered": a real error
                     raise
