@@ -462,22 +462,35 @@ proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_co
       // ---- y = y1 + f W_2^T + b_2: each thread stores its own 512-byte row; padded rows +0 ----
       t_mbar_wait(g, bars + B_ACCY, i & 1);
       t_fence_after();
-      float4* dst = reinterpret_cast<float4*>(y + (int64_t)(row0 + r) * ldy);
+      // The rows leave through a per-warp transpose in shared memory (this warp's 32 rows of the hidden-chunk buffer,
+      // which nothing reads between the last second product and this warp's next chunk): a thread owns a row, but a
+      // store instruction that writes 16 bytes to each of 32 rows wastes half of every sector, so 32 columns at a time
+      // are written swizzled and read back with eight lanes per row -- each store then covers four full 128-byte lines.
+      const uint32_t scr = base + OFF_F + (warp & 3) * 4096;
+      const int rr0 = lane >> 3, jj = lane & 7;
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         uint32_t a[32];
         tmem_ld32(tl + COL_Y + 32 * c, a);
         tmem_wait_ld();
-        if (row0 + r < rows) {
 #pragma unroll
-          for (int e = 0; e < 32; e += 4) {
-            const float4 bb = ld_v4f(s_b2 + (32 * c + e) * 4);
-            float4 o = make_float4(v[32 * c + e] + __uint_as_float(a[e]) + bb.x, v[32 * c + e + 1] + __uint_as_float(a[e + 1]) + bb.y,
-                                   v[32 * c + e + 2] + __uint_as_float(a[e + 2]) + bb.z, v[32 * c + e + 3] + __uint_as_float(a[e + 3]) + bb.w);
-            if (!real) o = make_float4(0.f, 0.f, 0.f, 0.f);
-            dst[8 * c + (e >> 2)] = o;
-          }
+        for (int e = 0; e < 32; e += 4) {
+          const float4 bb = ld_v4f(s_b2 + (32 * c + e) * 4);
+          float4 o = make_float4(v[32 * c + e] + __uint_as_float(a[e]) + bb.x, v[32 * c + e + 1] + __uint_as_float(a[e + 1]) + bb.y,
+                                 v[32 * c + e + 2] + __uint_as_float(a[e + 2]) + bb.z, v[32 * c + e + 3] + __uint_as_float(a[e + 3]) + bb.w);
+          if (!real) o = make_float4(0.f, 0.f, 0.f, 0.f);
+          st_v4(scr + lane * 128 + ((((e >> 2)) ^ (lane & 7)) << 4), __float_as_uint(o.x), __float_as_uint(o.y), __float_as_uint(o.z),
+                __float_as_uint(o.w));
         }
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const int rr = 4 * k + rr0;
+          const float4 o = ld_v4f(scr + rr * 128 + ((jj ^ (rr & 7)) << 4));
+          const int grow = row0 + ((warp & 3) << 5) + rr;
+          if (grow < rows) *reinterpret_cast<float4*>(y + (int64_t)grow * ldy + 32 * c + 4 * jj) = o;
+        }
+        __syncwarp();
       }
       t_fence_before();  // orders these TMEM reads before the next tile's products (which wait for this thread's arrivals)
       real = real_next;
