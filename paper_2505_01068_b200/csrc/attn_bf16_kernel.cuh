@@ -5,6 +5,7 @@ namespace gsit {
 namespace {
 
 template <bool V> struct BoolTag { static constexpr bool value = V; };
+template <int V> struct IntTag { static constexpr int value = V; };
 
 template <typename C>
 __global__ void __launch_bounds__(NTHREADS, C::MINB)
@@ -120,14 +121,20 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       }
     }
 
-    // One pipeline stage (KT keys) for all query slabs of this warp.  RAGGED: the stage holds fewer than KT real keys.
-    auto process = [&](auto ragged_tag, const uint32_t sKs, const uint32_t sVs, const int krem) {
+    // One pipeline stage (KT keys) for all query slabs of this warp.  RAGGED: the stage holds fewer than KT real keys;
+    // the instantiation then covers only the first NTV score n-tiles (8 keys each, NTV even: whole 16-key groups of
+    // P V), so that a tile with few real keys costs proportionally less, and only its last two n-tiles are masked
+    // element by element.  Everything stays straight-line code inside an instantiation.
+    auto process = [&](auto ragged_tag, auto ntv_tag, const uint32_t sKs, const uint32_t sVs, const int krem) {
       constexpr bool RAGGED = decltype(ragged_tag)::value;
+      constexpr int NTV = decltype(ntv_tag)::value;  // n-tiles computed (== NT for a full tile)
+      static_assert(NTV % 2 == 0 && NTV >= 2 && NTV <= NT && (KT == KSTEP || !RAGGED || NTV == NT), "n-tile count");
       if constexpr (RAGGED) {
         // Rows past the valid length hold whatever follows in memory: clear this head's part of them in V so that a
         // zero weight times a NaN/Inf value cannot poison the accumulator (their scores become -inf below).  Warps
         // sharing the head write the same zeros.
-        for (int idx = lane; idx < (KT - krem) * (HD / 8); idx += 32) {
+        constexpr int KROWS = (KT == KSTEP) ? NTV * 8 : KT;  // key rows of the stage that the products read
+        for (int idx = lane; idx < (KROWS - krem) * (HD / 8); idx += 32) {
           const int row = krem + idx / (HD / 8), ch = cb + idx % (HD / 8);
           asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(sVs + swz<SWZ>(row * PITCH + ch * 16)), "r"(0) : "memory");
         }
@@ -167,12 +174,12 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if constexpr (HOIST) {
           if constexpr (HD == 8) {
 #pragma unroll
-            for (int j = 0; j < KSTEP / 32; ++j) { load_k8(j); load_v8(j); }
+            for (int j = 0; j < (NTV + 3) / 4; ++j) { load_k8(j); load_v8(j); }
           } else {
 #pragma unroll
-            for (int p = 0; p < NT / 2; ++p) load_k_pair(p);
+            for (int p = 0; p < NTV / 2; ++p) load_k_pair(p);
 #pragma unroll
-            for (int kk = 0; kk < KSTEP / 16; ++kk)
+            for (int kk = 0; kk < NTV / 2; ++kk)
 #pragma unroll
               for (int np = 0; np < NTO / 2; ++np) load_v_pair(kk, np);
           }
@@ -189,14 +196,15 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           // ---- S = Q K^T (raw dot products) ----
           if constexpr (HD == 8) {
 #pragma unroll
-            for (int j = 0; j < KSTEP / 32; ++j) {
+            for (int j = 0; j < (NTV + 3) / 4; ++j) {
               if constexpr (!HOIST) load_k8(j);
 #pragma unroll
-              for (int n = 4 * j; n < 4 * j + 4; ++n) mma_k8(S[n], QF[r_][0][0], QF[r_][0][1], KF[n][0][0]);
+              for (int n = 4 * j; n < 4 * j + 4; ++n)
+                if (n < NTV) mma_k8(S[n], QF[r_][0][0], QF[r_][0][1], KF[n][0][0]);
             }
           } else {
 #pragma unroll
-            for (int p = 0; p < NT / 2; ++p) {
+            for (int p = 0; p < NTV / 2; ++p) {
               if constexpr (!HOIST) load_k_pair(p);
 #pragma unroll
               for (int ks = 0; ks < KSQ; ++ks) {
@@ -211,19 +219,22 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           if constexpr (RAGGED) {
             const int c0 = kb + (lane & 3) * 2;
 #pragma unroll
-            for (int n = 0; n < NT; ++n) {
+            for (int n = (KT == KSTEP ? NTV - 2 : 0); n < NTV; ++n) {  // the invalid keys are a suffix of the last 16-key group
               if (c0 + n * 8 >= krem) S[n][0] = S[n][2] = -INFINITY;
               if (c0 + n * 8 + 1 >= krem) S[n][1] = S[n][3] = -INFINITY;
             }
           }
           // ---- online softmax (base 2, scale folded into sl2); pairwise trees keep dependency chains short ----
-          float t0[NT], t1[NT];
+          float t0[NTV], t1[NTV];
 #pragma unroll
-          for (int n = 0; n < NT; ++n) { t0[n] = fmaxf(S[n][0], S[n][1]); t1[n] = fmaxf(S[n][2], S[n][3]); }
+          for (int n = 0; n < NTV; ++n) { t0[n] = fmaxf(S[n][0], S[n][1]); t1[n] = fmaxf(S[n][2], S[n][3]); }
 #pragma unroll
-          for (int w = NT / 2; w >= 1; w >>= 1)
+          for (int cnt = NTV; cnt > 1; cnt = (cnt + 1) / 2)  // pairwise tree over any count
 #pragma unroll
-            for (int n = 0; n < w; ++n) { t0[n] = fmaxf(t0[n], t0[n + w]); t1[n] = fmaxf(t1[n], t1[n + w]); }
+            for (int n = 0; n < cnt / 2; ++n) {
+              t0[n] = fmaxf(t0[n], t0[n + (cnt + 1) / 2]);
+              t1[n] = fmaxf(t1[n], t1[n + (cnt + 1) / 2]);
+            }
           float mx0 = t0[0], mx1 = t1[0];
           mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
           mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
@@ -241,9 +252,9 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           // those same bf16 weights (a column of ones appended to V), so numerator and denominator of the softmax see
           // identical values.
           const float2 sl2v = make_float2(sl2, sl2), nm0 = make_float2(-ms0, -ms0), nm1 = make_float2(-ms1, -ms1);
-          uint32_t P[NT][2];
+          uint32_t P[NTV][2];
 #pragma unroll
-          for (int n = 0; n < NT; ++n) {
+          for (int n = 0; n < NTV; ++n) {
             const float2 x0 = __ffma2_rn(make_float2(S[n][0], S[n][1]), sl2v, nm0);
             const float2 x1 = __ffma2_rn(make_float2(S[n][2], S[n][3]), sl2v, nm1);
             P[n][0] = pack_bf16(ex2(x0.x), ex2(x0.y));
@@ -258,7 +269,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           }
           // ---- O += P V and l += P 1, the weights being the A operand ----
 #pragma unroll
-          for (int kk = 0; kk < KSTEP / 16; ++kk) {
+          for (int kk = 0; kk < NTV / 2; ++kk) {
             const uint32_t a0 = P[2 * kk][0], a1 = P[2 * kk][1], a2 = P[2 * kk + 1][0], a3 = P[2 * kk + 1][1];
             mma_k16(l[r_], a0, a1, a2, a3, 0x3F803F80u, 0x3F803F80u);  // B = ones: every column of the result is the row sum
             if constexpr (HD == 8) {
@@ -295,8 +306,16 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       int krem, yrow;
       locate(i, krem, yrow);
       const uint32_t sKs = sK + st * C::KV_BYTES, sVs = sV + st * C::KV_BYTES;
-      if (krem < KT) process(BoolTag<true>{}, sKs, sVs, krem);
-      else process(BoolTag<false>{}, sKs, sVs, KT);
+      if (krem >= KT) {
+        process(BoolTag<false>{}, IntTag<NT>{}, sKs, sVs, KT);
+      } else if constexpr (KT == KSTEP && NT == 8) {  // as many 16-key groups as hold real keys
+        if (krem <= 16) process(BoolTag<true>{}, IntTag<2>{}, sKs, sVs, krem);
+        else if (krem <= 32) process(BoolTag<true>{}, IntTag<4>{}, sKs, sVs, krem);
+        else if (krem <= 48) process(BoolTag<true>{}, IntTag<6>{}, sKs, sVs, krem);
+        else process(BoolTag<true>{}, IntTag<8>{}, sKs, sVs, krem);
+      } else {
+        process(BoolTag<true>{}, IntTag<NT>{}, sKs, sVs, krem);
+      }
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_empty + 8 * st);  // this warp is done with the stage
     }
