@@ -241,8 +241,9 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
           mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
           const float mn0 = fmaxf(m[r_][0], mx0), mn1 = fmaxf(m[r_][1], mx1);
-          const float ms0 = (mn0 == -INFINITY) ? 0.f : mn0 * sl2;
-          const float ms1 = (mn1 == -INFINITY) ? 0.f : mn1 * sl2;
+          // every key tile that is walked holds at least one real key, so the new maximum is finite (only the old one can
+          // be -inf, on the first tile, where the factor below becomes exp2(-inf) = 0)
+          const float ms0 = mn0 * sl2, ms1 = mn1 * sl2;
           const float al0 = ex2(fmaf(m[r_][0], sl2, -ms0)), al1 = ex2(fmaf(m[r_][1], sl2, -ms1));
           m[r_][0] = mn0;
           m[r_][1] = mn1;
