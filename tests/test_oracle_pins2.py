@@ -276,6 +276,55 @@ def test_stack_composition_shapes_and_concat():
     assert np.array_equal(y[..., :d], a) and np.array_equal(y[..., d:], b)
 
 
+def _torch_layer(tx, t, seg, pad, H, ring):
+    """One IM layer out of torch library routines (LayerNorm, linear, SDPA with a boolean mask built here from segment
+    ids); `ring` is the key-segment shift of the block pattern: 1 forward, 2 backward, 0 intra."""
+    B, L, d = tx.shape
+    h = F.layer_norm(tx, (d,), t["ln1_g"], t["ln1_b"], 1e-5)
+    qkv = F.linear(h, t["w_qkv"], t["b_qkv"]).view(B, L, 3, H, d // H)
+    seg_id = np.repeat(np.arange(3), seg)
+    mask = torch.from_numpy((seg_id[None, :] == (seg_id[:, None] + ring) % 3)[None, None] & ~pad[:, None, None, :])
+    att = F.scaled_dot_product_attention(qkv[:, :, 0].transpose(1, 2), qkv[:, :, 1].transpose(1, 2),
+                                         qkv[:, :, 2].transpose(1, 2), attn_mask=mask)
+    att = att.transpose(1, 2).reshape(B, L, d)
+    y1 = tx + F.linear(att, t["w_o"], t["b_o"])
+    h2 = F.layer_norm(y1, (d,), t["ln2_g"], t["ln2_b"], 1e-5)
+    y = y1 + F.linear(F.relu(F.linear(h2, t["w_1"], t["b_1"])), t["w_2"], t["b_2"])
+    return torch.where(torch.from_numpy(pad)[:, :, None], torch.zeros_like(y), y)
+
+
+def test_stack_against_library_composition_with_distinct_intra_heads():
+    """Eq. "All-Modal-In-One fusion": G_inter^{forward} and G_inter^{backward} encoders from the same input with their own
+    weights, feature concat, then the G_intra encoder -- here with a head count different from the ring encoders', two
+    layers per encoder, affine LayerNorms, biases and ragged lengths, composed independently from torch routines.  A wrong
+    block pattern, head count or operand order in any leg of oracle.gsit_stack_fwd moves the result far beyond 1e-10."""
+    rng = np.random.default_rng(18)
+    seg, B, d, H, IH = (5, 7, 6), 2, 8, 2, 4
+    x = rng.standard_normal((B, sum(seg), d))
+    vl = np.array([[5, 4, 6], [3, 7, 2]], dtype=np.int32)
+    pad = wk.padded_row_mask(seg, vl, B)
+    fw = [_layer_weights(rng, d, 4 * d) for _ in range(2)]
+    bw = [_layer_weights(rng, d, 4 * d) for _ in range(2)]
+    iw = [_layer_weights(rng, 2 * d, 8 * d) for _ in range(2)]
+    got = oracle.gsit_stack_fwd(x, fw, bw, iw, seg, H, IH, vl)
+    tt = lambda w: {k: (None if a is None else torch.from_numpy(a)) for k, a in w.items()}
+    a = b = torch.from_numpy(x)
+    for w in fw:
+        a = _torch_layer(a, tt(w), seg, pad, H, 1)
+    for w in bw:
+        b = _torch_layer(b, tt(w), seg, pad, H, 2)
+    c = torch.cat([a, b], dim=-1)
+    for w in iw:
+        c = _torch_layer(c, tt(w), seg, pad, IH, 0)
+    ref = c.numpy()
+    assert np.abs(got[~pad] - ref[~pad]).max() <= 1e-10
+    assert np.all(got[pad] == 0.0)
+    # the pins bite: the ring head count in the intra leg, or the rings swapped, is far outside the bound
+    wrong_heads = oracle.gsit_stack_fwd(x, fw, bw, iw, seg, H, H, vl)
+    swapped = oracle.gsit_stack_fwd(x, bw, fw, iw, seg, H, IH, vl)
+    assert np.abs(wrong_heads[~pad] - ref[~pad]).max() > 1e-4 and np.abs(swapped[~pad] - ref[~pad]).max() > 1e-4
+
+
 def test_workload_generators_are_seeded_and_shaped():
     a, b = wk.make_inputs(3, batch=2), wk.make_inputs(3, batch=2)
     assert np.array_equal(a["x"], b["x"]) and np.array_equal(a["valid_len"], b["valid_len"])
