@@ -174,9 +174,12 @@ gsit_status gsit_stack_head_fwd(const gsit_shape* shape, const float* c, int64_t
  *   - Limit: gsit_workspace_bytes(shape, GSIT_CALL_LAYER, d_ff) must not exceed GSIT_STATIC_SCRATCH_BYTES;
  *     larger problems are rejected with GSIT_ERR_WORKSPACE before anything is launched (split the batch).
  *   - The first call on each GPU looks up the array's device address (that GPU must be current); make that
- *     first call before starting any stream capture.
+ *     first call before starting any stream capture.  The CUDA driver loads device arrays lazily, so it is also at
+ *     this first call that the GPU's free memory drops by the array's size, once; later calls leave it unchanged.
  *   - All calls on a GPU share the one array, and it keeps the previous call's intermediates.  The layer
- *     overwrites every scratch region before reading it, so nothing needs clearing -- but two calls that
+ *     writes every scratch row that contributes to a real output row before reading it, so nothing needs clearing
+ *     (stale rows past the last real one may be read by a row tile; what is computed from them is discarded) -- but
+ *     two calls that
  *     overlap in time on the same GPU (different streams, or different host threads) race on it and both
  *     results are then undefined.  Order them on one stream or with events. */
 #define GSIT_STATIC_SCRATCH_BYTES (4u << 20)

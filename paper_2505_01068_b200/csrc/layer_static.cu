@@ -48,8 +48,9 @@ extern "C" gsit_status gsit_im_layer_fwd_static(const gsit_shape* shape, const g
   if (need > (size_t)GSIT_STATIC_SCRATCH_BYTES) return GSIT_ERR_WORKSPACE;  // problem too large for the fixed array
   void* scratch = nullptr;
   if (scratch_address(&scratch) != cudaSuccess) return GSIT_ERR_CUDA;
-  // Every region of the layer's scratch is written in full before it is read, so nothing has to be cleared even
-  // though the array still holds the previous call's intermediate results.
+  // Every scratch row that contributes to a real output row is written before it is read, so nothing has to be
+  // cleared even though the array still holds the previous call's intermediate results.  (Row tiles may read a few
+  // stale rows past the last real one; what is computed from them is discarded.)
   return gsit_im_layer_fwd(shape, weights, x, x_row_stride, y, y_row_stride, scratch,
                            (size_t)GSIT_STATIC_SCRATCH_BYTES, stream);
 }

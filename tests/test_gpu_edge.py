@@ -90,6 +90,22 @@ def test_custom_block_patterns_union_softmax(g, dtype):
         _run(g, q, k, v, seg, valid, oracle.PHASE_CUSTOM, dtype, custom=bits)
 
 
+@pytest.mark.parametrize("H,hd", [(4, 16), (2, 32), (2, 64), (8, 16), (1, 64)])
+def test_custom_block_patterns_every_head_width(g, H, hd):
+    """The union walk (two and three open blocks in a block row, a closed row, the empty mask) in every bf16 kernel
+    family: head_dim 16 and 32, and head_dim 64 (the tensor-memory kernel), over several key tiles per open block,
+    ragged last tiles and an empty key segment."""
+    rng = np.random.default_rng(500 + H * 64 + hd)
+    seg, B = (70, 200, 150), 3
+    q, k, v = wk.draw_qkv(rng, B, sum(seg), H, hd, "bf16")
+    valid = np.array([[70, 200, 150], [33, 129, 65], [70, 0, 1]], dtype=np.int32)
+    # unmasked naive graph; two open blocks in rows 0 and 1 with row 2 closed; three in row 2 only; a permutation-like
+    # ablation pattern; one block; nothing open
+    for bits in (0x1FF, 0b000101011, 0b111000000, 0b010001100, 0b000010000, 0):
+        _run(g, q, k, v, seg, valid, oracle.PHASE_CUSTOM, "bf16", custom=bits)
+        _run(g, q, k, v, seg, None, oracle.PHASE_CUSTOM, "bf16", custom=bits, nan_pad=False)
+
+
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
 def test_explicit_scale_and_fused_vs_separate(g, dtype):
     rng = np.random.default_rng(32)

@@ -7,7 +7,7 @@ import torch
 
 import oracle
 import workloads as wk
-from gpu_util import check_close, pad_mask, to_dev, to_np64, weights_to_dev
+from gpu_util import STACK_TOL, check_close, pad_mask, to_dev, to_np64, weights_to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -37,8 +37,8 @@ def test_cfg4_full_batch_stack_sampled_samples(g):
         ref = oracle.gsit_stack_fwd(inp["x"][b:b + 1], inp["fwd_layers"], inp["bwd_layers"], inp["intra_layers"], wl.seg_len,
                                     wl.heads, ih, valid[b:b + 1])
         err = np.abs(y[b:b + 1] - ref)
-        # ten bf16 layers deep: the per-call tolerance scaled by depth (single layers are held to it in test_gpu_parity)
-        assert err.max() <= 10 * 2e-2 and err.mean() <= 10 * 2e-3, (b, err.max(), err.mean())
+        # ten layers in sequence: the measured compounding of the storage rounding times 1.5 (see STACK_TOL)
+        assert err.max() <= STACK_TOL["max_abs"] and err.mean() <= STACK_TOL["mean_abs"], (b, err.max(), err.mean())
     # one layer of the same batch, held to the per-call tolerance
     w = inp["fwd_layers"][0]
     y1 = to_np64(g.im_layer_fwd(x_dev, weights_to_dev(w, "bf16"), wl.seg_len, wl.heads, vl, oracle.PHASE_INTER_FWD))

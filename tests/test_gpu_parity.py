@@ -6,7 +6,7 @@ import torch
 
 import oracle
 import workloads as wk
-from gpu_util import check_close, pad_mask, to_dev, to_np64, weights_to_dev
+from gpu_util import STACK_TOL, check_close, pad_mask, to_dev, to_np64, weights_to_dev
 
 pytestmark = pytest.mark.gpu
 PHASES = [oracle.PHASE_INTER_FWD, oracle.PHASE_INTER_BWD, oracle.PHASE_INTRA]
@@ -117,8 +117,35 @@ def test_cfg4_full_stack_bf16(g):
     got = to_np64(y)
     assert np.isfinite(got).all() and np.all(got[pm] == 0.0)
     err = np.abs(got - ref)
-    # ten bf16 layers deep: report against the per-call tolerance scaled by depth (each layer alone is checked above)
-    assert err.max() <= 10 * 2e-2 and err.mean() <= 10 * 2e-3, (err.max(), err.mean())
+    # ten layers in sequence: the measured compounding of the storage rounding times 1.5 (see STACK_TOL)
+    assert err.max() <= STACK_TOL["max_abs"] and err.mean() <= STACK_TOL["mean_abs"], (err.max(), err.mean())
+
+
+def test_cfg4_every_stack_layer_teacher_forced(g):
+    """Each of the ten layers of the MOSEI-shaped stack on its own, fed the ORACLE's previous activation (rounded to the
+    float32 residual stream the library stores), against the oracle's output of that layer at the per-call tolerance:
+    an error of one layer cannot hide behind, or be blamed on, the layers before it."""
+    inp = wk.make_inputs(4, batch=2)
+    wl = inp["workload"]
+    n_f, n_b, n_i, ih = wl.stack
+    valid = inp["valid_len"]
+    vl = torch.from_numpy(valid).cuda()
+    pm = pad_mask(wl.seg_len, valid, 2)
+
+    def ring(layers, phase, heads, a, name):
+        for i, w in enumerate(layers):
+            a32 = a.astype(np.float32)
+            ref = oracle.im_layer_fwd(a32, w, wl.seg_len, heads, valid, phase)
+            xd = to_dev(wk.fill_padding(a32, wl.seg_len, valid, np.nan))
+            y = g.im_layer_fwd(xd, weights_to_dev(w, "bf16"), wl.seg_len, heads, vl, phase)
+            check_close(to_np64(y), ref, "bf16", pm, f"{name} layer {i}, teacher-forced")
+            a = ref
+        return a
+
+    a = ring(inp["fwd_layers"], oracle.PHASE_INTER_FWD, wl.heads, inp["x"].astype(np.float64), "forward-ring")
+    b = ring(inp["bwd_layers"], oracle.PHASE_INTER_BWD, wl.heads, inp["x"].astype(np.float64), "backward-ring")
+    ring(inp["intra_layers"], oracle.PHASE_INTRA, ih, np.concatenate([a, b], axis=-1), "intra")
+    assert g.last_device_status() == (0, 0)
 
 
 def test_cfg5_scaled_hd64_bf16(g):
@@ -306,7 +333,7 @@ def test_host_pipeline_delivers_every_step(g):
         assert torch.equal(want.cpu(), y_host[i]), i
     ref = oracle.gsit_stack_fwd(xs[0], inp["fwd_layers"], inp["bwd_layers"], inp["intra_layers"], wl.seg_len, wl.heads, ih, vs[0])
     err = np.abs(y_host[0].numpy().astype(np.float64) - ref)
-    assert err.max() <= 10 * 2e-2 and err.mean() <= 10 * 2e-3, (err.max(), err.mean())
+    assert err.max() <= STACK_TOL["max_abs"] and err.mean() <= STACK_TOL["mean_abs"], (err.max(), err.mean())
     assert g.last_device_status() == (0, 0)
 
 
