@@ -12,7 +12,7 @@ CSRC = PKG / "csrc"
 INCLUDE = PKG.parent / "include"
 OBJ_DIR = PKG / "_build"
 LIB = PKG / "libgsit.so"
-SOURCES = ["gsit_api.cu", "attn_f32.cu", "attn_bf16.cu", "attn_tc.cu", "linear.cu", "gemm_tc.cu", "fused_layer.cu", "fused_layer_tc.cu", "fused_layer_tc128.cu", "layer_static.cu", "stack_head.cu", "rows.cu"]
+SOURCES = ["gsit_api.cu", "attn_f32.cu", "attn_bf16.cu", "attn_tc.cu", "attn_tcs.cu", "linear.cu", "gemm_tc.cu", "fused_layer.cu", "fused_layer_tc.cu", "fused_layer_tc128.cu", "layer_static.cu", "stack_head.cu", "rows.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", str(INCLUDE), "-I", str(CSRC)]
 

@@ -51,6 +51,9 @@ cudaError_t launch_attn_bf16(const Geometry& g, const __nv_bfloat16* q, const __
   const int var = g_attn_variant;
   // head_dim 64 is a dense contraction: tcgen05 / TMEM kernel (variant 9 keeps the mma.sync kernel for comparison)
   if (g.hd == 64 && var != 9) return launch_attn_tc_hd64(g, q, k, v, row_stride, out, lse, scale, st);
+  // head_dim 8 / 16 / 32 at widths that are multiples of 64: thread-per-row softmax on tensor-memory tiles (any non-zero
+  // knob value keeps the mma.sync kernel below, which also serves the narrower widths)
+  if (var == 0 && attn_tcs_supported(g)) return launch_attn_tcs(g, q, k, v, row_stride, out, lse, scale, st);
 #define GSIT_CASE(VAR_, HD_, CW_, R_, KS_, MB_)         \
   if (g.hd == HD_ && cw == CW_ && (var == VAR_ || VAR_ == 0)) \
     return launch_one<Cfg<HD_, CW_, R_, KS_, MB_>>(g, q, k, v, row_stride, out, lse, scale, st);

@@ -78,6 +78,11 @@ cudaError_t launch_attn_tc_hd64(const Geometry& g, const __nv_bfloat16* q, const
                                 const __nv_bfloat16* v, int64_t row_stride, __nv_bfloat16* out, float* lse,
                                 float scale, cudaStream_t st);
 
+// bf16 attention for head_dim 8 / 16 / 32 and d_model a multiple of 64 on tcgen05 with thread-per-row softmax (attn_tcs.cu)
+bool attn_tcs_supported(const Geometry& g);
+cudaError_t launch_attn_tcs(const Geometry& g, const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
+                            int64_t row_stride, __nv_bfloat16* out, float* lse, float scale, cudaStream_t st);
+
 // Linear layers  C = act(A W^T + bias) (+ residual), rows that are padding written as zero when
 // `mask_rows` is set.  A [M,K] (lda), W [N,K], C [M,N] (ldc), residual float [M,N] (ldr) or nullptr.
 struct LinearArgs {

@@ -25,14 +25,17 @@ EncodeTiledFn encode_tiled_fn() {
 
 // 2-D map over a [rows, d] bf16 view with row pitch `row_stride` elements; box = [CW columns, box_rows rows],
 // shared-memory swizzle matched to the box width.  Out-of-range rows read as zero.
-bool make_map(CUtensorMap* tm, const void* base, int64_t rows, int d, int64_t row_stride, int cw, int box_rows) {
+// `plain`: no swizzle (box rows are stored back to back), for boxes narrower than 32 bytes.
+bool make_map(CUtensorMap* tm, const void* base, int64_t rows, int d, int64_t row_stride, int cw, int box_rows,
+              bool plain = false) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (fn == nullptr) return false;
   const cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
   const cuuint64_t strides[1] = {(cuuint64_t)row_stride * 2};
   const cuuint32_t box[2] = {(cuuint32_t)cw, (cuuint32_t)box_rows};
   const cuuint32_t estr[2] = {1, 1};
-  const CUtensorMapSwizzle sw = (cw == 64) ? CU_TENSOR_MAP_SWIZZLE_128B
+  const CUtensorMapSwizzle sw = plain ? CU_TENSOR_MAP_SWIZZLE_NONE
+                                : (cw == 64) ? CU_TENSOR_MAP_SWIZZLE_128B
                                 : (cw == 32) ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
   return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
