@@ -116,7 +116,11 @@ gsit_status gsit_im_qkv_proj(const gsit_shape* shape, const void* x, int64_t x_r
  *            d for three separate tensors, 3d for the fused buffer written by gsit_im_qkv_proj
  *   out      [B, L, d] contiguous, heads concatenated along features
  *   lse      float [B, H, L] or NULL: natural-log-sum-exp of the scaled scores of each row
- *   workspace / workspace_bytes: gsit_workspace_bytes(shape, GSIT_CALL_ATTENTION, 0) bytes (may be 0/NULL). */
+ *   workspace / workspace_bytes: gsit_workspace_bytes(shape, GSIT_CALL_ATTENTION, 0) bytes, 4-byte aligned, or NULL / 0.
+ *            Optional: given the scratch, the bf16 kernels hand their work items to the SMs through a counter kept there
+ *            (cleared on `stream` by the call itself), which balances samples of different valid lengths; without it
+ *            the items are assigned in a fixed round-robin order.  The result is the same either way.  Calls that may
+ *            overlap in time need separate scratch. */
 gsit_status gsit_im_attention_fwd(const gsit_shape* shape, const void* q, const void* k, const void* v,
                                   int64_t row_stride, void* out, float* lse, void* workspace,
                                   size_t workspace_bytes, gsit_stream stream);
@@ -199,23 +203,6 @@ size_t gsit_workspace_bytes(const gsit_shape* shape, int which_call, int32_t d_f
 /* Synchronises `stream`, reads and clears the device status flags into *flags (HOST, may be NULL).
  * Returns GSIT_ERR_TIMEOUT if GSIT_DEVFLAG_TIMEOUT was set, GSIT_ERR_CUDA on a CUDA error, else GSIT_OK. */
 gsit_status gsit_last_device_status(gsit_stream stream, uint32_t* flags);
-
-/* Profiling aid (host state, off by default).  While enabled, every kernel launch of the library is bracketed
- * by a pair of CUDA events on the launching stream (up to 8192 launches are kept; later ones go unrecorded).
- * Do not enable it while a stream is being captured into a CUDA graph. */
-typedef enum { GSIT_KERNEL_ATTENTION = 0, GSIT_KERNEL_LINEAR = 1, GSIT_KERNEL_LAYERNORM = 2 } gsit_kernel_kind;
-gsit_status gsit_trace_enable(int on);
-/* Waits for the recorded events, returns the summed device time (ms) and launch count of one kernel kind since the
- * last gsit_trace_reset(); both outputs are HOST pointers. */
-gsit_status gsit_trace_read(int kernel_kind, float* total_ms, int32_t* launches);
-/* Per-launch device times (ms) of one kernel kind, in launch order, into out_ms[0..capacity); *launches receives
- * the number written.  HOST pointers. */
-gsit_status gsit_trace_launches(int kernel_kind, float* out_ms, int32_t capacity, int32_t* launches);
-gsit_status gsit_trace_reset(void);
-
-/* Tuning knob (host state): selects an alternative tile configuration of the bf16 attention kernel where the
- * shape has one; 0 restores the defaults.  Results are identical up to floating-point summation order. */
-gsit_status gsit_tune_attention(int variant);
 
 const char* gsit_status_string(gsit_status status);
 int gsit_version(void);

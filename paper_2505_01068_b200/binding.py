@@ -41,10 +41,12 @@ class LayerWeights(ctypes.Structure):
 
 EXPORTS = ("gsit_im_qkv_proj", "gsit_im_attention_fwd", "gsit_im_layer_fwd", "gsit_workspace_bytes",
            "gsit_last_device_status", "gsit_status_string", "gsit_version", "gsit_trace_enable", "gsit_trace_read",
-           "gsit_trace_launches", "gsit_trace_reset", "gsit_tune_attention", "gsit_im_layer_fwd_static", "gsit_stack_head_fwd",
+           "gsit_trace_launches", "gsit_trace_reset", "gsit_tune_attention", "gsit_test_expire_wait", "gsit_im_layer_fwd_static",
+           "gsit_stack_head_fwd",
            "gsit_plan_rows", "gsit_pack_rows", "gsit_unpack_rows")
 STATIC_SCRATCH_BYTES = 4 << 20
 KERNEL_ATTENTION, KERNEL_LINEAR, KERNEL_LAYERNORM = 0, 1, 2
+ATTN_DEFAULT, ATTN_UNFUSED, ATTN_LEGACY, ATTN_TMEM = 0, 8, 9, 10   # gsit_kernel_choice of include/gsit_test.h
 
 
 def load():
@@ -144,7 +146,15 @@ def last_device_status() -> tuple[int, int]:
 
 
 def tune_attention(variant: int):
+    """Test / measurement hook: selects a kernel family (ATTN_* above, or 1..7 for alternative mma.sync tile shapes)."""
     _check(load().gsit_tune_attention(int(variant)), "gsit_tune_attention")
+
+
+def expire_wait_selftest():
+    """Test hook: launches the kernel whose bounded wait must run out (see include/gsit_test.h)."""
+    lib = load()
+    lib.gsit_test_expire_wait.argtypes = [ctypes.c_void_p]
+    _check(lib.gsit_test_expire_wait(_stream()), "gsit_test_expire_wait")
 
 
 def trace_enable(on: bool):
@@ -179,9 +189,10 @@ def im_qkv_proj(x, w_qkv, b_qkv, seg_len, heads, valid_len=None, out=None):
 
 
 def im_attention_fwd(q, k, v, seg_len, valid_len=None, phase=PHASE_INTER_FWD, custom_mask=0, scale=0.0,
-                     want_lse=False, out=None):
+                     want_lse=False, out=None, workspace=None):
     """q, k, v: [B, L, H, hd] views sharing strides (e.g. qkv[:, :, i] of the fused buffer).  Returns out [B, L, d]
-    (and lse [B, H, L] float when want_lse)."""
+    (and lse [B, H, L] float when want_lse).  workspace: uint8 device tensor of workspace_bytes(shape, CALL_ATTENTION)
+    bytes (allocated here when not given)."""
     B, L, H, hd = q.shape
     d = H * hd
     for t in (q, k, v):
@@ -191,8 +202,12 @@ def im_attention_fwd(q, k, v, seg_len, valid_len=None, phase=PHASE_INTER_FWD, cu
     if out is None:
         out = torch.empty((B, L, d), dtype=q.dtype, device=q.device)
     lse = torch.empty((B, H, L), dtype=torch.float32, device=q.device) if want_lse else None
+    need = workspace_bytes(shape, CALL_ATTENTION)
+    if workspace is None and need > 0:
+        workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
     _check(load().gsit_im_attention_fwd(ctypes.byref(shape), _ptr(q), _ptr(k), _ptr(v), q.stride(1), _ptr(out),
-                                        _ptr(lse), None, 0, _stream()), "gsit_im_attention_fwd")
+                                        _ptr(lse), _ptr(workspace), 0 if workspace is None else workspace.numel(),
+                                        _stream()), "gsit_im_attention_fwd")
     return (out, lse) if want_lse else out
 
 

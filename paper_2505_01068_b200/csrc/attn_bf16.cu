@@ -12,6 +12,7 @@
 #include <cuda.h>
 
 #include "common.cuh"
+#include "ptx.cuh"
 #include "tensor_map.cuh"
 
 namespace gsit {

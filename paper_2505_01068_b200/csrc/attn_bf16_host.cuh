@@ -41,19 +41,21 @@ cudaError_t launch_one(const Geometry& g, const __nv_bfloat16* q, const __nv_bfl
 
 }  // namespace
 
-int g_attn_variant = 0;  // 0 = default tile configuration per shape; 1.. = alternatives (tuning knob)
+int g_attn_variant = 0;  // gsit_kernel_choice, or 1..7 = alternative tile configurations of the mma.sync attention
 
 cudaError_t launch_attn_bf16(const Geometry& g, const __nv_bfloat16* q, const __nv_bfloat16* k,
                              const __nv_bfloat16* v, int64_t row_stride, __nv_bfloat16* out, float* lse,
-                             float scale, cudaStream_t st) {
+                             float scale, int* next_item, cudaStream_t st) {
   if (g.batch > 65535 || g.d % 16 != 0) return cudaErrorNotSupported;
   const int cw = (g.d % 64 == 0) ? 64 : (g.d % 32 == 0) ? 32 : 16;
   const int var = g_attn_variant;
-  // head_dim 64 is a dense contraction: tcgen05 / TMEM kernel (variant 9 keeps the mma.sync kernel for comparison)
-  if (g.hd == 64 && var != 9) return launch_attn_tc_hd64(g, q, k, v, row_stride, out, lse, scale, st);
-  // head_dim 8 / 16 / 32 at widths that are multiples of 64: thread-per-row softmax on tensor-memory tiles (any non-zero
-  // knob value keeps the mma.sync kernel below, which also serves the narrower widths)
-  if (var == 0 && attn_tcs_supported(g)) return launch_attn_tcs(g, q, k, v, row_stride, out, lse, scale, st);
+  // head_dim 64 is a dense contraction: tcgen05 / TMEM kernel (GSIT_ATTN_LEGACY keeps the mma.sync kernel for comparison)
+  if (g.hd == 64 && var != GSIT_ATTN_LEGACY) return launch_attn_tc_hd64(g, q, k, v, row_stride, out, lse, scale, st);
+  // head_dim 16 / 32: thread-per-row softmax on tensor-memory tiles.  At head_dim 8 that kernel measures slower than the
+  // mma.sync kernel below (61 against 46 us at the MOSEI cross shape: a tcgen05 hand-over per 64 keys of one head costs
+  // more than the 8192 exponentials it feeds), so there it is selected by the knob only.
+  if (attn_tcs_supported(g) && (var == GSIT_ATTN_TMEM || (var == 0 && g.hd >= 16)))
+    return launch_attn_tcs(g, q, k, v, row_stride, out, lse, scale, next_item, st);
 #define GSIT_CASE(VAR_, HD_, CW_, R_, KS_, MB_)         \
   if (g.hd == HD_ && cw == CW_ && (var == VAR_ || VAR_ == 0)) \
     return launch_one<Cfg<HD_, CW_, R_, KS_, MB_>>(g, q, k, v, row_stride, out, lse, scale, st);

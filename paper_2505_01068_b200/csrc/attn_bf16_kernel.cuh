@@ -7,6 +7,11 @@ namespace {
 template <bool V> struct BoolTag { static constexpr bool value = V; };
 template <int V> struct IntTag { static constexpr int value = V; };
 
+#ifndef GSIT_MS_POLY
+#define GSIT_MS_POLY 0
+#endif
+constexpr unsigned MS_POLY = GSIT_MS_POLY;  // bit i: score n-tile i of a step takes the polynomial 2^x
+
 template <typename C>
 __global__ void __launch_bounds__(NTHREADS, C::MINB)
 attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -258,8 +263,14 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           for (int n = 0; n < NTV; ++n) {
             const float2 x0 = __ffma2_rn(make_float2(S[n][0], S[n][1]), sl2v, nm0);
             const float2 x1 = __ffma2_rn(make_float2(S[n][2], S[n][3]), sl2v, nm1);
-            P[n][0] = pack_bf16(ex2(x0.x), ex2(x0.y));
-            P[n][1] = pack_bf16(ex2(x1.x), ex2(x1.y));
+            if ((MS_POLY >> (n & 7)) & 1) {
+              const float2 p0 = ptx::ex2_poly2(x0), p1 = ptx::ex2_poly2(x1);
+              P[n][0] = __byte_perm(__float_as_uint(p0.x), __float_as_uint(p0.y), 0x7632);
+              P[n][1] = __byte_perm(__float_as_uint(p1.x), __float_as_uint(p1.y), 0x7632);
+            } else {
+              P[n][0] = __byte_perm(__float_as_uint(ex2(x0.x)), __float_as_uint(ex2(x0.y)), 0x7632);
+              P[n][1] = __byte_perm(__float_as_uint(ex2(x1.x)), __float_as_uint(ex2(x1.y)), 0x7632);
+            }
           }
           l[r_][0] *= al0;
           l[r_][2] *= al1;

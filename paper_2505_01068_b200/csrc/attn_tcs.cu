@@ -4,29 +4,32 @@
 // exponential, half a packed add and half a conversion.
 //
 // Decomposition (paper, Section "Inner Decomposition for Efficiency"; Appendix A "From Set to Set Aggregation"): a work
-// item is 128 query rows of one modality segment of one sample and a slice of 64 features (8 heads of 8, 4 of 16 or 2 of
-// 32); it walks only the key tiles (64 keys) of the segment(s) the Interlaced Mask opens for that block row, up to the
-// sample's valid length, and inside a key tile the heads of the slice one after the other.  A (key tile, head) pair is a
-// "unit".
+// item is 128 query rows of one modality segment of one sample and a narrow slice of features -- 32 bytes of every row
+// (a pair of heads of 8, or one head of 16), 64 bytes for one head of 32.  It walks only the key tiles (64 keys) of the
+// segment(s) the Interlaced Mask opens for that block row, up to the sample's valid length.  A (key tile, head) pair is a
+// "unit".  Items are small (at most 16 units at the MOSEI shape) and are handed out through an atomic counter, longest
+// first, so that all SMs finish together although the valid lengths differ from sample to sample.
 //
-// The grid is persistent, two CTAs per SM.  Roles inside a CTA of 6 warps:
-//   warp 0      TMA producer: the Q tile of an item, K and V tiles (64 keys x 128 bytes, 128-byte swizzle) in four-stage
-//               rings, straight out of the fused qkv buffer; it also decodes the work items and hands them to the others
-//   warp 1      owns 256 TMEM columns and issues every tcgen05.mma:
+// The grid is persistent, FOUR light CTAs per SM (128 TMEM columns, at most 80 registers per thread, 32 to 48 KB of shared
+// memory each): a thread-per-row softmax is a long dependent chain per warp, and it is the number of softmax warps per
+// scheduler (four) that keeps the exponential unit and the issue slots busy, not a deep pipeline inside one CTA.
+// Roles inside a CTA of 6 warps:
+//   warp 0      takes the next item from the counter, decodes it and hands it to the other warps through a ring of records;
+//               TMA producer: the Q tile of an item (two buffers), K and V tiles of 64 keys x 32 (64) bytes in rings
+//   warp 1      owns the TMEM columns and issues every tcgen05.mma:
 //                 S = Q_h K_h^T  M 128, N 64 (16 per 16-key group of a ragged tile), K 16 per step.  With head_dim 8 a
-//                   K step spans a pair of heads in the K tile; the A operand is then [q_h, 0] or [0, q_h]: the Q tile is
-//                   loaded head by head as 16-byte rows and the second core matrix of the step is a block of zeros,
+//                   K step spans the pair of heads in the K tile; the A operand is then [q_h, 0] or [0, q_h]: the Q tile is
+//                   loaded head by head as 16-byte rows and the other core matrix of the step is a block of zeros,
 //                   reached through the descriptor's leading byte offset, so the neighbour head contributes nothing
-//                 O_h += P V_h   M 128, N 16 (32 for head_dim 32), K 16 per step; A = P from TMEM, B = the V tile as
-//                   loaded (N-contiguous).  With head_dim 8, N = 16 covers the head pair; the neighbour's 8 columns of
-//                   the accumulator are never read
-//               S is double-buffered, so the scores of unit u+1 are computed while the softmax works on unit u
-//   warps 2..5  softmax: thread = query row = TMEM lane.  tcgen05.ld of the scores, running maximum and sum per head in
-//               shared memory, P (bf16 pairs) written over the scores it came from, O rescaled in TMEM only when the
-//               maximum has grown by more than 2^8.  Warps whose 32 rows hold no real query skip the arithmetic.
-// TMEM columns: [0,64) and [64,128) S fp32 / P bf16x2 (first 32 columns of each), [128,256) O, one block of 16 (32)
-// columns per head.  Every wait is bounded; when one expires GSIT_DEVFLAG_TIMEOUT is raised, the CTA's other waits give
-// up at once, and the CTA still releases its TMEM and returns.
+//                 O_h += P V     M 128, N 16 (32), K 16 per step; A = P from TMEM, B = the V tile as loaded
+//                   (N-contiguous).  With head_dim 8, N = 16 covers the head pair; the neighbour's 8 columns of each
+//                   head's accumulator are never read
+//   warps 2..5  softmax: thread = query row = TMEM lane.  Two passes over the scores in groups of 16 columns (maximum,
+//               then weights), running maximum and sum in registers, O rescaled in TMEM only when the maximum has grown by
+//               more than 2^8.  Warps whose 32 rows hold no real query skip the arithmetic.
+// TMEM columns: [0,64) S fp32, [64,96) P bf16x2, [96,128) one accumulator of 16 (32) columns per head.  Every wait is
+// bounded; when one expires GSIT_DEVFLAG_TIMEOUT is raised, the CTA's other waits give up at once, and the CTA still
+// releases its TMEM and returns.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -39,33 +42,53 @@ namespace {
 
 using namespace ptx;
 
-constexpr int SQ = 128, SK = 64, SLICE = 64;
-constexpr int S_STAGES = 4;
-constexpr int S_KV_BYTES = SK * 128;
+constexpr int SQ = 128, SK = 64;
 constexpr int S_THREADS = 192;
-constexpr int S_TMEM_COLS = 256, S_COL_O = 128;
+constexpr int S_TMEM_COLS = 128, S_COL_P = 64, S_COL_O = 96;
+constexpr int S_CTAS_PER_SM = 4;
 constexpr int S_ITEM_SLOTS = 4;
+constexpr int S_QBUF = 8192;  // bytes reserved per Q buffer
+#ifndef GSIT_POLY_PAIRS
+#define GSIT_POLY_PAIRS 0x52
+#endif
+// The weights are cut to bf16 by dropping the low 16 bits (one byte permute on the integer pipe per pair; the rounding
+// conversion would occupy the special-function unit as long as an exponential).  Dropping bits loses on average
+// 0.72 * 2^-9 of a value whose mantissa is spread like that of an exponential, so every weight is raised by that factor
+// beforehand (it is one constant added to the exponent) and the row sum, which is taken of the raised values in float, is
+// lowered by it at the end: the weights are then unbiased, with the same spread as round-to-nearest.
+constexpr float TRUNC_GAIN = 1.0f + 0.72f / 512.0f;
+constexpr float TRUNC_LOG2 = 0.0020273f;  // log2(TRUNC_GAIN)
+constexpr unsigned POLY_PAIRS = GSIT_POLY_PAIRS;  // bit i: pair i of every 16-key group takes the polynomial 2^x
 // barriers (8 bytes each), relative to the barrier block
-constexpr int B_QFULL = 0, B_QEMPTY = 8, B_KFULL = 16, B_VFULL = 48, B_KEMPTY = 80, B_VEMPTY = 112, B_SFULL = 144,
-              B_PFULL = 160, B_OFINAL = 176, B_TMEM_SLOT = 184, B_GAVE_UP = 188, B_ITEMBAR = 192, B_ITEMS = 256,
-              B_STATE = 512;
+constexpr int B_QFULL = 0, B_QEMPTY = 16, B_SFULL = 32, B_PFULL = 48, B_OFINAL = 64, B_TMEM_SLOT = 72, B_GAVE_UP = 76,
+              B_ITEMBAR = 80, B_ITEMS = 256, B_KFULL = 512, B_VFULL = 576, B_KEMPTY = 640, B_VEMPTY = 704, B_END = 768;
 
 template <int HD>
 struct SCfg {
-  static constexpr int G = SLICE / HD;             // heads per slice
-  static constexpr int NPV = HD < 16 ? 16 : HD;    // N of O_h += P V
-  // head_dim 8: per head pair [q_even 2 KB][zeros 2 KB][q_odd 2 KB], rows of 16 bytes; otherwise 128 rows x 128 bytes
-  static constexpr int Q_BYTES = (HD == 8) ? 4 * 6144 : SQ * 128;
-  static constexpr int OFF_K = Q_BYTES, OFF_V = OFF_K + S_STAGES * S_KV_BYTES, OFF_BAR = OFF_V + S_STAGES * S_KV_BYTES;
-  static constexpr int SMEM = OFF_BAR + B_STATE + G * 2 * SQ * 4 + 1024 /* alignment slack */;
+  static constexpr int SLW = (HD == 32) ? 32 : 16;   // features per slice
+  static constexpr int ROWB = SLW * 2;               // bytes per tile row
+  static constexpr int G = SLW / HD;                 // heads per slice
+  static constexpr int NPV = SLW;                    // N of O_h += P V
+  static constexpr uint32_t SWZ = (ROWB == 32) ? 6u : 4u;   // descriptor code of the 32-byte / 64-byte swizzle
+  static constexpr uint32_t SBO = 8 * ROWB;          // bytes between groups of 8 rows
+  static constexpr int KV_BYTES = SK * ROWB;
+  static constexpr int STAGES = 4;
+  static constexpr int Q_TX = SQ * ROWB;             // bytes TMA delivers per Q tile
+  static constexpr int OFF_K = 2 * S_QBUF, OFF_V = OFF_K + STAGES * KV_BYTES, OFF_BAR = OFF_V + STAGES * KV_BYTES;
+  static constexpr int SMEM = OFF_BAR + B_END + 1024 /* alignment slack */;
 };
+
+// Descriptor of a swizzled tile as TMA wrote it (rows of 32 or 64 bytes): groups of 8 rows `sbo` bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw(uint32_t addr, uint32_t sbo, uint32_t code) {
+  return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)(sbo >> 4) << 32) | (1ull << 46) | ((uint64_t)code << 61);
+}
 
 // One work item (16 ints = one 64-byte record of the hand-over ring).
 struct SItem {
   int b, c, s, q0;
   int rows_in_tile;  // rows of the tile this CTA writes (padding included in the padded layout)
   int q_real;        // rows that receive a computed result
-  int T;             // key tiles to walk
+  int T;             // key tiles to walk; -1 = no more items
   int kn0, kn1, kn2, nk0, nk1;  // real keys per open key segment, key tiles of the first two
   int kb0, kb1, kb2;            // first row of each key segment in the activation matrices
   int grow0;                    // first row of the query tile in the activation matrices
@@ -122,9 +145,8 @@ __device__ __forceinline__ void publish_item(uint32_t bars, const SItem& it, int
   }
   __syncwarp();
 }
-__device__ __forceinline__ SItem fetch_item(const WaitCtx& wc, uint32_t bars, int k, int lane) {
-  const int slot = k % S_ITEM_SLOTS;
-  mbar_wait(wc, bars + B_ITEMBAR + 8 * slot, (k / S_ITEM_SLOTS) & 1);
+// Copies record `slot` to registers and releases the slot (one arrival per warp).
+__device__ __forceinline__ SItem read_item(uint32_t bars, int slot, int lane) {
   const uint32_t a = bars + B_ITEMS + 64 * slot;
   SItem it;
   asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(it.b), "=r"(it.c), "=r"(it.s), "=r"(it.q0) : "r"(a) : "memory");
@@ -135,40 +157,43 @@ __device__ __forceinline__ SItem fetch_item(const WaitCtx& wc, uint32_t bars, in
   if (lane == 0) mbar_arrive(bars + B_ITEMBAR + 8 * S_ITEM_SLOTS + 8 * slot);
   return it;
 }
-
-template <int V> struct IntTag { static constexpr int value = V; };
-template <bool V> struct BoolTag { static constexpr bool value = V; };
+__device__ __forceinline__ SItem fetch_item(const WaitCtx& wc, uint32_t bars, int k, int lane) {
+  const int slot = k % S_ITEM_SLOTS;
+  const bool ok = mbar_wait(wc, bars + B_ITEMBAR + 8 * slot, (k / S_ITEM_SLOTS) & 1);
+  SItem it = read_item(bars, slot, lane);
+  if (!ok) it.T = -1;  // the hand-over itself timed out: stop (the flag has been raised)
+  return it;
+}
 
 template <int HD>
-__global__ void __launch_bounds__(S_THREADS, 2)
+__global__ void __launch_bounds__(S_THREADS, S_CTAS_PER_SM)
 attn_tcs_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const Geometry g, __nv_bfloat16* __restrict__ out,
                 float* __restrict__ lse, const float sl2 /* scale * log2(e) */, const int slices, const int seg_order,
-                const int n_items) {
+                const int n_items, int* __restrict__ next_item /* zeroed counter, or nullptr = static round robin */) {
   using C = SCfg<HD>;
-  constexpr int G = C::G, NPV = C::NPV;
+  constexpr int G = C::G, NPV = C::NPV, STAGES = C::STAGES, KVB = C::KV_BYTES, ROWB = C::ROWB;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t sQ = base, sK = base + C::OFF_K, sV = base + C::OFF_V, bars = base + C::OFF_BAR;
-  const uint32_t sState = bars + B_STATE;  // running maximum and sum: float [G][2][128]
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const WaitCtx wc{g.status, bars + B_GAVE_UP};
 
   // ---- set-up, once per CTA: barriers, the zero blocks of the Q layout, tensor memory ----
   if (tid == 0) {
-    mbar_init(bars + B_QFULL, 1);
-    mbar_init(bars + B_QEMPTY, 1);
 #pragma unroll
-    for (int i = 0; i < S_STAGES; ++i) {
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bars + B_QFULL + 8 * i, 1);
+      mbar_init(bars + B_QEMPTY + 8 * i, 1);
+    }
+    mbar_init(bars + B_SFULL, 1);
+    mbar_init(bars + B_PFULL, 4);  // one arrival per softmax warp
+#pragma unroll
+    for (int i = 0; i < STAGES; ++i) {
       mbar_init(bars + B_KFULL + 8 * i, 1);
       mbar_init(bars + B_VFULL + 8 * i, 1);
       mbar_init(bars + B_KEMPTY + 8 * i, 1);
       mbar_init(bars + B_VEMPTY + 8 * i, 1);
-    }
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(bars + B_SFULL + 8 * i, 1);
-      mbar_init(bars + B_PFULL + 8 * i, 4);  // one arrival per softmax warp
     }
     mbar_init(bars + B_OFINAL, 1);
     for (int i = 0; i < S_ITEM_SLOTS; ++i) {
@@ -179,8 +204,8 @@ attn_tcs_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     mbar_init_fence();
   }
   if constexpr (HD == 8) {
-    for (int i = tid; i < 4 * 128; i += S_THREADS)  // 4 pairs x 2 KB of zeros, 16 bytes per step
-      st_shared_v4(sQ + (i >> 7) * 6144 + 2048 + (i & 127) * 16, 0, 0, 0, 0);
+    // Q buffer: [q_even 2 KB][zeros 2 KB][q_odd 2 KB], rows of 16 bytes
+    for (int i = tid; i < 2 * 128; i += S_THREADS) st_shared_v4(sQ + (i >> 7) * S_QBUF + 2048 + (i & 127) * 16, 0, 0, 0, 0);
     fence_async_smem();
   }
   if (warp == 1) tmem_alloc(bars + B_TMEM_SLOT, S_TMEM_COLS);
@@ -191,98 +216,127 @@ attn_tcs_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tmem) : "r"(bars + B_TMEM_SLOT) : "memory");
 
   if (warp == 0) {
-    // ================================ TMA producer ================================
-    int n_q = 0, n_kv = 0, k = 0;
-    for (int w = blockIdx.x; w < n_items; w += gridDim.x, ++k) {
-      const SItem it = decode_item(g, w, slices, seg_order);
+    // ================================ scheduler and TMA producer ================================
+    int n_q = 0, n_kv = 0;
+    for (int k = 0;; ++k) {
+      int w;
+      if (next_item != nullptr) {
+        w = (lane == 0) ? atomicAdd(next_item, 1) : 0;
+        w = __shfl_sync(0xffffffffu, w, 0);
+      } else {
+        w = blockIdx.x + k * gridDim.x;
+      }
       if (k >= S_ITEM_SLOTS)
         mbar_wait(wc, bars + B_ITEMBAR + 8 * S_ITEM_SLOTS + 8 * (k % S_ITEM_SLOTS), ((k / S_ITEM_SLOTS) - 1) & 1);
+      if (w >= n_items || cta_gave_up(wc)) {
+        SItem end = {};
+        end.T = -1;
+        publish_item(bars, end, k, lane);
+        break;
+      }
+      const SItem it = decode_item(g, w, slices, seg_order);
       publish_item(bars, it, k, lane);
       if (it.T == 0) continue;
-      if (n_q > 0) mbar_wait(wc, bars + B_QEMPTY, (n_q - 1) & 1);
+      const int qb = n_q & 1;
+      if (n_q >= 2) mbar_wait(wc, bars + B_QEMPTY + 8 * qb, ((n_q >> 1) - 1) & 1);
       if (elect_one()) {
-        mbar_expect_tx(bars + B_QFULL, SQ * 128);
+        mbar_expect_tx(bars + B_QFULL + 8 * qb, C::Q_TX);
         if constexpr (HD == 8) {
-#pragma unroll
-          for (int h = 0; h < 8; ++h)
-            tma_load_2d(sQ + (h >> 1) * 6144 + (h & 1) * 4096, &tmQ, it.c * SLICE + h * 8, it.grow0, bars + B_QFULL);
+          tma_load_2d(sQ + qb * S_QBUF, &tmQ, it.c * 16, it.grow0, bars + B_QFULL + 8 * qb);
+          tma_load_2d(sQ + qb * S_QBUF + 4096, &tmQ, it.c * 16 + 8, it.grow0, bars + B_QFULL + 8 * qb);
         } else {
-          tma_load_2d(sQ, &tmQ, it.c * SLICE, it.grow0, bars + B_QFULL);
+          tma_load_2d(sQ + qb * S_QBUF, &tmQ, it.c * C::SLW, it.grow0, bars + B_QFULL + 8 * qb);
         }
       }
       ++n_q;
       for (int i = 0; i < it.T; ++i, ++n_kv) {
         int krem, yrow;
         locate(it, i, krem, yrow);
-        const int st = n_kv % S_STAGES, use = n_kv / S_STAGES;
+        const int st = n_kv % STAGES, use = n_kv / STAGES;
         if (use > 0) mbar_wait(wc, bars + B_KEMPTY + 8 * st, (use - 1) & 1);
         if (elect_one()) {
-          mbar_expect_tx(bars + B_KFULL + 8 * st, S_KV_BYTES);
-          tma_load_2d(sK + st * S_KV_BYTES, &tmK, it.c * SLICE, yrow, bars + B_KFULL + 8 * st);
+          mbar_expect_tx(bars + B_KFULL + 8 * st, KVB);
+          tma_load_2d(sK + st * KVB, &tmK, it.c * C::SLW, yrow, bars + B_KFULL + 8 * st);
         }
         if (use > 0) mbar_wait(wc, bars + B_VEMPTY + 8 * st, (use - 1) & 1);
         if (elect_one()) {
-          mbar_expect_tx(bars + B_VFULL + 8 * st, S_KV_BYTES);
-          tma_load_2d(sV + st * S_KV_BYTES, &tmV, it.c * SLICE, yrow, bars + B_VFULL + 8 * st);
+          mbar_expect_tx(bars + B_VFULL + 8 * st, KVB);
+          tma_load_2d(sV + st * KVB, &tmV, it.c * C::SLW, yrow, bars + B_VFULL + 8 * st);
         }
       }
     }
   } else if (warp == 1) {
     // ================================ MMA issuer ================================
     constexpr uint32_t IDESC_PV = idesc_bf16(NPV, true);
-    int n_q = 0, n_kv = 0, n_u = 0, k = 0;  // Q tiles, key tiles and units consumed so far
-    for (int w = blockIdx.x; w < n_items; w += gridDim.x, ++k) {
-      const SItem it = fetch_item(wc, bars, k, lane);
+    int n_q = 0, n_kv = 0, n_u = 0;  // Q tiles, key tiles and units consumed so far
+    for (int k = 0;; ++k) {
+      SItem it;
+      {
+        const int slot = k % S_ITEM_SLOTS;
+        const bool ok = mbar_wait(wc, bars + B_ITEMBAR + 8 * slot, (k / S_ITEM_SLOTS) & 1);
+        it = read_item(bars, slot, lane);
+        if (!ok) it.T = -1;
+      }
+      if (it.T < 0) break;
       if (it.T == 0) continue;
-      const int U = it.T * G;
-      // S[nu & 1] = Q_h K_h^T for unit u of the item.  The buffer was last read (as P) by the P V of unit u - 2, which
-      // this thread has issued before; tcgen05.mma instructions of one thread execute in issue order.
-      auto issue_qk = [&](int u) {
-        const int j = u / G, h = u - j * G, n = n_kv + j, st = n % S_STAGES, nu = n_u + u;
-        if (h == 0) mbar_wait(wc, bars + B_KFULL + 8 * st, (n / S_STAGES) & 1);
-        int krem, yrow;
-        locate(it, j, krem, yrow);
-        const int ncols = (krem >= SK) ? SK : ((krem + 15) >> 4) << 4;
+      const int U = it.T * G, qb = n_q & 1;
+      const uint32_t sQb = sQ + qb * S_QBUF;
+      mbar_wait(wc, bars + B_QFULL + 8 * qb, (n_q >> 1) & 1);
+      // Round u: the P V of unit u - 1 (once its weights are in TMEM), then the scores of unit u.  The softmax warps have
+      // finished reading S before they release P, so S may be overwritten then; and tcgen05.mma instructions of one
+      // thread execute in issue order, so P is read by the P V before the softmax of unit u (which waits for the scores
+      // issued after it) writes it again.
+      int krem_prev = 0;
+#pragma unroll 1
+      for (int u = 0; u <= U; ++u) {
+        int krem = 0, st = 0, h = 0, j = 0;
+        if (u < U) {
+          j = u / G; h = u - j * G;
+          const int n = n_kv + j;
+          st = n % STAGES;
+          int yrow;
+          locate(it, j, krem, yrow);
+          if (h == 0) mbar_wait(wc, bars + B_KFULL + 8 * st, (n / STAGES) & 1);
+        }
+        int pst = 0, ph = 0, pj = 0;
+        if (u > 0) {
+          const int v = u - 1, nu = n_u + v;
+          pj = v / G; ph = v - pj * G;
+          const int n = n_kv + pj;
+          pst = n % STAGES;
+          // P of unit v is in TMEM (and, for the first unit of an item, the previous item's O has been read)
+          mbar_wait(wc, bars + B_PFULL, nu & 1);
+          if (ph == 0) mbar_wait(wc, bars + B_VFULL + 8 * pst, (n / STAGES) & 1);
+        }
         tc_fence_after();
         if (elect_one()) {
-          const uint32_t d = tmem + 64 * (nu & 1), idesc = idesc_bf16(ncols, false);
-          const uint32_t kt = sK + st * S_KV_BYTES;
-          if constexpr (HD == 8) {
-            // [q_h, 0] for an even head, [0, q_h] for an odd one: start at q_even or at the zeros, 2 KB to the other half
-            const uint64_t a = smem_desc_plain(sQ + (h >> 1) * 6144 + (h & 1) * 2048, 2048, 128);
-            umma_ss(d, a, smem_desc_sw128(kt + 32 * (h >> 1)), idesc, 0);
-          } else {
-#pragma unroll
-            for (int ks = 0; ks < HD / 16; ++ks)
-              umma_ss(d, smem_desc_sw128(sQ + 2 * HD * h + 32 * ks), smem_desc_sw128(kt + 2 * HD * h + 32 * ks), idesc, ks > 0);
+          if (u > 0) {
+            const int ksteps = (krem_prev >= SK) ? SK / 16 : (krem_prev + 15) >> 4;
+            const uint32_t vt = sV + pst * KVB;
+            for (int kk = 0; kk < ksteps; ++kk)  // 16 keys per step: two groups of 8 rows of the V tile
+              umma_ts(tmem + S_COL_O + NPV * ph, tmem + S_COL_P + 8 * kk, smem_desc_sw(vt + 2 * C::SBO * kk, C::SBO, C::SWZ),
+                      IDESC_PV, (pj > 0 || kk > 0) ? 1u : 0u);
+            if (ph == G - 1) umma_commit(bars + B_VEMPTY + 8 * pst);  // also: O holds key tiles 0..pj of every head
+            if (u == U) umma_commit(bars + B_OFINAL);
           }
-          if (h == G - 1) umma_commit(bars + B_KEMPTY + 8 * st);
-          if (u == U - 1) umma_commit(bars + B_QEMPTY);
-          umma_commit(bars + B_SFULL + 8 * (nu & 1));
+          if (u < U) {
+            const int ncols = (krem >= SK) ? SK : ((krem + 15) >> 4) << 4;
+            const uint32_t idesc = idesc_bf16(ncols, false), kt = sK + st * KVB;
+            if constexpr (HD == 8) {
+              // [q_h, 0] for the even head, [0, q_h] for the odd one: start at q_even or at the zeros, 2 KB to the other half
+              umma_ss(tmem, smem_desc_plain(sQb + h * 2048, 2048, 128), smem_desc_sw(kt, C::SBO, C::SWZ), idesc, 0);
+            } else {
+#pragma unroll
+              for (int ks = 0; ks < HD / 16; ++ks)
+                umma_ss(tmem, smem_desc_sw(sQb + 32 * ks, C::SBO, C::SWZ), smem_desc_sw(kt + 32 * ks, C::SBO, C::SWZ), idesc, ks > 0);
+            }
+            if (h == G - 1) umma_commit(bars + B_KEMPTY + 8 * st);
+            if (u == U - 1) umma_commit(bars + B_QEMPTY + 8 * qb);
+            umma_commit(bars + B_SFULL);
+          }
         }
         __syncwarp();
-      };
-      mbar_wait(wc, bars + B_QFULL, n_q & 1);
-      issue_qk(0);
-      for (int u = 0; u < U; ++u) {
-        if (u + 1 < U) issue_qk(u + 1);  // scores of the next unit, ahead of this unit's P V
-        const int j = u / G, h = u - j * G, n = n_kv + j, st = n % S_STAGES, nu = n_u + u;
-        int krem, yrow;
-        locate(it, j, krem, yrow);
-        const int ksteps = (krem >= SK) ? SK / 16 : (krem + 15) >> 4;
-        // P of this unit is in TMEM (and, for the first unit of an item, the previous item's O has been read)
-        mbar_wait(wc, bars + B_PFULL + 8 * (nu & 1), (nu >> 1) & 1);
-        if (h == 0) mbar_wait(wc, bars + B_VFULL + 8 * st, (n / S_STAGES) & 1);
-        tc_fence_after();
-        if (elect_one()) {
-          const uint32_t vt = sV + st * S_KV_BYTES + ((HD == 8) ? 32 * (h >> 1) : 2 * HD * h);
-          for (int kk = 0; kk < ksteps; ++kk)  // 16 keys per step: two 8-row groups = 2048 bytes of the V tile
-            umma_ts(tmem + S_COL_O + NPV * h, tmem + 64 * (nu & 1) + 8 * kk, smem_desc_sw128(vt + 2048 * kk), IDESC_PV,
-                    (j > 0 || kk > 0) ? 1u : 0u);
-          if (h == G - 1) umma_commit(bars + B_VEMPTY + 8 * st);  // also: O holds key tiles 0..j of every head
-          if (u == U - 1) umma_commit(bars + B_OFINAL);
-        }
-        __syncwarp();
+        krem_prev = krem;
       }
       n_kv += it.T;
       n_u += U;
@@ -294,145 +348,161 @@ attn_tcs_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const int r = (wq << 5) + lane;                        // row in the tile = TMEM lane
     const uint32_t tl = tmem + ((uint32_t)(wq << 5) << 16);
     const float2 sl2v = make_float2(sl2, sl2);
-    const uint32_t my_state = sState + r * 4;              // + (2 h + {0: maximum, 1: sum}) * 512
-    int n_kv = 0, n_u = 0, n_items_done = 0, k = 0;
+    int n_kv = 0, n_u = 0, n_items_done = 0;
 
-    for (int w = blockIdx.x; w < n_items; w += gridDim.x, ++k) {
+    for (int k = 0;; ++k) {
       const SItem it = fetch_item(wc, bars, k, lane);
+      if (it.T < 0) break;
       const int64_t grow = (int64_t)it.grow0 + r;
-      uint4* dst = reinterpret_cast<uint4*>(out + grow * g.d + it.c * SLICE);
+      uint4* dst = reinterpret_cast<uint4*>(out + grow * g.d + it.c * C::SLW);
       float* lse_row = (lse != nullptr) ? lse + ((int64_t)it.b * g.heads + it.c * G) * g.L + g.seg_off[it.s] + it.q0 + r : nullptr;
-      if (it.T == 0) {  // nothing to attend (padding rows only, or an empty key set): exact zeros, lse = -inf
+      const bool warp_active = (wq << 5) < it.q_real;  // some row of this warp receives a result
+      if (it.T == 0 || !warp_active) {
+        // nothing to compute for these rows (padding only, or an empty key set): exact zeros, lse = -inf
         if (r < it.rows_in_tile) {
 #pragma unroll
-          for (int c = 0; c < 8; ++c) dst[c] = make_uint4(0, 0, 0, 0);
+          for (int c = 0; c < ROWB / 16; ++c) dst[c] = make_uint4(0, 0, 0, 0);
           if (lse_row != nullptr)
             for (int h = 0; h < G; ++h) lse_row[(int64_t)h * g.L] = -INFINITY;
         }
-        continue;
+        if (it.T == 0) continue;
       }
-      const bool warp_active = (wq << 5) < it.q_real;  // some row of this warp receives a result
-
-      // One unit: NCH = 16-key groups of the tile that hold real keys (4 = all), MASKED = the last group is partly padding.
-      auto unit = [&](auto nch_tag, auto masked_tag, const int j, const int h, const int n, const int nu, const int krem) {
-        constexpr int NCH = decltype(nch_tag)::value;
-        constexpr bool MASKED = decltype(masked_tag)::value;
-        const int sb = nu & 1;
-        const uint32_t tS = tl + 64 * sb;
-        uint32_t sr[NCH][16];
-#pragma unroll
-        for (int c = 0; c < NCH; ++c) tmem_ld16(tS + 16 * c, sr[c]);
-        float m_used = -INFINITY, l = 0.f;
-        if (j > 0) {
-          asm volatile("ld.shared.f32 %0, [%1];" : "=f"(m_used) : "r"(my_state + (2 * h) * 512) : "memory");
-          asm volatile("ld.shared.f32 %0, [%1];" : "=f"(l) : "r"(my_state + (2 * h + 1) * 512) : "memory");
-        }
-        tmem_wait_ld();
-        if constexpr (MASKED) {  // keys past the valid length get weight exactly zero
-#pragma unroll
-          for (int e = 0; e < 16; ++e)
-            if ((NCH - 1) * 16 + e >= krem) sr[NCH - 1][e] = 0xff800000u;  // -inf
-        }
-        float mx4[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) mx4[i] = -INFINITY;
-#pragma unroll
-        for (int c = 0; c < NCH; ++c)
-#pragma unroll
-          for (int e = 0; e < 16; e += 2)
-            mx4[(e >> 1) & 3] = fmax3(mx4[(e >> 1) & 3], __uint_as_float(sr[c][e]), __uint_as_float(sr[c][e + 1]));
-        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-        // rescale only when the maximum has grown by more than 2^8 (P stays below 256: exact enough in bf16 and f32)
-        const bool grow_m = (j == 0) || ((mx - m_used) * sl2 > 8.f);
-        if (j > 0 && __any_sync(0xffffffffu, grow_m)) {
-          const float alpha = grow_m ? ex2((m_used - mx) * sl2) : 1.f;
-          l *= alpha;
-          // O_h must hold every earlier key tile before it is rescaled: wait for the last P V of key tile n - 1
-          mbar_wait(wc, bars + B_VEMPTY + 8 * ((n - 1) % S_STAGES), ((n - 1) / S_STAGES) & 1);
-          tc_fence_after();
-          const uint32_t tO = tl + S_COL_O + NPV * h + ((HD == 8) ? 8 * (h & 1) : 0);
-#pragma unroll
-          for (int c = 0; c < HD / 8; ++c) {
-            uint32_t o[8];
-            tmem_ld8(tO + 8 * c, o);
-            tmem_wait_ld();
-#pragma unroll
-            for (int e = 0; e < 8; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-            tmem_st8(tO + 8 * c, o);
-          }
-        }
-        if (grow_m) m_used = mx;
-        const float nm = -m_used * sl2;
-        const float2 nmv = make_float2(nm, nm);
-        float2 sum[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-#pragma unroll
-        for (int c = 0; c < NCH; ++c) {
-          uint32_t pr[8];
-#pragma unroll
-          for (int e = 0; e < 16; e += 2) {
-            const float2 x = __ffma2_rn(make_float2(__uint_as_float(sr[c][e]), __uint_as_float(sr[c][e + 1])), sl2v, nmv);
-            const float2 p = make_float2(ex2(x.x), ex2(x.y));
-            sum[(e >> 1) & 1] = __fadd2_rn(sum[(e >> 1) & 1], p);
-            pr[e >> 1] = pack_bf16(p.x, p.y);
-          }
-          tmem_st8(tS + 8 * c, pr);
-        }
-        const float2 s01 = __fadd2_rn(sum[0], sum[1]);
-        l += s01.x + s01.y;
-        asm volatile("st.shared.f32 [%0], %1;" ::"r"(my_state + (2 * h) * 512), "f"(m_used) : "memory");
-        asm volatile("st.shared.f32 [%0], %1;" ::"r"(my_state + (2 * h + 1) * 512), "f"(l) : "memory");
-        tmem_wait_st();
-      };
-
+      // running maximum (the one the weights are taken against) and sum, per head of the slice
+      float m0 = -INFINITY, l0 = 0.f, m1 = -INFINITY, l1 = 0.f;
       const int U = it.T * G;
+      int krem = 0;
+#pragma unroll 1
       for (int u = 0; u < U; ++u) {
         const int j = u / G, h = u - j * G, n = n_kv + j, nu = n_u + u;
-        int krem, yrow;
-        locate(it, j, krem, yrow);
-        mbar_wait(wc, bars + B_SFULL + 8 * (nu & 1), (nu >> 1) & 1);
+        if (h == 0) { int yrow; locate(it, j, krem, yrow); }
+        mbar_wait(wc, bars + B_SFULL, nu & 1);
         tc_fence_after();
         if (krem < SK && h == 0) {
           // Rows of the V tile past the valid length hold whatever follows in memory; a zero weight times NaN or Inf
           // would still poison the accumulator, so clear them (up to the end of the last 16-key group that is
           // multiplied) before the first P V of the tile reads them.
-          const int st = n % S_STAGES;
-          mbar_wait(wc, bars + B_VFULL + 8 * st, (n / S_STAGES) & 1);
+          const int st = n % STAGES;
+          mbar_wait(wc, bars + B_VFULL + 8 * st, (n / STAGES) & 1);
           const int row = krem + r;
           if (row < (((krem + 15) >> 4) << 4)) {
-            const uint32_t a = sV + st * S_KV_BYTES + row * 128;
+            const uint32_t a = sV + st * KVB + row * ROWB;
 #pragma unroll
-            for (int c = 0; c < 8; ++c) st_shared_v4(a + 16 * c, 0, 0, 0, 0);
+            for (int c = 0; c < ROWB / 16; ++c) st_shared_v4(a + 16 * c, 0, 0, 0, 0);
           }
           fence_async_smem();
         }
         if (warp_active) {
-          if (krem >= SK) unit(IntTag<4>{}, BoolTag<false>{}, j, h, n, nu, SK);
-          else if (krem > 48) unit(IntTag<4>{}, BoolTag<true>{}, j, h, n, nu, krem);
-          else if (krem > 32) unit(IntTag<3>{}, BoolTag<true>{}, j, h, n, nu, krem);
-          else if (krem > 16) unit(IntTag<2>{}, BoolTag<true>{}, j, h, n, nu, krem);
-          else unit(IntTag<1>{}, BoolTag<true>{}, j, h, n, nu, krem);
+          // One unit, in four groups of 16 keys; groups without a real key are skipped (the branches are uniform over the
+          // CTA), the group that straddles the valid length is masked element by element.  Two register buffers of 16
+          // scores: a group is requested from TMEM while the one before it is being worked on.
+          float mu = (G == 2 && h == 1) ? m1 : m0, lsum = (G == 2 && h == 1) ? l1 : l0;
+          uint32_t sa[16], sb[16];
+          auto fix = [&](uint32_t (&a)[16], const int c) {  // keys past the valid length get weight exactly zero
+            if (krem < 16 * c + 16) {
+#pragma unroll
+              for (int e = 0; e < 16; ++e)
+                if (16 * c + e >= krem) a[e] = 0xff800000u;  // -inf
+            }
+          };
+          // ---- pass 1: row maximum ----
+          float mx4[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) mx4[i] = -INFINITY;
+          auto maxc = [&](const uint32_t (&a)[16]) {
+#pragma unroll
+            for (int e = 0; e < 16; e += 2)
+              mx4[(e >> 1) & 3] = fmax3(mx4[(e >> 1) & 3], __uint_as_float(a[e]), __uint_as_float(a[e + 1]));
+          };
+          tmem_ld16(tl + 0, sa);
+          if (16 < krem) tmem_ld16(tl + 16, sb);
+          tmem_wait_ld();
+          fix(sa, 0);
+          maxc(sa);
+          if (16 < krem) { fix(sb, 1); maxc(sb); }
+          if (32 < krem) {
+            tmem_ld16(tl + 32, sa);
+            if (48 < krem) tmem_ld16(tl + 48, sb);
+            tmem_wait_ld();
+            fix(sa, 2);
+            maxc(sa);
+            if (48 < krem) { fix(sb, 3); maxc(sb); }
+          }
+          const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+          // rescale only when the maximum has grown by more than 2^8 (P stays below 256: exact enough in bf16 and f32)
+          const bool grow_m = (j == 0) || ((mx - mu) * sl2 > 8.f);
+          if (j > 0 && __any_sync(0xffffffffu, grow_m)) {
+            const float alpha = grow_m ? ex2((mu - mx) * sl2) : 1.f;
+            lsum *= alpha;
+            // O_h must hold every earlier key tile before it is rescaled: wait for the last P V of key tile n - 1
+            mbar_wait(wc, bars + B_VEMPTY + 8 * ((n - 1) % STAGES), ((n - 1) / STAGES) & 1);
+            tc_fence_after();
+            const uint32_t tO = tl + S_COL_O + NPV * h + ((HD == 8) ? 8 * h : 0);
+#pragma unroll
+            for (int c = 0; c < HD / 8; ++c) {
+              uint32_t o[8];
+              tmem_ld8(tO + 8 * c, o);
+              tmem_wait_ld();
+#pragma unroll
+              for (int e = 0; e < 8; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+              tmem_st8(tO + 8 * c, o);
+            }
+          }
+          if (grow_m) mu = mx;
+          // ---- pass 2: weights.  Groups 2 and 3 are still in registers when the tile has them; 0 and 1 are read again. ----
+          const float nm = fmaf(-mu, sl2, TRUNC_LOG2);
+          const float2 nmv = make_float2(nm, nm);
+          float2 sum[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+          auto weights = [&](const uint32_t (&a)[16], const int c) {
+            uint32_t pr[8];
+#pragma unroll
+            for (int e = 0; e < 16; e += 2) {
+              const float2 x = __ffma2_rn(make_float2(__uint_as_float(a[e]), __uint_as_float(a[e + 1])), sl2v, nmv);
+              // a fixed share of the exponentials goes to the FMA pipe, so that it and the special-function unit finish together
+              const float2 p = ((POLY_PAIRS >> (e >> 1)) & 1) ? ex2_poly2(x) : make_float2(ex2(x.x), ex2(x.y));
+              sum[(e >> 1) & 1] = __fadd2_rn(sum[(e >> 1) & 1], p);
+              pr[e >> 1] = __byte_perm(__float_as_uint(p.x), __float_as_uint(p.y), 0x7632);  // upper halves: bf16 pair
+            }
+            tmem_st8(tl + S_COL_P + 8 * c, pr);
+          };
+          if (32 < krem) {
+            weights(sa, 2);
+            tmem_ld16(tl + 0, sa);
+            if (48 < krem) weights(sb, 3);
+            tmem_wait_ld();
+            if (16 < krem) tmem_ld16(tl + 16, sb);
+            fix(sa, 0);  // never masks here (the tile has more than 32 keys); kept for symmetry, compiles to nothing taken
+            weights(sa, 0);
+            tmem_wait_ld();
+            weights(sb, 1);
+          } else {
+            // at most two groups: both are still in registers from pass 1 (masked already)
+            weights(sa, 0);
+            if (16 < krem) weights(sb, 1);
+          }
+          const float2 s01 = __fadd2_rn(sum[0], sum[1]);
+          lsum += s01.x + s01.y;
+          if (G == 2 && h == 1) { m1 = mu; l1 = lsum; } else { m0 = mu; l0 = lsum; }
+          tmem_wait_st();
         }
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(bars + B_PFULL + 8 * (nu & 1));
+        if (lane == 0) mbar_arrive(bars + B_PFULL);
       }
       n_kv += it.T;
       n_u += U;
 
-      // ---- epilogue: O_h / l_h -> bf16, each thread its own 128-byte row of the slice; padded rows +0 ----
+      // ---- epilogue: O_h / l_h -> bf16, each thread its own 32 (64) bytes of the row; padded rows +0 ----
       mbar_wait(wc, bars + B_OFINAL, n_items_done & 1);
       ++n_items_done;
       tc_fence_after();
-      const bool real = r < it.q_real;
       if (warp_active) {
-        uint32_t orow[32];
+        const bool real = r < it.q_real;
+        uint32_t orow[ROWB / 4];
 #pragma unroll
         for (int h = 0; h < G; ++h) {
-          float m_used, l;
-          asm volatile("ld.shared.f32 %0, [%1];" : "=f"(m_used) : "r"(my_state + (2 * h) * 512) : "memory");
-          asm volatile("ld.shared.f32 %0, [%1];" : "=f"(l) : "r"(my_state + (2 * h + 1) * 512) : "memory");
-          const float inv = (l > 0.f) ? 1.f / l : 0.f;
-          const uint32_t tO = tl + S_COL_O + NPV * h + ((HD == 8) ? 8 * (h & 1) : 0);
+          const float lh = (h == 1) ? l1 : l0, mh = (h == 1) ? m1 : m0;
+          const float inv = (lh > 0.f) ? TRUNC_GAIN / lh : 0.f;
+          const uint32_t tO = tl + S_COL_O + NPV * h + ((HD == 8) ? 8 * h : 0);
 #pragma unroll
           for (int c = 0; c < HD / 8; ++c) {
             uint32_t o[8];
@@ -444,19 +514,14 @@ attn_tcs_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           }
           if (lse_row != nullptr && r < it.rows_in_tile) {
             const float ln2 = 0.6931471805599453f;
-            lse_row[(int64_t)h * g.L] = (real && l > 0.f) ? (m_used * sl2 + log2f(l)) * ln2 : -INFINITY;
+            lse_row[(int64_t)h * g.L] = (real && lh > 0.f) ? (mh * sl2 + log2f(lh) - TRUNC_LOG2) * ln2 : -INFINITY;
           }
         }
         if (r < it.rows_in_tile) {
 #pragma unroll
-          for (int c = 0; c < 8; ++c)
+          for (int c = 0; c < ROWB / 16; ++c)
             dst[c] = real ? make_uint4(orow[4 * c], orow[4 * c + 1], orow[4 * c + 2], orow[4 * c + 3]) : make_uint4(0, 0, 0, 0);
         }
-      } else if (r < it.rows_in_tile) {
-#pragma unroll
-        for (int c = 0; c < 8; ++c) dst[c] = make_uint4(0, 0, 0, 0);
-        if (lse_row != nullptr)
-          for (int h = 0; h < G; ++h) lse_row[(int64_t)h * g.L] = -INFINITY;
       }
     }
   }
@@ -474,13 +539,13 @@ constexpr int MAX_DEVICES = 64;
 
 template <int HD>
 cudaError_t launch_tcs(const Geometry& g, const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
-                       int64_t row_stride, __nv_bfloat16* out, float* lse, float scale, cudaStream_t st) {
+                       int64_t row_stride, __nv_bfloat16* out, float* lse, float scale, int* next_item, cudaStream_t st) {
   using C = SCfg<HD>;
   const int64_t rows = matrix_rows(g);
   alignas(64) CUtensorMap tmQ, tmK, tmV;
   const bool okq = (HD == 8) ? make_map(&tmQ, q, rows, g.d, row_stride, 8, SQ, true)
-                             : make_map(&tmQ, q, rows, g.d, row_stride, SLICE, SQ);
-  if (!okq || !make_map(&tmK, k, rows, g.d, row_stride, SLICE, SK) || !make_map(&tmV, v, rows, g.d, row_stride, SLICE, SK))
+                             : make_map(&tmQ, q, rows, g.d, row_stride, C::SLW, SQ);
+  if (!okq || !make_map(&tmK, k, rows, g.d, row_stride, C::SLW, SK) || !make_map(&tmV, v, rows, g.d, row_stride, C::SLW, SK))
     return cudaErrorInvalidValue;
   static int n_sm[MAX_DEVICES] = {};  // per device: SM count, and whether the kernel's shared-memory size has been set
   int dev = 0;
@@ -497,9 +562,9 @@ cudaError_t launch_tcs(const Geometry& g, const __nv_bfloat16* q, const __nv_bfl
   }
   int tiles = 0;
   for (int s = 0; s < 3; ++s) tiles += (g.seg_len[s] + SQ - 1) / SQ;
-  const int slices = g.d / SLICE;
+  const int slices = g.d / C::SLW;
   const int64_t n_items = (int64_t)tiles * slices * g.batch;
-  if (n_items > 0x7fffffffLL) return cudaErrorNotSupported;
+  if (n_items > 0x3fffffffLL) return cudaErrorNotSupported;
   // query segments in descending order of the keys their tiles walk (longest work first)
   int cost[3], ord[3] = {0, 1, 2};
   for (int s = 0; s < 3; ++s) {
@@ -511,22 +576,30 @@ cudaError_t launch_tcs(const Geometry& g, const __nv_bfloat16* q, const __nv_bfl
     for (int j = i + 1; j < 3; ++j)
       if (cost[ord[j]] > cost[ord[i]]) { const int t = ord[i]; ord[i] = ord[j]; ord[j] = t; }
   const int seg_order = ord[0] | (ord[1] << 2) | (ord[2] << 4);
-  const unsigned grid = (unsigned)((n_items < 2 * n_sm[dev]) ? n_items : 2 * n_sm[dev]);  // two resident CTAs per SM
+  const int64_t resident = (int64_t)S_CTAS_PER_SM * n_sm[dev];
+  const unsigned grid = (unsigned)((n_items < resident) ? n_items : resident);
+  if (next_item != nullptr) {
+    e = cudaMemsetAsync(next_item, 0, sizeof(int), st);
+    if (e != cudaSuccess) return e;
+  }
   attn_tcs_kernel<HD><<<grid, S_THREADS, C::SMEM, st>>>(tmQ, tmK, tmV, g, out, lse, scale * 1.4426950408889634f, slices,
-                                                         seg_order, (int)n_items);
+                                                         seg_order, (int)n_items, next_item);
   return cudaGetLastError();
 }
 
 }  // namespace
 
-bool attn_tcs_supported(const Geometry& g) { return g.d % SLICE == 0 && (g.hd == 8 || g.hd == 16 || g.hd == 32); }
+bool attn_tcs_supported(const Geometry& g) {
+  return (g.hd == 8 || g.hd == 16) ? (g.d % 16 == 0) : (g.hd == 32 && g.d % 32 == 0);
+}
 
 cudaError_t launch_attn_tcs(const Geometry& g, const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
-                            int64_t row_stride, __nv_bfloat16* out, float* lse, float scale, cudaStream_t st) {
+                            int64_t row_stride, __nv_bfloat16* out, float* lse, float scale, int* next_item,
+                            cudaStream_t st) {
   if (!attn_tcs_supported(g)) return cudaErrorNotSupported;
-  if (g.hd == 8) return launch_tcs<8>(g, q, k, v, row_stride, out, lse, scale, st);
-  if (g.hd == 16) return launch_tcs<16>(g, q, k, v, row_stride, out, lse, scale, st);
-  return launch_tcs<32>(g, q, k, v, row_stride, out, lse, scale, st);
+  if (g.hd == 8) return launch_tcs<8>(g, q, k, v, row_stride, out, lse, scale, next_item, st);
+  if (g.hd == 16) return launch_tcs<16>(g, q, k, v, row_stride, out, lse, scale, next_item, st);
+  return launch_tcs<32>(g, q, k, v, row_stride, out, lse, scale, next_item, st);
 }
 
 }  // namespace gsit

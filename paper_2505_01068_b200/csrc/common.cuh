@@ -5,6 +5,7 @@
 #include <stdint.h>
 
 #include "gsit.h"
+#include "gsit_test.h"
 
 namespace gsit {
 
@@ -71,17 +72,19 @@ cudaError_t launch_attn_f32(const Geometry& g, const float* q, const float* k, c
 // bf16 attention, mma.sync tiles fed by TMA (attn_bf16.cu); returns cudaErrorNotSupported for shapes it lacks
 cudaError_t launch_attn_bf16(const Geometry& g, const __nv_bfloat16* q, const __nv_bfloat16* k,
                              const __nv_bfloat16* v, int64_t row_stride, __nv_bfloat16* out, float* lse,
-                             float scale, cudaStream_t st);
+                             float scale, int* next_item, cudaStream_t st);
 
 // bf16 attention for head_dim 64 on tcgen05 tensor cores with TMEM accumulators (attn_tc.cu)
 cudaError_t launch_attn_tc_hd64(const Geometry& g, const __nv_bfloat16* q, const __nv_bfloat16* k,
                                 const __nv_bfloat16* v, int64_t row_stride, __nv_bfloat16* out, float* lse,
                                 float scale, cudaStream_t st);
 
-// bf16 attention for head_dim 8 / 16 / 32 and d_model a multiple of 64 on tcgen05 with thread-per-row softmax (attn_tcs.cu)
+// bf16 attention for head_dim 8 / 16 / 32 on tcgen05 with thread-per-row softmax (attn_tcs.cu).  next_item: a device int
+// the call may use as its work counter (it is cleared on the stream before the launch), or nullptr for a fixed
+// assignment of work items to CTAs.
 bool attn_tcs_supported(const Geometry& g);
 cudaError_t launch_attn_tcs(const Geometry& g, const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
-                            int64_t row_stride, __nv_bfloat16* out, float* lse, float scale, cudaStream_t st);
+                            int64_t row_stride, __nv_bfloat16* out, float* lse, float scale, int* next_item, cudaStream_t st);
 
 // Linear layers  C = act(A W^T + bias) (+ residual), rows that are padding written as zero when
 // `mask_rows` is set.  A [M,K] (lda), W [N,K], C [M,N] (ldc), residual float [M,N] (ldr) or nullptr.

@@ -2,6 +2,7 @@
 #include <math.h>
 
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace gsit {
 
@@ -96,9 +97,11 @@ gsit_status from_cuda(cudaError_t e) {
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+constexpr size_t ATTENTION_SCRATCH = 256;  // bytes gsit_im_attention_fwd can use (one work counter)
+
 // Scratch layout of one layer call; every region 256-byte aligned.
 struct LayerScratch {
-  size_t h, qkv, att, y1, f, total;
+  size_t h, qkv, att, y1, f, sched, total;
 };
 LayerScratch layer_scratch(const Geometry& g, int dtype, int d_ff) {
   // packed layout: every call addresses the packed matrices by absolute row, whatever part of the batch it covers
@@ -110,6 +113,7 @@ LayerScratch layer_scratch(const Geometry& g, int dtype, int d_ff) {
   s.att = off; off += align_up(rows * g.d * es, 256);
   s.y1 = off;  off += align_up(rows * g.d * 4, 256);        // float residual stream after attention
   s.f = off;   off += align_up(rows * (size_t)d_ff * es, 256);
+  s.sched = off; off += ATTENTION_SCRATCH;                   // work counter of the attention kernel
   s.total = off;
   return s;
 }
@@ -152,14 +156,30 @@ gsit_status run_layernorm(const Geometry& g, const float* x, int64_t ldx, const 
 }
 
 gsit_status run_attention(const Geometry& g, int dtype, const void* q, const void* k, const void* v,
-                          int64_t row_stride, void* out, float* lse, float scale, cudaStream_t st) {
+                          int64_t row_stride, void* out, float* lse, float scale, void* scratch, cudaStream_t st) {
   TraceScope t(GSIT_KERNEL_ATTENTION, st);
   if (dtype == GSIT_BF16)
     return from_cuda(launch_attn_bf16(g, static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k),
                                       static_cast<const __nv_bfloat16*>(v), row_stride,
-                                      static_cast<__nv_bfloat16*>(out), lse, scale, st));
+                                      static_cast<__nv_bfloat16*>(out), lse, scale, static_cast<int*>(scratch), st));
   return from_cuda(launch_attn_f32(g, static_cast<const float*>(q), static_cast<const float*>(k),
                                    static_cast<const float*>(v), row_stride, static_cast<float*>(out), lse, scale, st));
+}
+
+// A bounded wait that must run out: the barrier expects one arrival and nobody arrives.
+__global__ void expire_wait_kernel(unsigned int* status) {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ uint32_t gave_up;
+  const uint32_t b = smem_u32(&bar);
+  if (threadIdx.x == 0) {
+    gave_up = 0;
+    ptx::mbar_init(b, 1);
+    ptx::mbar_init_fence();
+  }
+  __syncthreads();
+  const ptx::WaitCtx wc{status, smem_u32(&gave_up)};
+  if (threadIdx.x == 0) ptx::mbar_wait(wc, b, 0, 1 << 12);
+  __syncthreads();
 }
 
 float pick_scale(const gsit_shape* s, const Geometry& g) {
@@ -194,7 +214,6 @@ gsit_status gsit_im_qkv_proj(const gsit_shape* shape, const void* x, int64_t x_r
 gsit_status gsit_im_attention_fwd(const gsit_shape* shape, const void* q, const void* k, const void* v,
                                   int64_t row_stride, void* out, float* lse, void* workspace,
                                   size_t workspace_bytes, gsit_stream stream) {
-  (void)workspace; (void)workspace_bytes;  // this call needs no scratch
   Geometry g;
   gsit_status st = make_geometry(shape, &g);
   if (st != GSIT_OK) return st;
@@ -203,7 +222,10 @@ gsit_status gsit_im_attention_fwd(const gsit_shape* shape, const void* q, const 
   if (shape->dtype == GSIT_BF16 && row_stride % 8 != 0) return GSIT_ERR_INVALID_ARG;
   if (g.row_start != nullptr && (shape->dtype != GSIT_BF16 || g.hd > 32)) return GSIT_ERR_UNSUPPORTED;
   if (from_cuda(status_ptr(&g.status)) != GSIT_OK) return GSIT_ERR_CUDA;
-  return run_attention(g, shape->dtype, q, k, v, row_stride, out, lse, pick_scale(shape, g),
+  // optional scratch: with it the bf16 kernels hand out their work items through a counter instead of a fixed assignment
+  void* scratch = (workspace != nullptr && workspace_bytes >= sizeof(int) && (reinterpret_cast<uintptr_t>(workspace) & 3u) == 0)
+                      ? workspace : nullptr;
+  return run_attention(g, shape->dtype, q, k, v, row_stride, out, lse, pick_scale(shape, g), scratch,
                        static_cast<cudaStream_t>(stream));
 }
 
@@ -237,11 +259,11 @@ gsit_status gsit_im_layer_fwd(const gsit_shape* shape, const gsit_layer_weights*
       !(bf && g.hd <= 32 && (fused_layer_tc_supported(g, w->d_ff) || fused_layer_tc128_supported(g, w->d_ff))))
     return GSIT_ERR_UNSUPPORTED;  // the packed layout is implemented by the tcgen05 fused halves and the mma.sync attention
 
-  if (bf && fused_layer_supported(g, w->d_ff) && (g_attn_variant != 8 || g.row_start != nullptr)) {
+  if (bf && fused_layer_supported(g, w->d_ff) && (g_attn_variant != GSIT_ATTN_UNFUSED || g.row_start != nullptr)) {
     // three launches: LN1 + shared projection, IM attention, out-projection + residual + LN2 + MLP + residual
-    // d_model 64 and 128 run both halves on tcgen05 (tuning knob 9 keeps the mma.sync kernels)
-    const bool tc = fused_layer_tc_supported(g, w->d_ff) && (g_attn_variant != 9 || g.row_start != nullptr);
-    const bool tc128 = fused_layer_tc128_supported(g, w->d_ff) && (g_attn_variant != 9 || g.row_start != nullptr);
+    // d_model 64 and 128 run both halves on tcgen05 (GSIT_ATTN_LEGACY keeps the mma.sync kernels)
+    const bool tc = fused_layer_tc_supported(g, w->d_ff) && (g_attn_variant != GSIT_ATTN_LEGACY || g.row_start != nullptr);
+    const bool tc128 = fused_layer_tc128_supported(g, w->d_ff) && (g_attn_variant != GSIT_ATTN_LEGACY || g.row_start != nullptr);
     {
       TraceScope t(GSIT_KERNEL_LINEAR, cs);
       st = from_cuda(tc ? launch_ln_qkv_tc(g, x, x_row_stride, w->ln1_gamma, w->ln1_beta, eps,
@@ -257,7 +279,7 @@ gsit_status gsit_im_layer_fwd(const gsit_shape* shape, const gsit_layer_weights*
     if (st != GSIT_OK) return st;
     const uint8_t* qb = static_cast<const uint8_t*>(qkv);
     if ((st = run_attention(g, dtype, qb, qb + (size_t)d * es, qb + (size_t)2 * d * es, 3 * (int64_t)d, att, nullptr,
-                            pick_scale(shape, g), cs)) != GSIT_OK) return st;
+                            pick_scale(shape, g), ws + sc.sched, cs)) != GSIT_OK) return st;
     TraceScope t(GSIT_KERNEL_LINEAR, cs);
     if (tc)
       return from_cuda(launch_proj_mlp_tc(g, static_cast<const __nv_bfloat16*>(att), x, x_row_stride,
@@ -284,7 +306,7 @@ gsit_status gsit_im_layer_fwd(const gsit_shape* shape, const gsit_layer_weights*
   // att = IM attention over the open blocks
   const uint8_t* qb = static_cast<const uint8_t*>(qkv);
   if ((st = run_attention(g, dtype, qb, qb + (size_t)d * es, qb + (size_t)2 * d * es, 3 * (int64_t)d, att, nullptr,
-                          pick_scale(shape, g), cs)) != GSIT_OK) return st;
+                          pick_scale(shape, g), ws + sc.sched, cs)) != GSIT_OK) return st;
   // y1 = x + att W_o^T + b_o   (float)
   a = LinearArgs{};
   a.A = att; a.lda = d; a.W = w->w_o; a.bias = w->b_o; a.residual = x; a.ldr = x_row_stride;
@@ -363,7 +385,8 @@ size_t gsit_workspace_bytes(const gsit_shape* shape, int which_call, int32_t d_f
     if (d_ff < 1) return (size_t)-1;
     return layer_scratch(g, shape->dtype, d_ff).total;
   }
-  if (which_call == GSIT_CALL_QKV_PROJ || which_call == GSIT_CALL_ATTENTION) return 0;
+  if (which_call == GSIT_CALL_ATTENTION) return (shape->dtype == GSIT_BF16) ? ATTENTION_SCRATCH : 0;
+  if (which_call == GSIT_CALL_QKV_PROJ) return 0;
   return (size_t)-1;
 }
 
@@ -429,6 +452,13 @@ const char* gsit_status_string(gsit_status s) {
     case GSIT_ERR_TIMEOUT: return "device-side wait timed out";
     default: return "unknown status";
   }
+}
+
+gsit_status gsit_test_expire_wait(gsit_stream stream) {
+  unsigned int* p = nullptr;
+  if (status_ptr(&p) != cudaSuccess) return GSIT_ERR_CUDA;
+  expire_wait_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(p);
+  return from_cuda(cudaGetLastError());
 }
 
 gsit_status gsit_tune_attention(int variant) {

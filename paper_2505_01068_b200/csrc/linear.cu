@@ -211,10 +211,10 @@ cudaError_t launch_linear_f32(const Geometry& g, const LinearArgs& a, cudaStream
   return cudaGetLastError();
 }
 
-extern int g_attn_variant;  // tuning knob (attn_bf16.cu): 9 keeps every bf16 kernel on the mma.sync path
+extern int g_attn_variant;  // kernel selection (attn_bf16.cu): GSIT_ATTN_LEGACY keeps every bf16 kernel on the mma.sync path
 
 cudaError_t launch_linear_bf16(const Geometry& g, const LinearArgs& a, cudaStream_t st) {
-  if (g_attn_variant != 9 && linear_tc_supported(a)) return launch_linear_tc_bf16(g, a, st);
+  if (g_attn_variant != GSIT_ATTN_LEGACY && linear_tc_supported(a)) return launch_linear_tc_bf16(g, a, st);
   if (a.K % 8 != 0 || a.N % 2 != 0 || a.lda % 8 != 0) return cudaErrorNotSupported;
   const bool wide = (a.N % 128 == 0) || a.N > 256;
   const int bn = wide ? 128 : 64;

@@ -33,6 +33,17 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
+// One poll that lets the hardware park the thread for up to `ns` nanoseconds (it wakes as soon as the phase completes):
+// for roles that wait long, so that their polling does not take issue slots from the warps that compute.
+__device__ __forceinline__ bool mbar_try_park(uint32_t bar, uint32_t parity, uint32_t ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity), "r"(ns) : "memory");
+  return ok != 0;
+}
 // One poll that never parks the thread.
 __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -64,6 +75,43 @@ __device__ __forceinline__ bool mbar_wait(const WaitCtx& w, uint32_t bar, uint32
   for (int it = 0; it < limit; ++it) {
     if (mbar_try(bar, parity)) return true;
     if ((it & 63) == 63 && cta_gave_up(w)) return false;
+  }
+  asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(w.gave_up), "r"(1u) : "memory");
+  atomicOr(w.status, GSIT_DEVFLAG_TIMEOUT);
+  return false;
+}
+
+// The same with parked polls of up to ten microseconds each (2^15 of them at most: a third of a second).
+__device__ __forceinline__ bool mbar_wait_parked(const WaitCtx& w, uint32_t bar, uint32_t parity, int limit = 1 << 15) {
+  for (int it = 0; it < limit; ++it) {
+    if (mbar_try_park(bar, parity, 10000u)) return true;
+    if ((it & 15) == 15 && cta_gave_up(w)) return false;
+  }
+  asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(w.gave_up), "r"(1u) : "memory");
+  atomicOr(w.status, GSIT_DEVFLAG_TIMEOUT);
+  return false;
+}
+
+// Bounded wait that sleeps between polls.  A try_wait that fails comes back within tens of clocks, so a warp that waits
+// by polling alone keeps issuing instructions; with several waiting warps per scheduler that takes most of the issue
+// slots from the warps that compute.  Here a poll never parks (test_wait) and is followed by a sleep of about `ns`
+// nanoseconds during which the warp issues nothing.  Gives up after `limit` polls like mbar_wait.
+__device__ __forceinline__ bool mbar_wait_sleep(const WaitCtx& w, uint32_t bar, uint32_t parity, unsigned ns, int limit = 1 << 17) {
+  for (int it = 0; it < limit; ++it) {
+    if (mbar_test(bar, parity)) return true;
+    __nanosleep(ns);
+    if ((it & 63) == 63 && cta_gave_up(w)) return false;
+  }
+  asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(w.gave_up), "r"(1u) : "memory");
+  atomicOr(w.status, GSIT_DEVFLAG_TIMEOUT);
+  return false;
+}
+
+// Bounded wait that spins on non-parking polls: the shortest hand-over latency, at the price of issue slots.
+__device__ __forceinline__ bool mbar_wait_spin(const WaitCtx& w, uint32_t bar, uint32_t parity, int limit = 1 << 22) {
+  for (int it = 0; it < limit; ++it) {
+    if (mbar_test(bar, parity)) return true;
+    if ((it & 1023) == 1023 && cta_gave_up(w)) return false;
   }
   asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(w.gave_up), "r"(1u) : "memory");
   atomicOr(w.status, GSIT_DEVFLAG_TIMEOUT);
@@ -143,6 +191,22 @@ __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+// 2^x for a pair of arguments on the FMA and integer pipes instead of the special-function unit: x = n + f with n the
+// nearest integer (taken from the low mantissa bits of x + 1.5 * 2^23) and |f| <= 1/2, 2^f by a cubic with relative
+// error 7.6e-5 (well below the 2^-9 of the bf16 rounding that follows), n added into the exponent field.  Arguments
+// are clamped at -126 (the result then flushes towards 2^-126 instead of wrapping); valid up to x < 128.
+__device__ __forceinline__ float2 ex2_poly2(float2 x) {
+  x.x = fmaxf(x.x, -126.f);
+  x.y = fmaxf(x.y, -126.f);
+  const float2 t = __fadd2_rn(x, make_float2(12582912.f, 12582912.f));
+  const float2 n = __fadd2_rn(t, make_float2(-12582912.f, -12582912.f));
+  const float2 f = __ffma2_rn(n, make_float2(-1.f, -1.f), x);
+  float2 p = __ffma2_rn(make_float2(0.055205505f, 0.055205505f), f, make_float2(0.24261397f, 0.24261397f));
+  p = __ffma2_rn(p, f, make_float2(0.69325477f, 0.69325477f));
+  p = __ffma2_rn(p, f, make_float2(0.9999277f, 0.9999277f));
+  return make_float2(__int_as_float(__float_as_int(p.x) + (__float_as_int(t.x) << 23)),
+                     __int_as_float(__float_as_int(p.y) + (__float_as_int(t.y) << 23)));
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t r;

@@ -1,4 +1,4 @@
-"""The C-ABI library builds, loads without a GPU, and exports every function include/gsit.h declares."""
+"""The C-ABI library builds, loads without a GPU, and exports every function the headers under include/ declare."""
 import ctypes
 import re
 from pathlib import Path
@@ -7,9 +7,11 @@ ROOT = Path(__file__).resolve().parent.parent
 
 
 def _declared():
-    text = (ROOT / "include" / "gsit.h").read_text()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(gsit_[a-z_0-9]+)\s*\(", text)))
+    names = set()
+    for header in sorted((ROOT / "include").glob("*.h")):
+        text = re.sub(r"/\*.*?\*/", "", header.read_text(), flags=re.S)
+        names |= set(re.findall(r"\b(gsit_[a-z_0-9]+)\s*\(", text))
+    return sorted(names)
 
 
 def test_library_exports_every_declared_symbol():
@@ -39,6 +41,8 @@ def test_workspace_query_needs_no_gpu():
 
     sh = g.make_shape(2, (8, 12, 10), 32, 4, None, g.DTYPE_F32, g.PHASE_INTRA)
     assert g.workspace_bytes(sh, g.CALL_ATTENTION) == 0
+    sh16 = g.make_shape(2, (8, 12, 10), 32, 4, None, g.DTYPE_BF16, g.PHASE_INTRA)
+    assert 0 < g.workspace_bytes(sh16, g.CALL_ATTENTION) <= 4096
     rows = 2 * 30
     assert g.workspace_bytes(sh, g.CALL_LAYER, 128) >= rows * (32 * 4 * 3 + 96 * 4 + 128 * 4)
     bad = g.make_shape(2, (8, 12, 10), 30, 4, None, g.DTYPE_F32, g.PHASE_INTRA)

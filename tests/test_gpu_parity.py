@@ -197,7 +197,7 @@ def test_layer_bf16_affine_biases_ragged(g, d, heads, d_ff, seg, B):
 
 
 def test_qkv_proj_tcgen05_matches_mma_sync_kernel(g):
-    """The shared projection through the tcgen05 GEMM and through the mma.sync kernel (tuning knob 9) on the same inputs:
+    """The shared projection through the tcgen05 GEMM and through the mma.sync kernel (kernel choice ATTN_LEGACY) on the same inputs:
     both within the bf16 tolerance of the oracle, and within rounding of each other."""
     rng = np.random.default_rng(31)
     seg, B, d, H = (37, 300, 129), 3, 256, 4
@@ -208,7 +208,7 @@ def test_qkv_proj_tcgen05_matches_mma_sync_kernel(g):
     xd = to_dev(wk.fill_padding(x, seg, valid, np.nan), "bf16")
     wd, bd = to_dev(w["w_qkv"], "bf16"), to_dev(w["b_qkv"])
     new = to_np64(g.im_qkv_proj(xd, wd, bd, seg, H, vl)).reshape(B, sum(seg), -1)
-    g.tune_attention(9)
+    g.tune_attention(g.ATTN_LEGACY)
     try:
         old = to_np64(g.im_qkv_proj(xd, wd, bd, seg, H, vl)).reshape(B, sum(seg), -1)
     finally:
@@ -224,7 +224,7 @@ def test_qkv_proj_tcgen05_matches_mma_sync_kernel(g):
 
 @pytest.mark.parametrize("d,heads,d_ff", [(64, 8, 256), (128, 8, 512)])
 def test_fused_layer_tcgen05_matches_mma_sync_fused_kernels(g, d, heads, d_ff):
-    """The tcgen05 fused halves and the mma.sync fused halves (tuning knob 9) compute the same layer."""
+    """The tcgen05 fused halves and the mma.sync fused halves (kernel choice ATTN_LEGACY) compute the same layer."""
     rng = np.random.default_rng(d)
     seg, B = (50, 333, 190), 2
     x = rng.standard_normal((B, sum(seg), d), dtype=np.float32)
@@ -233,7 +233,7 @@ def test_fused_layer_tcgen05_matches_mma_sync_fused_kernels(g, d, heads, d_ff):
     vl = torch.from_numpy(valid).cuda()
     xd = to_dev(wk.fill_padding(x, seg, valid, np.nan))
     new = to_np64(g.im_layer_fwd(xd, w, seg, heads, vl, oracle.PHASE_INTER_BWD))
-    g.tune_attention(9)
+    g.tune_attention(g.ATTN_LEGACY)
     try:
         old = to_np64(g.im_layer_fwd(xd, w, seg, heads, vl, oracle.PHASE_INTER_BWD))
     finally:

@@ -50,7 +50,9 @@ def test_static_scratch_layer_matches_workspace_layer_bit_for_bit(g):
     x, w, vl = _case(g, "f32", 1, (4, 4, 4), 32, 4, None, 1)
     g.im_layer_fwd_static(x, w, (4, 4, 4), 4, None, g.PHASE_INTRA)
     torch.cuda.synchronize()
+    got = want = out = None
     for call, (dtype, B, seg, d, heads, valid, phase) in enumerate(cases):
+        del got, want, out  # the previous round's tensors go now, not in the middle of the measurement below
         x, w, vl = _case(g, dtype, B, seg, d, heads, valid, 900 + call)
         want = g.im_layer_fwd(x, w, seg, heads, vl, phase)
         out = torch.full_like(want, float("nan"))
