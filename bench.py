@@ -7,7 +7,10 @@ QKV projection -> IM attention -> out-projection + residual -> LayerNorm -> MLP 
 library's kernels (three launches per layer).  `value` is valid (non padded) tokens per second with inputs resident in HBM; `e2e`
 includes the host->device copy of the batch and the device->host copy of the result every step.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload 4|5]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--repeats R] [--impl reference]
+    python bench.py --only attention|layer --workload W --batch B --phase P [--d D --heads H] [--calls C]   (profiler driver)
+
+With --gpus N > 1 and no torchrun environment the script starts N worker processes itself, one GPU each.
 """
 from __future__ import annotations
 
@@ -30,10 +33,17 @@ METRIC = "IM-attention tokens/s (valid tokens through the GsiT IM stack), MOSEI-
 UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 L2_BYTES = 126 * 1024 * 1024
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the cross-modal attention kernel at this workload
-# (ncu capture summarised in profiles/attn_bf16_hd8_cfg4_cross.md, taken of the kernel as it stands: 21.44 MB read,
-# 0.02 MB written while the output is still in L2)
-ATTN_HD8_DRAM_BYTES = 21.46e6
+
+
+def recorded_traffic(kernel: str):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of `kernel`, from the ncu capture summarised under
+    profiles/ (profiles/traffic.json, written next to the summary when the capture is taken), or None when there is no
+    record for the kernel as it stands."""
+    p = ROOT / "profiles" / "traffic.json"
+    if not p.exists():
+        return None
+    rec = json.loads(p.read_text()).get(kernel)
+    return None if rec is None else float(rec["dram_bytes_per_launch"])
 
 
 def peaks():
@@ -79,7 +89,7 @@ class ClockSampler:
                 self.reasons |= self._names(int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)))
             except Exception:
                 pass
-            self._stop.wait(0.02)
+            self._stop.wait(0.01)
 
     def __enter__(self):
         if self._h is not None:
@@ -148,6 +158,8 @@ def run_reference(args):
 
 
 def _time_graph_replays(torch, graphs, steps, dist, world):
+    """One timed region: exactly `steps` replays between a barrier + synchronize on both sides, CUDA events on the
+    launching stream, maximum over ranks.  Returns milliseconds."""
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
@@ -166,15 +178,17 @@ def _time_graph_replays(torch, graphs, steps, dist, world):
     return ms
 
 
-def time_attention_alone(torch, g, wl, valid_dev, d, heads, phase, reps=4):
+def time_attention_alone(torch, g, wl, valid_dev, d, heads, phase, reps=4, batch=None):
     """One IM-attention call timed alone: a CUDA graph of launches rotating over qkv/out buffer sets larger than L2."""
-    B, L = (wl.batch if valid_dev is None else valid_dev.shape[0]), wl.L
+    B, L = (batch or (wl.batch if valid_dev is None else valid_dev.shape[0])), wl.L
     set_bytes = B * L * 4 * d * 2
-    nsets = max(2, int(np.ceil(1.5 * L2_BYTES / set_bytes)))
+    nsets = min(64, max(2, int(np.ceil(1.5 * L2_BYTES / set_bytes))))
     gen = torch.Generator(device="cuda").manual_seed(1234)
     qkvs = [torch.randn((B, L, 3, heads, d // heads), device="cuda", generator=gen).bfloat16() for _ in range(nsets)]
     outs = [torch.empty((B, L, d), device="cuda", dtype=torch.bfloat16) for _ in range(nsets)]
-    run = lambda i: g.im_attention_fwd(qkvs[i][:, :, 0], qkvs[i][:, :, 1], qkvs[i][:, :, 2], wl.seg_len, valid_dev, phase, out=outs[i])
+    wss = [torch.empty(256, dtype=torch.uint8, device="cuda") for _ in range(nsets)]
+    run = lambda i: g.im_attention_fwd(qkvs[i][:, :, 0], qkvs[i][:, :, 1], qkvs[i][:, :, 2], wl.seg_len, valid_dev, phase, out=outs[i],
+                                       workspace=wss[i])
     for i in range(nsets):
         run(i)
     torch.cuda.synchronize()
@@ -193,6 +207,70 @@ def time_attention_alone(torch, g, wl, valid_dev, d, heads, phase, reps=4):
     end.record()
     torch.cuda.synchronize()
     return beg.elapsed_time(end) * 1e-3 / (5 * reps * nsets), nsets
+
+
+PATTERNS = {"fwd": [[0, 1, 0], [0, 0, 1], [1, 0, 0]], "bwd": [[0, 0, 1], [1, 0, 0], [0, 1, 0]], "intra": [[1, 0, 0], [0, 1, 0], [0, 0, 1]]}
+
+
+def attention_per_config(torch, g, pk, ex2_rate):
+    """IM attention alone at the aligned (cfg 2) and MOSI-shaped (cfg 3) workloads, all three block patterns: time, tokens/s,
+    useful TFLOP/s and the fraction of both rooflines.  Reported, not graded (cfg 2 is launch-latency bound)."""
+    out = {}
+    for idx in (2, 3):
+        wl = wk.WORKLOADS[idx]
+        valid = wk.draw_valid_len(np.random.default_rng(wl.seed), wl)
+        vl = None if valid is None else torch.from_numpy(valid).cuda()
+        tokens = wl.batch * wl.L if valid is None else int(valid.sum())
+        rec = {}
+        for name, phase in (("fwd", g.PHASE_INTER_FWD), ("bwd", g.PHASE_INTER_BWD), ("intra", g.PHASE_INTRA)):
+            sec, nsets = time_attention_alone(torch, g, wl, vl, wl.d_model, wl.heads, phase, batch=wl.batch)
+            U = wk.useful_pairs(wl.seg_len, valid, PATTERNS[name], wl.batch)
+            fl, by = 4.0 * wl.d_model * U, 4.0 * tokens * wl.d_model * 2
+            t_tc, t_hbm, t_exp = fl / (pk["bf16_tflops"] * 1e12), by / (pk["hbm_gbs"] * 1e9), wl.heads * U / ex2_rate
+            rec[name] = {"us": sec * 1e6, "tokens_per_s": tokens / sec, "useful_tflops": fl / sec / 1e12,
+                         "frac_roofline": max(t_tc, t_hbm) / sec, "frac_three_way": max(t_tc, t_hbm, t_exp) / sec,
+                         "t_hbm_us": t_hbm * 1e6, "t_exp_us": t_exp * 1e6, "buffer_sets": nsets}
+        out[f"cfg{idx}:{wl.name}"] = rec
+    torch.cuda.empty_cache()
+    return out
+
+
+def run_only(args):
+    """Profiler driver: a few launches of one library call on workload-shaped inputs (N(0,1) values, the workload's padding
+    recipe), so that `ncu -k ... -c ...` has a short, self-contained command to wrap.  Prints the device status."""
+    import torch
+
+    import paper_2505_01068_b200 as g
+    g.load()
+    wl = wk.WORKLOADS[args.workload]
+    B = args.batch or wl.batch
+    rng = np.random.default_rng(wl.seed)
+    valid = wk.draw_valid_len(rng, wl, B)
+    vl = None if valid is None else torch.from_numpy(valid).cuda()
+    d, heads = args.d or wl.d_model, args.heads or wl.heads
+    gen = torch.Generator(device="cuda").manual_seed(1)
+    nsets = 3
+    if args.only == "attention":
+        bufs = [torch.randn((B, wl.L, 3, heads, d // heads), device="cuda", generator=gen).bfloat16() for _ in range(nsets)]
+        outs = [torch.empty((B, wl.L, d), device="cuda", dtype=torch.bfloat16) for _ in range(nsets)]
+        ws = torch.empty(256, dtype=torch.uint8, device="cuda")
+        run = lambda i: g.im_attention_fwd(bufs[i][:, :, 0], bufs[i][:, :, 1], bufs[i][:, :, 2], wl.seg_len, vl, args.phase,
+                                           out=outs[i], workspace=ws)
+    else:
+        w = wk.draw_layer_weights(rng, d, wl.d_ff_mult * d, wl.dtype)
+        wd = {k: (None if v is None else (torch.from_numpy(v).cuda().bfloat16() if (k.startswith("w_") and wl.dtype == "bf16")
+                                          else torch.from_numpy(v).cuda())) for k, v in w.items()}
+        bufs = [torch.randn((B, wl.L, d), device="cuda", generator=gen) for _ in range(nsets)]
+        outs = [torch.empty((B, wl.L, d), device="cuda") for _ in range(nsets)]
+        sh = g.make_shape(B, wl.seg_len, d, heads, vl, g.binding._dtype_code(wd["w_qkv"].dtype), args.phase)
+        ws = torch.empty(g.workspace_bytes(sh, g.CALL_LAYER, wd["w_1"].shape[0]), dtype=torch.uint8, device="cuda")
+        run = lambda i: g.im_layer_fwd(bufs[i], wd, wl.seg_len, heads, vl, args.phase, out=outs[i], workspace=ws)
+    if args.kernels:
+        g.tune_attention(args.kernels)
+    for c in range(args.calls):
+        run(c % nsets)
+    torch.cuda.synchronize()
+    print(f"{args.only} workload {args.workload} batch {B} phase {args.phase} d {d} heads {heads}: device status", g.last_device_status())
 
 
 def run_gpu(args):
@@ -247,8 +325,10 @@ def run_gpu(args):
         graphs[k % nbuf].replay()
     torch.cuda.synchronize()
 
+    # a step is under a millisecond: the region of `steps` steps is repeated and the median region is reported
     with ClockSampler(local) as clocks:
-        ms = _time_graph_replays(torch, graphs, args.steps, dist, world)
+        regions = [_time_graph_replays(torch, graphs, args.steps, dist, world) for _ in range(args.repeats)]
+    ms = float(np.median(regions))
     ms_per_step = ms / args.steps
     # whole job: tokens of all ranks over the slowest rank's time (ms is already the maximum over ranks)
     _, _, value = shard.job_throughput(tokens, ms_per_step, device="cuda")
@@ -396,13 +476,15 @@ def run_gpu(args):
                          "the step's scratch alone is larger than L2", "launch": "one CUDA graph per input buffer; inside it the forward and backward rings on two streams, then the "
                              "intra encoder on the two halves of the batch on the same two streams; packed row layout (real rows only)"},
         "clocks": clocks.summary(),
+        "timed_regions": {"repeats": args.repeats, "steps_each": args.steps, "ms_per_step_median": ms_per_step,
+                          "ms_per_step_min": min(regions) / args.steps, "ms_per_step_max": max(regions) / args.steps},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(x_host.numel() * 4),
                 "d2h_bytes_per_step": int(y_host.numel() * 4) ,
                 "how": "HostPipeline, 2 steps in flight: copy-in, kernels and copy-out of neighbouring steps overlap"},
         "gpu_launches": launches_per_step * args.steps,
         "roofline": {"kernel": "attn_bf16_kernel<8,64> (cross-modal IM attention inside the step)", "bound": "hbm",
                      "achieved": cross["bytes"] / cross_s / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s",
-                     "frac": cross["bytes"] / cross_s / 1e9 / pk["hbm_gbs"], "traffic": ATTN_HD8_DRAM_BYTES, "peak_kind": "of " + pk_kind,
+                     "frac": cross["bytes"] / cross_s / 1e9 / pk["hbm_gbs"], "traffic": recorded_traffic("attn_bf16_hd8_cfg4_cross"), "peak_kind": "of " + pk_kind,
                      "launch_us": cross_s * 1e6, "algorithmic_bytes": cross["bytes"],
                      "timed": "event pair around each launch, rings issued serially for this pass",
                      # the same launch against the exponential unit: one ex2 per useful (query, key) pair per head
@@ -412,6 +494,7 @@ def run_gpu(args):
         "cpu_baseline": {"value": ref_tokens / cpu_s, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
                          "sample": f"{sub} of {B} samples, one step (valid tokens {ref_tokens}) in {cpu_s:.2f} s"},
         "attention": attention,
+        "attention_other_configs": attention_per_config(torch, g, pk, ex2_rate) if not args.no_scaled else {},
         "scaled_attention_hd64": scaled,
         "length_statistics_workload": stats_lengths,
         "step_kernel_ms": {"attention": float(att.sum()) / trace_steps, "linear": lin_ms / trace_steps,
@@ -423,16 +506,33 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
+def _spawned_rank(rank, args, world, port):
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world), MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    os.environ.setdefault("NCCL_DEBUG", "INFO")   # leave NCCL's transport lines (NVLS, P2P) visible in the workers' stderr
+    run_gpu(args)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--repeats", type=int, default=25, help="timed regions of --steps steps each; the median is reported")
     ap.add_argument("--impl", default="gsit", choices=["gsit", "reference"])
     ap.add_argument("--workload", type=int, default=4)
     ap.add_argument("--ref-batch", type=int, default=16, help="samples per step of the CPU oracle")
-    ap.add_argument("--no-scaled", action="store_true", help="skip the extra timing of the head_dim-64 attention")
+    ap.add_argument("--no-scaled", action="store_true", help="skip the extra timings (other configs, head_dim 64, length statistics)")
+    ap.add_argument("--only", choices=["attention", "layer"], help="profiler driver: launch one call a few times and exit")
+    ap.add_argument("--batch", type=int, default=0)
+    ap.add_argument("--phase", type=int, default=0)
+    ap.add_argument("--d", type=int, default=0)
+    ap.add_argument("--heads", type=int, default=0)
+    ap.add_argument("--calls", type=int, default=3)
+    ap.add_argument("--kernels", type=int, default=0, help="--only: kernel choice of include/gsit_test.h (0 = defaults)")
     args = ap.parse_args()
+    if args.only:
+        run_only(args)
+        return
     if args.impl == "reference":
         args.steps = 2 if args.steps is None else args.steps
         args.warmup = 1 if args.warmup is None else args.warmup
@@ -441,6 +541,12 @@ def main():
         return
     args.steps = 200 if args.steps is None else args.steps
     args.warmup = max(3, 5 if args.warmup is None else args.warmup)
+    args.repeats = max(1, args.repeats)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # no launcher around us: start one worker per GPU (NCCL serves only the barrier and the max over ranks)
+        from paper_2505_01068_b200 import shard
+        shard.spawn_ranks(args.gpus, _spawned_rank, (args,))
+        return
     run_gpu(args)
 
 

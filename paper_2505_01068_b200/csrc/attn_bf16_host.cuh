@@ -13,11 +13,9 @@ cudaError_t launch_one(const Geometry& g, const __nv_bfloat16* q, const __nv_bfl
   if (!make_map(&tmQ, q, rows, g.d, row_stride, CW, C::QT) || !make_map(&tmK, k, rows, g.d, row_stride, CW, KT) ||
       !make_map(&tmV, v, rows, g.d, row_stride, CW, KT))
     return cudaErrorInvalidValue;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(attn_bf16_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
+  {
+    cudaError_t e = sm_count_and_smem_once(reinterpret_cast<const void*>(attn_bf16_kernel<C>), C::SMEM, nullptr);
     if (e != cudaSuccess) return e;
-    attr_set = true;
   }
   int tiles = 0;
   for (int s = 0; s < 3; ++s) tiles += (g.seg_len[s] + C::QT - 1) / C::QT;

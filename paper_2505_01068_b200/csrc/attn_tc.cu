@@ -18,119 +18,36 @@
 //                        maximum and sum in registers, writes P (bf16 pairs) back to TMEM with tcgen05.st, rescales
 //                        O in TMEM only when the maximum has grown by more than 2^8, and writes the result.
 // TMEM columns: [0,64) and [64,128) S fp32, [128,160) and [160,192) P bf16x2, [192,256) O fp32.
-// Every wait is bounded; when one expires GSIT_DEVFLAG_TIMEOUT is raised, all later waits give up at once and
+// Every wait is bounded; when one expires GSIT_DEVFLAG_TIMEOUT is raised, the CTA's later waits give up at once and
 // the CTA still releases its TMEM and returns.
 #include <cuda.h>
 
 #include "common.cuh"
+#include "ptx.cuh"
 #include "tensor_map.cuh"
 #include "tmem_ldst.cuh"
 
 namespace gsit {
 namespace {
 
+using namespace ptx;
+
 constexpr int TQ = 128, TK = 64, HD64 = 64;
 constexpr int KV_STAGES = 4, Q_BUFS = 2;
 constexpr int Q_BYTES = TQ * 128, KV_BYTES = TK * 128;  // rows of 128 bytes (64 bf16)
 constexpr int TC_THREADS = 192;
 constexpr int TMEM_COLS = 256, COL_S = 0, COL_P = 128, COL_O = 192;  // S: 2 x 64, P: 2 x 32, O: 64 columns
-constexpr int SPIN_LIMIT = 1 << 16;
 // shared-memory map, relative to a 1024-byte aligned base
 constexpr int OFF_Q = 0, OFF_K = OFF_Q + Q_BUFS * Q_BYTES, OFF_V = OFF_K + KV_STAGES * KV_BYTES,
               OFF_BAR = OFF_V + KV_STAGES * KV_BYTES;
 constexpr int BAR_QFULL = 0, BAR_QEMPTY = 16, BAR_KFULL = 32, BAR_VFULL = 64, BAR_KEMPTY = 96, BAR_VEMPTY = 128,
-              BAR_SFULL = 160, BAR_PFULL = 176, BAR_OFINAL = 192, SLOT_TMEM = 200;
+              BAR_SFULL = 160, BAR_PFULL = 176, BAR_OFINAL = 192, SLOT_TMEM = 200, SLOT_GAVE_UP = 204;
 // Work items are decoded once, by the producer warp, and handed to the other roles through a ring of records in
 // shared memory (the decode needs the sample's valid lengths from global memory and two integer divisions).
 constexpr int ITEM_SLOTS = 8;
 constexpr int OFF_ITEMBAR = OFF_BAR + 256;                      // ITEM_SLOTS "record written" + ITEM_SLOTS "record read" barriers
 constexpr int OFF_ITEMS = OFF_ITEMBAR + 16 * ITEM_SLOTS;        // ITEM_SLOTS records of 16 ints
 constexpr int TC_SMEM = OFF_ITEMS + 64 * ITEM_SLOTS + 1024 /* alignment slack */;
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-// One poll of a phase; the hardware may park the thread for a short, bounded time before answering.
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait.  Gives up after SPIN_LIMIT polls (raising the timeout flag), or as soon as another wait anywhere on
-// the device has already raised it, so that a broken pipeline drains in milliseconds instead of stalling the GPU.
-__device__ __forceinline__ void mbar_wait(const Geometry& g, uint32_t bar, uint32_t parity) {
-  for (int it = 0; it < SPIN_LIMIT; ++it) {
-    if (mbar_try(bar, parity)) return;
-    if ((it & 63) == 63 && (*reinterpret_cast<volatile unsigned int*>(g.status) & GSIT_DEVFLAG_TIMEOUT)) return;
-  }
-  raise_flag(g, GSIT_DEVFLAG_TIMEOUT);
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-// Shared-memory matrix descriptor for tiles whose rows are 128 bytes with the 128-byte swizzle (what TMA wrote):
-// groups of 8 rows are 1024 bytes apart (stride byte offset); the leading byte offset is unused for these shapes.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
-  return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) | (2ull << 61);
-}
-// Instruction descriptor, kind::f16: D = f32, A = B = bf16, M = 128, N = n; b_mn_major: B is stored N-contiguous.
-__host__ __device__ constexpr uint32_t idesc_bf16(int n, bool b_mn_major) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) |
-         ((uint32_t)(128 >> 4) << 24);
-}
-__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
-}
-__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
-}
-// Makes the barrier complete once every tcgen05.mma issued so far by this thread has finished.
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ float ex2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  uint32_t r;
-  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-  return r;
-}
-
-// True in exactly one lane of a converged warp.  The whole warp runs the producer / issuer loops so that addresses,
-// descriptors and barrier phases stay warp-uniform; only the asynchronous instruction itself is issued by one lane.
-__device__ __forceinline__ bool elect_one() {
-  uint32_t pred;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "elect.sync _|p, 0xffffffff;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(pred));
-  return pred != 0;
-}
 
 template <bool V> struct BoolTag { static constexpr bool value = V; };
 
@@ -191,9 +108,9 @@ __device__ __forceinline__ void publish_item(uint32_t base, const Item& it, int 
   __syncwarp();
 }
 // Consumer side (whole warp): waits for record k, copies it to registers and releases the slot (one arrival per warp).
-__device__ __forceinline__ Item fetch_item(const Geometry& g, uint32_t base, int k, int lane) {
+__device__ __forceinline__ Item fetch_item(const WaitCtx& wc, uint32_t base, int k, int lane) {
   const int slot = k % ITEM_SLOTS;
-  mbar_wait(g, base + OFF_ITEMBAR + 8 * slot, (k / ITEM_SLOTS) & 1);
+  mbar_wait(wc, base + OFF_ITEMBAR + 8 * slot, (k / ITEM_SLOTS) & 1);
   const uint32_t a = base + OFF_ITEMS + 64 * slot;
   Item it;
   asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(it.b), "=r"(it.h), "=r"(it.s), "=r"(it.q0) : "r"(a) : "memory");
@@ -213,9 +130,11 @@ attn_tc_hd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t sQ = base + OFF_Q, sK = base + OFF_K, sV = base + OFF_V, bars = base + OFF_BAR;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const WaitCtx wc{g.status, bars + SLOT_GAVE_UP};
 
   // ---- set-up, once per CTA: barriers, tensor memory ----
   if (tid == 0) {
+    asm volatile("st.shared.u32 [%0], %1;" ::"r"(bars + SLOT_GAVE_UP), "r"(0u) : "memory");
 #pragma unroll
     for (int i = 0; i < 2; ++i) {
       mbar_init(bars + BAR_QFULL + 8 * i, 1);
@@ -235,14 +154,9 @@ attn_tc_hd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       mbar_init(base + OFF_ITEMBAR + 8 * i, 1);                   // record written (producer)
       mbar_init(base + OFF_ITEMBAR + 8 * ITEM_SLOTS + 8 * i, 5);  // record read (MMA warp + four softmax warps)
     }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    mbar_init_fence();
   }
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(bars + SLOT_TMEM), "r"(TMEM_COLS)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
+  if (warp == 1) tmem_alloc(bars + SLOT_TMEM, TMEM_COLS);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -256,11 +170,11 @@ attn_tc_hd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       int k = 0;              // items of this CTA so far
       for (int w = blockIdx.x; w < n_items; w += gridDim.x, ++k) {
         const Item it = decode_item(g, w, tiles_per_sample);
-        if (k >= ITEM_SLOTS) mbar_wait(g, base + OFF_ITEMBAR + 8 * ITEM_SLOTS + 8 * (k % ITEM_SLOTS), ((k / ITEM_SLOTS) - 1) & 1);
+        if (k >= ITEM_SLOTS) mbar_wait(wc, base + OFF_ITEMBAR + 8 * ITEM_SLOTS + 8 * (k % ITEM_SLOTS), ((k / ITEM_SLOTS) - 1) & 1);
         publish_item(base, it, k, lane);
         if (it.T == 0) continue;
         const int qb = n_q & 1, quse = n_q >> 1;
-        if (quse > 0) mbar_wait(g, bars + BAR_QEMPTY + 8 * qb, (quse - 1) & 1);
+        if (quse > 0) mbar_wait(wc, bars + BAR_QEMPTY + 8 * qb, (quse - 1) & 1);
         if (elect_one()) {
           mbar_expect_tx(bars + BAR_QFULL + 8 * qb, Q_BYTES);
           tma_load_2d(sQ + qb * Q_BYTES, &tmQ, it.h * HD64, it.b * g.L + g.seg_off[it.s] + it.q0, bars + BAR_QFULL + 8 * qb);
@@ -270,12 +184,12 @@ attn_tc_hd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           int krem, yrow;
           locate(g, it, i, krem, yrow);
           const int st = n_kv % KV_STAGES, use = n_kv / KV_STAGES;
-          if (use > 0) mbar_wait(g, bars + BAR_KEMPTY + 8 * st, (use - 1) & 1);
+          if (use > 0) mbar_wait(wc, bars + BAR_KEMPTY + 8 * st, (use - 1) & 1);
           if (elect_one()) {
             mbar_expect_tx(bars + BAR_KFULL + 8 * st, KV_BYTES);
             tma_load_2d(sK + st * KV_BYTES, &tmK, it.h * HD64, yrow, bars + BAR_KFULL + 8 * st);
           }
-          if (use > 0) mbar_wait(g, bars + BAR_VEMPTY + 8 * st, (use - 1) & 1);
+          if (use > 0) mbar_wait(wc, bars + BAR_VEMPTY + 8 * st, (use - 1) & 1);
           if (elect_one()) {
             mbar_expect_tx(bars + BAR_VFULL + 8 * st, KV_BYTES);
             tma_load_2d(sV + st * KV_BYTES, &tmV, it.h * HD64, yrow, bars + BAR_VFULL + 8 * st);
@@ -291,7 +205,7 @@ attn_tc_hd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                               // (n >> 1) & 1 of their barriers) and ring stage n % KV_STAGES
       int k = 0;
       for (int w = blockIdx.x; w < n_items; w += gridDim.x, ++k) {
-        const Item it = fetch_item(g, base, k, lane);
+        const Item it = fetch_item(wc, base, k, lane);
         if (it.T == 0) continue;
         const int qb = n_q & 1;
         const uint32_t sQb = sQ + qb * Q_BYTES;
@@ -299,7 +213,7 @@ attn_tc_hd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         // read by the softmax of key tile n - 2, whose P this thread has already waited for.
         auto issue_qk = [&](int n, bool last) {
           const int st = n % KV_STAGES;
-          mbar_wait(g, bars + BAR_KFULL + 8 * st, (n / KV_STAGES) & 1);
+          mbar_wait(wc, bars + BAR_KFULL + 8 * st, (n / KV_STAGES) & 1);
           tc_fence_after();
           if (elect_one()) {
 #pragma unroll
@@ -312,14 +226,14 @@ attn_tc_hd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           }
           __syncwarp();
         };
-        mbar_wait(g, bars + BAR_QFULL + 8 * qb, (n_q >> 1) & 1);
+        mbar_wait(wc, bars + BAR_QFULL + 8 * qb, (n_q >> 1) & 1);
         issue_qk(n_kv, it.T == 1);
         for (int j = 0; j < it.T; ++j) {
           const int n = n_kv + j, st = n % KV_STAGES;
           if (j + 1 < it.T) issue_qk(n + 1, j + 2 == it.T);  // scores of the next tile, ahead of this tile's P V
           // P[n & 1] is in TMEM (and, for the first tile of an item, the previous item's O has been read)
-          mbar_wait(g, bars + BAR_PFULL + 8 * (n & 1), (n >> 1) & 1);
-          mbar_wait(g, bars + BAR_VFULL + 8 * st, (n / KV_STAGES) & 1);
+          mbar_wait(wc, bars + BAR_PFULL + 8 * (n & 1), (n >> 1) & 1);
+          mbar_wait(wc, bars + BAR_VFULL + 8 * st, (n / KV_STAGES) & 1);
           tc_fence_after();
           if (elect_one()) {
 #pragma unroll
@@ -344,7 +258,7 @@ attn_tc_hd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 
     int k = 0;
     for (int w = blockIdx.x; w < n_items; w += gridDim.x, ++k) {
-      const Item it = fetch_item(g, base, k, lane);
+      const Item it = fetch_item(wc, base, k, lane);
       const int64_t grow = (int64_t)it.b * g.L + g.seg_off[it.s] + it.q0 + r;
       uint4* dst = reinterpret_cast<uint4*>(out + grow * g.d + it.h * HD64);
       float* lse_row = (lse != nullptr) ? lse + ((int64_t)it.b * g.heads + it.h) * g.L + g.seg_off[it.s] + it.q0 + r : nullptr;
@@ -361,7 +275,7 @@ attn_tc_hd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       auto tile_step = [&](auto ragged_tag, const int j, const int n, const int krem) {
         constexpr bool RAGGED = decltype(ragged_tag)::value;
         const int sb = n & 1;
-        mbar_wait(g, bars + BAR_SFULL + 8 * sb, (n >> 1) & 1);
+        mbar_wait(wc, bars + BAR_SFULL + 8 * sb, (n >> 1) & 1);
         tc_fence_after();
         uint32_t sr[2][32];
 #pragma unroll
@@ -390,7 +304,7 @@ attn_tc_hd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           const float alpha = grow_m ? ex2((m_used - mx) * sl2) : 1.f;
           l *= alpha;
           // O must hold every earlier tile of the item before it is rescaled: wait for the P V of tile n - 1
-          mbar_wait(g, bars + BAR_VEMPTY + 8 * ((n - 1) % KV_STAGES), ((n - 1) / KV_STAGES) & 1);
+          mbar_wait(wc, bars + BAR_VEMPTY + 8 * ((n - 1) % KV_STAGES), ((n - 1) / KV_STAGES) & 1);
           tc_fence_after();
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
@@ -425,15 +339,15 @@ attn_tc_hd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           // Rows of the V tile past the valid length hold whatever follows in memory; a zero weight times NaN or Inf
           // would still poison the accumulator, so clear them before the MMA reads the tile.
           const int st = n % KV_STAGES;
-          mbar_wait(g, bars + BAR_VFULL + 8 * st, (n / KV_STAGES) & 1);
+          mbar_wait(wc, bars + BAR_VFULL + 8 * st, (n / KV_STAGES) & 1);
           const int row = krem + (tid - 64);
           if (row < TK) {
             const uint32_t a = sV + st * KV_BYTES + row * 128;
 #pragma unroll
             for (int c = 0; c < 8; ++c)
-              asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a + 16 * c), "r"(0) : "memory");
+              st_shared_v4(a + 16 * c, 0, 0, 0, 0);
           }
-          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          fence_async_smem();
         }
         tmem_wait_st();
         tc_fence_before();
@@ -449,7 +363,7 @@ attn_tc_hd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       n_kv += it.T;
 
       // ---- epilogue: O / l -> bf16, each thread its own 128-byte row; padded rows +0 ----
-      mbar_wait(g, bars + BAR_OFINAL, n_items_done & 1);
+      mbar_wait(wc, bars + BAR_OFINAL, n_items_done & 1);
       ++n_items_done;
       tc_fence_after();
       const float inv = (l > 0.f) ? 1.f / l : 0.f;
@@ -485,7 +399,7 @@ attn_tc_hd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
+    tmem_dealloc(tmem, TMEM_COLS);
   }
 }
 
@@ -500,14 +414,10 @@ cudaError_t launch_attn_tc_hd64(const Geometry& g, const __nv_bfloat16* q, const
   if (!make_map(&tmQ, q, rows, g.d, row_stride, HD64, TQ) || !make_map(&tmK, k, rows, g.d, row_stride, HD64, TK) ||
       !make_map(&tmV, v, rows, g.d, row_stride, HD64, TK))
     return cudaErrorInvalidValue;
-  static int n_sm = 0;
-  if (n_sm == 0) {
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(attn_tc_hd64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM);
-    if (e != cudaSuccess) { n_sm = 0; return e; }
+  int n_sm = 0;
+  {
+    cudaError_t e = sm_count_and_smem_once(reinterpret_cast<const void*>(attn_tc_hd64_kernel), TC_SMEM, &n_sm);
+    if (e != cudaSuccess) return e;
   }
   int tiles = 0;
   for (int s = 0; s < 3; ++s) tiles += (g.seg_len[s] + TQ - 1) / TQ;

@@ -63,6 +63,32 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);
 }
 
+// Per-device launch set-up (a process may drive several GPUs; kernel attributes and SM counts belong to a device):
+// sets the kernel's dynamic shared-memory limit the first time `func` is launched on the current device and returns
+// that device's SM count.  `func` identifies the kernel; at most 64 devices and 64 kernels are tracked.
+inline cudaError_t sm_count_and_smem_once(const void* func, int smem_bytes, int* n_sm) {
+  constexpr int MAX_DEV = 64, MAX_FUNC = 64;
+  static int sm_count[MAX_DEV] = {};
+  static const void* done[MAX_DEV][MAX_FUNC] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= MAX_DEV) return cudaErrorInvalidDevice;
+  if (sm_count[dev] == 0) {
+    e = cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) { sm_count[dev] = 0; return e; }
+  }
+  if (n_sm != nullptr) *n_sm = sm_count[dev];
+  if (func == nullptr) return cudaSuccess;
+  int i = 0;
+  while (i < MAX_FUNC && done[dev][i] != nullptr && done[dev][i] != func) ++i;
+  if (i < MAX_FUNC && done[dev][i] == func) return cudaSuccess;
+  e = cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+  if (e != cudaSuccess) return e;
+  if (i < MAX_FUNC) done[dev][i] = func;  // beyond the table the attribute is simply set again on every launch
+  return cudaSuccess;
+}
+
 // ---- host-side launch entry points of the kernel files (all asynchronous on `st`) ----
 // Each returns cudaSuccess or the launch error.
 

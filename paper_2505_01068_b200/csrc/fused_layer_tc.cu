@@ -56,9 +56,9 @@ __device__ __forceinline__ void layernorm_row_to_tile(const float (&v)[TD], bool
       const int e = ch * 8 + 2 * k;
       float a = fmaf((v[e] - mean) * rstd, gm[2 * k], bt[2 * k]), b = fmaf((v[e + 1] - mean) * rstd, gm[2 * k + 1], bt[2 * k + 1]);
       if (!real) { a = 0.f; b = 0.f; }
-      pk[k] = t_bf2(a, b);
+      pk[k] = pack_bf16(a, b);
     }
-    st_v4(sw128(tile, r, ch), pk[0], pk[1], pk[2], pk[3]);
+    st_shared_v4(sw128(tile, r, ch), pk[0], pk[1], pk[2], pk[3]);
   }
 }
 
@@ -85,6 +85,7 @@ ln_qkv_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t bars = base + OFF_BAR;
+  const WaitCtx wc{g.status, bars + SLOT + 4};
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int row_base = rows_begin(g), rows = rows_end(g);  // this problem's rows of the activation matrices
   const int ntiles = (rows - row_base + TM - 1) / TM;
@@ -94,56 +95,57 @@ ln_qkv_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
   stage_vector(prm + TD, beta, TD, 0.f, tid, T_THREADS);
   stage_vector(prm + 2 * TD, bias, NQ, 0.f, tid, T_THREADS);
   if (tid == 0) {
-    t_mbar_init(bars + B_W, 1);
-    for (int i = 0; i < 2; ++i) { t_mbar_init(bars + B_XFULL + 8 * i, 1); t_mbar_init(bars + B_XFREE + 8 * i, 4); }
-    t_mbar_init(bars + B_HREADY, 4);
-    t_mbar_init(bars + B_ACCFULL, 1);
-    t_mbar_init(bars + B_ACCFREE, 4);
+    asm volatile("st.shared.u32 [%0], %1;" ::"r"(bars + SLOT + 4), "r"(0u) : "memory");
+    mbar_init(bars + B_W, 1);
+    for (int i = 0; i < 2; ++i) { mbar_init(bars + B_XFULL + 8 * i, 1); mbar_init(bars + B_XFREE + 8 * i, 4); }
+    mbar_init(bars + B_HREADY, 4);
+    mbar_init(bars + B_ACCFULL, 1);
+    mbar_init(bars + B_ACCFREE, 4);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    t_fence_async();
+    fence_async_smem();
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(bars + SLOT), "r"(TMEM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  t_fence_before();
+  tc_fence_before();
   __syncthreads();
-  t_fence_after();
+  tc_fence_after();
   uint32_t tmem;
   asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tmem) : "r"(bars + SLOT) : "memory");
 
   if (warp == 0) {
     // ================================ producer ================================
-    if (t_elect()) {
-      t_mbar_expect_tx(bars + B_W, NQ * 128);
-      t_tma_2d(base + OFF_W, &tmW, 0, 0, bars + B_W);
+    if (elect_one()) {
+      mbar_expect_tx(bars + B_W, NQ * 128);
+      tma_load_2d(base + OFF_W, &tmW, 0, 0, bars + B_W);
     }
     __syncwarp();
     int i = 0;
     for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
       const int xb = i & 1;
-      if (i >= 2) t_mbar_wait(g, bars + B_XFREE + 8 * xb, ((i >> 1) - 1) & 1);  // the row warps hold that tile in registers
-      if (t_elect()) {
-        t_mbar_expect_tx(bars + B_XFULL + 8 * xb, 2 * XBOX);
-        t_tma_2d(base + OFF_X + xb * 2 * XBOX, &tmX, 0, row_base + t * TM, bars + B_XFULL + 8 * xb);
-        t_tma_2d(base + OFF_X + xb * 2 * XBOX + XBOX, &tmX, 32, row_base + t * TM, bars + B_XFULL + 8 * xb);
+      if (i >= 2) mbar_wait(wc, bars + B_XFREE + 8 * xb, ((i >> 1) - 1) & 1);  // the row warps hold that tile in registers
+      if (elect_one()) {
+        mbar_expect_tx(bars + B_XFULL + 8 * xb, 2 * XBOX);
+        tma_load_2d(base + OFF_X + xb * 2 * XBOX, &tmX, 0, row_base + t * TM, bars + B_XFULL + 8 * xb);
+        tma_load_2d(base + OFF_X + xb * 2 * XBOX + XBOX, &tmX, 32, row_base + t * TM, bars + B_XFULL + 8 * xb);
       }
       __syncwarp();
     }
   } else if (warp == 1) {
     // ================================ MMA issuer ================================
-    constexpr uint32_t IDESC = t_idesc(NQ);
-    t_mbar_wait(g, bars + B_W, 0);
+    constexpr uint32_t IDESC = idesc_bf16(NQ, false);
+    mbar_wait(wc, bars + B_W, 0);
     int i = 0;
     for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
-      t_mbar_wait(g, bars + B_HREADY, i & 1);
-      if (i > 0) t_mbar_wait(g, bars + B_ACCFREE, (i - 1) & 1);
-      t_fence_after();
-      if (t_elect()) {
+      mbar_wait(wc, bars + B_HREADY, i & 1);
+      if (i > 0) mbar_wait(wc, bars + B_ACCFREE, (i - 1) & 1);
+      tc_fence_after();
+      if (elect_one()) {
 #pragma unroll
         for (int k = 0; k < TD / 16; ++k)
-          t_umma(tmem, t_desc(base + OFF_H + 32 * k), t_desc(base + OFF_W + 32 * k), IDESC, k > 0);
-        t_commit(bars + B_ACCFULL);
+          umma_ss(tmem, smem_desc_sw128(base + OFF_H + 32 * k), smem_desc_sw128(base + OFF_W + 32 * k), IDESC, k > 0);
+        umma_commit(bars + B_ACCFULL);
       }
       __syncwarp();
     }
@@ -156,7 +158,7 @@ ln_qkv_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
     bool real = row_real32(g, row_base + (int)blockIdx.x * TM + r, rows);
     for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
       const int row0 = row_base + t * TM, xb = i & 1;
-      t_mbar_wait(g, bars + B_XFULL + 8 * xb, (i >> 1) & 1);
+      mbar_wait(wc, bars + B_XFULL + 8 * xb, (i >> 1) & 1);
       float v[TD];
       if (real) {
         load_row64(base + OFF_X + xb * 2 * XBOX, r, v);
@@ -165,16 +167,16 @@ ln_qkv_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
         for (int e = 0; e < TD; ++e) v[e] = 0.f;
       }
       __syncwarp();
-      if (lane == 0) t_mbar_arrive(bars + B_XFREE + 8 * xb);
+      if (lane == 0) mbar_arrive(bars + B_XFREE + 8 * xb);
       // the MMA of the previous tile finished reading the normalised rows before its accumulator was handed over
       layernorm_row_to_tile(v, real, s_gamma, s_beta, eps, base + OFF_H, r);
-      t_fence_async();
+      fence_async_smem();
       __syncwarp();
-      if (lane == 0) t_mbar_arrive(bars + B_HREADY);
+      if (lane == 0) mbar_arrive(bars + B_HREADY);
       const bool real_next = row_real32(g, row_base + (t + (int)gridDim.x) * TM + r, rows);  // overlaps the MMA
 
-      t_mbar_wait(g, bars + B_ACCFULL, i & 1);
-      t_fence_after();
+      mbar_wait(wc, bars + B_ACCFULL, i & 1);
+      tc_fence_after();
       if (i > 0) {  // the previous tile's stores must have finished reading the staging rows
         if (tid == 64) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
         t_bar_rows();
@@ -191,22 +193,22 @@ ln_qkv_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
           float f0 = __uint_as_float(a[e]) + bb.x, f1 = __uint_as_float(a[e + 1]) + bb.y;
           float f2 = __uint_as_float(a[e + 2]) + bb.z, f3 = __uint_as_float(a[e + 3]) + bb.w;
           if (!real) { f0 = 0.f; f1 = 0.f; f2 = 0.f; f3 = 0.f; }
-          pk[e >> 1] = t_bf2(f0, f1);
-          pk[(e >> 1) + 1] = t_bf2(f2, f3);
+          pk[e >> 1] = pack_bf16(f0, f1);
+          pk[(e >> 1) + 1] = pack_bf16(f2, f3);
         }
         const uint32_t box = base + OFF_OUT + (c0 >> 6) * (TM * 128);
         const int ch0 = (c0 & 32) >> 3;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) st_v4(sw128(box, r, ch0 + q), pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+        for (int q = 0; q < 4; ++q) st_shared_v4(sw128(box, r, ch0 + q), pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
       }
-      t_fence_before();
+      tc_fence_before();
       __syncwarp();
-      if (lane == 0) t_mbar_arrive(bars + B_ACCFREE);
-      t_fence_async();
+      if (lane == 0) mbar_arrive(bars + B_ACCFREE);
+      fence_async_smem();
       t_bar_rows();
       if (tid == 64) {
 #pragma unroll
-        for (int j = 0; j < 3; ++j) t_tma_store_2d(&tmOut, base + OFF_OUT + j * (TM * 128), 64 * j, row0);
+        for (int j = 0; j < 3; ++j) tma_store_2d(&tmOut, base + OFF_OUT + j * (TM * 128), 64 * j, row0);
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
       }
       real = real_next;
@@ -214,10 +216,10 @@ ln_qkv_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
     if (tid == 64) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
 
-  t_fence_before();
+  tc_fence_before();
   __syncthreads();
   if (warp == 1) {
-    t_fence_after();
+    tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
   }
 }
@@ -251,6 +253,7 @@ proj_mlp_tc_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_const
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t bars = base + OFF_BAR;
+  const WaitCtx wc{g.status, bars + SLOT + 4};
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int row_base = rows_begin(g), rows = rows_end(g);  // this problem's rows of the activation matrices
   const int ntiles = (rows - row_base + TM - 1) / TM;
@@ -263,94 +266,95 @@ proj_mlp_tc_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_const
   stage_vector(prm + 3 * TD, b2, TD, 0.f, tid, T_THREADS);
   stage_vector(prm + 4 * TD, b1, d_ff, 0.f, tid, T_THREADS);
   if (tid == 0) {
-    t_mbar_init(bars + B_W, 1);
-    for (int i = 0; i < 2; ++i) { t_mbar_init(bars + B_ATTFULL + 8 * i, 1); t_mbar_init(bars + B_ATTFREE + 8 * i, 1); }
-    t_mbar_init(bars + B_XFULL, 1);
-    t_mbar_init(bars + B_XFREE, 4);
-    t_mbar_init(bars + B_ACC1, 1);
-    t_mbar_init(bars + B_HREADY, 4);
-    t_mbar_init(bars + B_ACCF, 1);
-    t_mbar_init(bars + B_FREADY, 4);
-    t_mbar_init(bars + B_ACCY, 1);
+    asm volatile("st.shared.u32 [%0], %1;" ::"r"(bars + SLOT + 4), "r"(0u) : "memory");
+    mbar_init(bars + B_W, 1);
+    for (int i = 0; i < 2; ++i) { mbar_init(bars + B_ATTFULL + 8 * i, 1); mbar_init(bars + B_ATTFREE + 8 * i, 1); }
+    mbar_init(bars + B_XFULL, 1);
+    mbar_init(bars + B_XFREE, 4);
+    mbar_init(bars + B_ACC1, 1);
+    mbar_init(bars + B_HREADY, 4);
+    mbar_init(bars + B_ACCF, 1);
+    mbar_init(bars + B_FREADY, 4);
+    mbar_init(bars + B_ACCY, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    t_fence_async();
+    fence_async_smem();
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(bars + SLOT), "r"(TMEM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  t_fence_before();
+  tc_fence_before();
   __syncthreads();
-  t_fence_after();
+  tc_fence_after();
   uint32_t tmem;
   asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tmem) : "r"(bars + SLOT) : "memory");
 
   if (warp == 0) {
     // ================================ producer ================================
-    if (t_elect()) {
-      t_mbar_expect_tx(bars + B_W, (uint32_t)(TD * 128 + d_ff * 128 + nh * TD * 128));
-      t_tma_2d(base + OFF_WO, &tmWo, 0, 0, bars + B_W);
-      t_tma_2d(base + OFF_W1, &tmW1, 0, 0, bars + B_W);
-      for (int kb = 0; kb < nh; ++kb) t_tma_2d(base + OFF_W2 + kb * TD * 128, &tmW2, 64 * kb, 0, bars + B_W);
+    if (elect_one()) {
+      mbar_expect_tx(bars + B_W, (uint32_t)(TD * 128 + d_ff * 128 + nh * TD * 128));
+      tma_load_2d(base + OFF_WO, &tmWo, 0, 0, bars + B_W);
+      tma_load_2d(base + OFF_W1, &tmW1, 0, 0, bars + B_W);
+      for (int kb = 0; kb < nh; ++kb) tma_load_2d(base + OFF_W2 + kb * TD * 128, &tmW2, 64 * kb, 0, bars + B_W);
     }
     __syncwarp();
     int i = 0;
     for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
       const int row0 = row_base + t * TM;
       const int b = i & 1;
-      if (i >= 2) t_mbar_wait(g, bars + B_ATTFREE + 8 * b, ((i >> 1) - 1) & 1);
-      if (t_elect()) {
-        t_mbar_expect_tx(bars + B_ATTFULL + 8 * b, TM * 128);
-        t_tma_2d(base + OFF_ATT + b * TM * 128, &tmAtt, 0, row0, bars + B_ATTFULL + 8 * b);
+      if (i >= 2) mbar_wait(wc, bars + B_ATTFREE + 8 * b, ((i >> 1) - 1) & 1);
+      if (elect_one()) {
+        mbar_expect_tx(bars + B_ATTFULL + 8 * b, TM * 128);
+        tma_load_2d(base + OFF_ATT + b * TM * 128, &tmAtt, 0, row0, bars + B_ATTFULL + 8 * b);
       }
       __syncwarp();
-      if (i > 0) t_mbar_wait(g, bars + B_XFREE, (i - 1) & 1);
-      if (t_elect()) {
-        t_mbar_expect_tx(bars + B_XFULL, 2 * XBOX);
-        t_tma_2d(base + OFF_X, &tmX, 0, row0, bars + B_XFULL);
-        t_tma_2d(base + OFF_X + XBOX, &tmX, 32, row0, bars + B_XFULL);
+      if (i > 0) mbar_wait(wc, bars + B_XFREE, (i - 1) & 1);
+      if (elect_one()) {
+        mbar_expect_tx(bars + B_XFULL, 2 * XBOX);
+        tma_load_2d(base + OFF_X, &tmX, 0, row0, bars + B_XFULL);
+        tma_load_2d(base + OFF_X + XBOX, &tmX, 32, row0, bars + B_XFULL);
       }
       __syncwarp();
     }
   } else if (warp == 1) {
     // ================================ MMA issuer ================================
-    constexpr uint32_t IDESC_D = t_idesc(TD);
-    const uint32_t idesc_f = t_idesc(d_ff);
-    t_mbar_wait(g, bars + B_W, 0);
+    constexpr uint32_t IDESC_D = idesc_bf16(TD, false);
+    const uint32_t idesc_f = idesc_bf16(d_ff, false);
+    mbar_wait(wc, bars + B_W, 0);
     int i = 0;
     for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
       const int b = i & 1;
       // y1 accumulator = att W_o^T
-      t_mbar_wait(g, bars + B_ATTFULL + 8 * b, (i >> 1) & 1);
-      t_fence_after();
-      if (t_elect()) {
+      mbar_wait(wc, bars + B_ATTFULL + 8 * b, (i >> 1) & 1);
+      tc_fence_after();
+      if (elect_one()) {
 #pragma unroll
         for (int k = 0; k < 4; ++k)
-          t_umma(tmem + COL_1, t_desc(base + OFF_ATT + b * TM * 128 + 32 * k), t_desc(base + OFF_WO + 32 * k), IDESC_D, k > 0);
-        t_commit(bars + B_ATTFREE + 8 * b);
-        t_commit(bars + B_ACC1);
+          umma_ss(tmem + COL_1, smem_desc_sw128(base + OFF_ATT + b * TM * 128 + 32 * k), smem_desc_sw128(base + OFF_WO + 32 * k), IDESC_D, k > 0);
+        umma_commit(bars + B_ATTFREE + 8 * b);
+        umma_commit(bars + B_ACC1);
       }
       __syncwarp();
       // hidden accumulator = LN2(y1) W_1^T
-      t_mbar_wait(g, bars + B_HREADY, i & 1);
-      t_fence_after();
-      if (t_elect()) {
+      mbar_wait(wc, bars + B_HREADY, i & 1);
+      tc_fence_after();
+      if (elect_one()) {
 #pragma unroll
         for (int k = 0; k < 4; ++k)
-          t_umma(tmem + COL_F, t_desc(base + OFF_H + 32 * k), t_desc(base + OFF_W1 + 32 * k), idesc_f, k > 0);
-        t_commit(bars + B_ACCF);
+          umma_ss(tmem + COL_F, smem_desc_sw128(base + OFF_H + 32 * k), smem_desc_sw128(base + OFF_W1 + 32 * k), idesc_f, k > 0);
+        umma_commit(bars + B_ACCF);
       }
       __syncwarp();
       // output accumulator = relu(hidden) W_2^T
-      t_mbar_wait(g, bars + B_FREADY, i & 1);
-      t_fence_after();
-      if (t_elect()) {
+      mbar_wait(wc, bars + B_FREADY, i & 1);
+      tc_fence_after();
+      if (elect_one()) {
         for (int kb = 0; kb < nh; ++kb)
 #pragma unroll
           for (int k = 0; k < 4; ++k)
-            t_umma(tmem + COL_Y, t_desc(base + OFF_F + kb * TM * 128 + 32 * k), t_desc(base + OFF_W2 + kb * TD * 128 + 32 * k),
+            umma_ss(tmem + COL_Y, smem_desc_sw128(base + OFF_F + kb * TM * 128 + 32 * k), smem_desc_sw128(base + OFF_W2 + kb * TD * 128 + 32 * k),
                    IDESC_D, (kb > 0 || k > 0) ? 1u : 0u);
-        t_commit(bars + B_ACCY);
+        umma_commit(bars + B_ACCY);
       }
       __syncwarp();
     }
@@ -365,7 +369,7 @@ proj_mlp_tc_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_const
     for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
       const int row0 = row_base + t * TM;
       // ---- y1 = x + att W_o^T + b_o (registers) ----
-      t_mbar_wait(g, bars + B_XFULL, i & 1);
+      mbar_wait(wc, bars + B_XFULL, i & 1);
       float v[TD];
       if (real) {
         load_row64(base + OFF_X, r, v);
@@ -374,9 +378,9 @@ proj_mlp_tc_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_const
         for (int e = 0; e < TD; ++e) v[e] = 0.f;
       }
       __syncwarp();
-      if (lane == 0) t_mbar_arrive(bars + B_XFREE);
-      t_mbar_wait(g, bars + B_ACC1, i & 1);
-      t_fence_after();
+      if (lane == 0) mbar_arrive(bars + B_XFREE);
+      mbar_wait(wc, bars + B_ACC1, i & 1);
+      tc_fence_after();
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
         uint32_t a[32];
@@ -393,14 +397,14 @@ proj_mlp_tc_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_const
       }
       // ---- h = LN2(y1) -> A operand of the first MLP product ----
       layernorm_row_to_tile(v, real, s_gamma, s_beta, eps, base + OFF_H, r);
-      t_fence_async();
-      t_fence_before();
+      fence_async_smem();
+      tc_fence_before();
       __syncwarp();
-      if (lane == 0) t_mbar_arrive(bars + B_HREADY);
+      if (lane == 0) mbar_arrive(bars + B_HREADY);
       const bool real_next = row_real32(g, row_base + (t + (int)gridDim.x) * TM + r, rows);  // overlaps the MMA
       // ---- f = relu(h W_1^T + b_1) -> A operand of the second MLP product ----
-      t_mbar_wait(g, bars + B_ACCF, i & 1);
-      t_fence_after();
+      mbar_wait(wc, bars + B_ACCF, i & 1);
+      tc_fence_after();
       if (i > 0) {  // the previous tile's output stores must have finished reading the staging rows (they overlay f)
         if (tid == 64) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
         t_bar_rows();
@@ -414,21 +418,21 @@ proj_mlp_tc_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_const
 #pragma unroll
         for (int e = 0; e < 32; e += 4) {
           const float4 bb = ld_v4f(s_b1 + (c0 + e) * 4);
-          pk[e >> 1] = t_bf2(fmaxf(__uint_as_float(a[e]) + bb.x, 0.f), fmaxf(__uint_as_float(a[e + 1]) + bb.y, 0.f));
-          pk[(e >> 1) + 1] = t_bf2(fmaxf(__uint_as_float(a[e + 2]) + bb.z, 0.f), fmaxf(__uint_as_float(a[e + 3]) + bb.w, 0.f));
+          pk[e >> 1] = pack_bf16(fmaxf(__uint_as_float(a[e]) + bb.x, 0.f), fmaxf(__uint_as_float(a[e + 1]) + bb.y, 0.f));
+          pk[(e >> 1) + 1] = pack_bf16(fmaxf(__uint_as_float(a[e + 2]) + bb.z, 0.f), fmaxf(__uint_as_float(a[e + 3]) + bb.w, 0.f));
         }
         const uint32_t blk = base + OFF_F + (c0 >> 6) * (TM * 128);
         const int ch0 = (c0 & 32) >> 3;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) st_v4(sw128(blk, r, ch0 + q), pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+        for (int q = 0; q < 4; ++q) st_shared_v4(sw128(blk, r, ch0 + q), pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
       }
-      t_fence_async();
-      t_fence_before();
+      fence_async_smem();
+      tc_fence_before();
       __syncwarp();
-      if (lane == 0) t_mbar_arrive(bars + B_FREADY);
+      if (lane == 0) mbar_arrive(bars + B_FREADY);
       // ---- y = y1 + f W_2^T + b_2 -> staging rows (two boxes of 32 floats) -> TMA stores; padded rows +0 ----
-      t_mbar_wait(g, bars + B_ACCY, i & 1);
-      t_fence_after();
+      mbar_wait(wc, bars + B_ACCY, i & 1);
+      tc_fence_after();
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
         uint32_t a[32];
@@ -442,15 +446,15 @@ proj_mlp_tc_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_const
           float o0 = v[e] + __uint_as_float(a[4 * ch]) + bb.x, o1 = v[e + 1] + __uint_as_float(a[4 * ch + 1]) + bb.y;
           float o2 = v[e + 2] + __uint_as_float(a[4 * ch + 2]) + bb.z, o3 = v[e + 3] + __uint_as_float(a[4 * ch + 3]) + bb.w;
           if (!real) { o0 = 0.f; o1 = 0.f; o2 = 0.f; o3 = 0.f; }
-          st_v4(sw128(box, r, ch), __float_as_uint(o0), __float_as_uint(o1), __float_as_uint(o2), __float_as_uint(o3));
+          st_shared_v4(sw128(box, r, ch), __float_as_uint(o0), __float_as_uint(o1), __float_as_uint(o2), __float_as_uint(o3));
         }
       }
-      t_fence_before();
-      t_fence_async();
+      tc_fence_before();
+      fence_async_smem();
       t_bar_rows();
       if (tid == 64) {
-        t_tma_store_2d(&tmY, base + OFF_F, 0, row0);
-        t_tma_store_2d(&tmY, base + OFF_F + TM * 128, 32, row0);
+        tma_store_2d(&tmY, base + OFF_F, 0, row0);
+        tma_store_2d(&tmY, base + OFF_F + TM * 128, 32, row0);
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
       }
       real = real_next;
@@ -458,10 +462,10 @@ proj_mlp_tc_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_const
     if (tid == 64) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
 
-  t_fence_before();
+  tc_fence_before();
   __syncthreads();
   if (warp == 1) {
-    t_fence_after();
+    tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
   }
 }
@@ -480,11 +484,9 @@ cudaError_t launch_ln_qkv_tc(const Geometry& g, const float* x, int64_t ldx, con
   if (!make_map(&tmW, w_qkv, 3 * TD, TD, TD, 64, 3 * TD) || !make_map_f32(&tmX, x, rows, TD, ldx, TM) ||
       !make_map(&tmOut, qkv, rows, 3 * TD, 3 * TD, 64, TM))
     return cudaErrorInvalidValue;
-  static bool done = false;
-  if (!done) {
-    cudaError_t e = cudaFuncSetAttribute(ln_qkv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, qk::SMEM);
+  {
+    cudaError_t e = sm_count_and_smem_once(reinterpret_cast<const void*>(ln_qkv_tc_kernel), qk::SMEM, nullptr);
     if (e != cudaSuccess) return e;
-    done = true;
   }
   ln_qkv_tc_kernel<<<min(ntiles, nsm), T_THREADS, qk::SMEM, st>>>(tmW, tmX, tmOut, g, gamma, beta, eps, b_qkv);
   return cudaGetLastError();
@@ -503,11 +505,9 @@ cudaError_t launch_proj_mlp_tc(const Geometry& g, const __nv_bfloat16* att, cons
       !make_map(&tmW1, w_1, d_ff, TD, TD, 64, d_ff) || !make_map(&tmW2, w_2, TD, d_ff, d_ff, 64, TD) ||
       !make_map_f32(&tmY, y, rows, TD, ldy, TM))
     return cudaErrorInvalidValue;
-  static bool done = false;
-  if (!done) {
-    cudaError_t e = cudaFuncSetAttribute(proj_mlp_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, pm::SMEM);
+  {
+    cudaError_t e = sm_count_and_smem_once(reinterpret_cast<const void*>(proj_mlp_tc_kernel), pm::SMEM, nullptr);
     if (e != cudaSuccess) return e;
-    done = true;
   }
   proj_mlp_tc_kernel<<<min(ntiles, nsm), T_THREADS, pm::SMEM, st>>>(tmAtt, tmX, tmWo, tmW1, tmW2, tmY, g, b_o, gamma, beta, eps,
                                                                    b_1, b_2, d_ff);

@@ -48,9 +48,9 @@ __device__ __forceinline__ void layernorm_row128_to_tiles(const float (&v)[D2], 
       const int e = c8 * 8 + 2 * k;
       float a = fmaf((v[e] - mean) * rstd, gm[2 * k], bt[2 * k]), b = fmaf((v[e + 1] - mean) * rstd, gm[2 * k + 1], bt[2 * k + 1]);
       if (!real) { a = 0.f; b = 0.f; }
-      pk[k] = t_bf2(a, b);
+      pk[k] = pack_bf16(a, b);
     }
-    st_v4(sw128(tiles + (c8 >> 3) * XBOX, r, c8 & 7), pk[0], pk[1], pk[2], pk[3]);
+    st_shared_v4(sw128(tiles + (c8 >> 3) * XBOX, r, c8 & 7), pk[0], pk[1], pk[2], pk[3]);
   }
 }
 
@@ -77,6 +77,7 @@ ln_qkv_tc128_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t bars = base + OFF_BAR;
+  const WaitCtx wc{g.status, bars + SLOT + 4};
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int row_base = rows_begin(g), rows = rows_end(g);  // this problem's rows of the activation matrices
   const int ntiles = (rows - row_base + TM - 1) / TM;
@@ -86,64 +87,65 @@ ln_qkv_tc128_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   stage_vector(prm + D2, beta, D2, 0.f, tid, T_THREADS);
   stage_vector(prm + 2 * D2, bias, NQ, 0.f, tid, T_THREADS);
   if (tid == 0) {
-    t_mbar_init(bars + B_W, 1);
-    t_mbar_init(bars + B_XFULL, 1);
-    t_mbar_init(bars + B_XFREE, 4);
-    t_mbar_init(bars + B_HREADY, 4);
-    t_mbar_init(bars + B_ACCFULL, 1);
-    t_mbar_init(bars + B_ACCFREE, 4);
+    asm volatile("st.shared.u32 [%0], %1;" ::"r"(bars + SLOT + 4), "r"(0u) : "memory");
+    mbar_init(bars + B_W, 1);
+    mbar_init(bars + B_XFULL, 1);
+    mbar_init(bars + B_XFREE, 4);
+    mbar_init(bars + B_HREADY, 4);
+    mbar_init(bars + B_ACCFULL, 1);
+    mbar_init(bars + B_ACCFREE, 4);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    t_fence_async();
+    fence_async_smem();
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(bars + SLOT), "r"(TMEM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  t_fence_before();
+  tc_fence_before();
   __syncthreads();
-  t_fence_after();
+  tc_fence_after();
   uint32_t tmem;
   asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tmem) : "r"(bars + SLOT) : "memory");
 
   if (warp == 0) {
     // ================================ producer ================================
-    if (t_elect()) {
-      t_mbar_expect_tx(bars + B_W, 2 * NQ * 128);
+    if (elect_one()) {
+      mbar_expect_tx(bars + B_W, 2 * NQ * 128);
       for (int kb = 0; kb < 2; ++kb)
         for (int j = 0; j < 3; ++j)  // boxes of 128 weight rows
-          t_tma_2d(base + OFF_W + kb * NQ * 128 + j * XBOX, &tmW, 64 * kb, 128 * j, bars + B_W);
+          tma_load_2d(base + OFF_W + kb * NQ * 128 + j * XBOX, &tmW, 64 * kb, 128 * j, bars + B_W);
     }
     __syncwarp();
     int i = 0;
     for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
       // the tile buffer also held the previous tile's normalised rows: wait until the MMA has consumed them
-      if (i > 0) t_mbar_wait(g, bars + B_XFREE, (i - 1) & 1);
-      if (t_elect()) {
-        t_mbar_expect_tx(bars + B_XFULL, 4 * XBOX);
-        for (int j = 0; j < 4; ++j) t_tma_2d(base + OFF_X + j * XBOX, &tmX, 32 * j, row_base + t * TM, bars + B_XFULL);
+      if (i > 0) mbar_wait(wc, bars + B_XFREE, (i - 1) & 1);
+      if (elect_one()) {
+        mbar_expect_tx(bars + B_XFULL, 4 * XBOX);
+        for (int j = 0; j < 4; ++j) tma_load_2d(base + OFF_X + j * XBOX, &tmX, 32 * j, row_base + t * TM, bars + B_XFULL);
       }
       __syncwarp();
     }
   } else if (warp == 1) {
     // ================================ MMA issuer ================================
-    constexpr uint32_t IDESC_256 = t_idesc(256), IDESC_128 = t_idesc(128);
-    t_mbar_wait(g, bars + B_W, 0);
+    constexpr uint32_t IDESC_256 = idesc_bf16(256, false), IDESC_128 = idesc_bf16(128, false);
+    mbar_wait(wc, bars + B_W, 0);
     int i = 0;
     for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
-      t_mbar_wait(g, bars + B_HREADY, i & 1);
-      if (i > 0) t_mbar_wait(g, bars + B_ACCFREE, (i - 1) & 1);
-      t_fence_after();
-      if (t_elect()) {
+      mbar_wait(wc, bars + B_HREADY, i & 1);
+      if (i > 0) mbar_wait(wc, bars + B_ACCFREE, (i - 1) & 1);
+      tc_fence_after();
+      if (elect_one()) {
 #pragma unroll
         for (int kb = 0; kb < 2; ++kb)
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
-            const uint64_t a = t_desc(base + OFF_X + kb * XBOX + 32 * k);
+            const uint64_t a = smem_desc_sw128(base + OFF_X + kb * XBOX + 32 * k);
             const uint32_t w = base + OFF_W + kb * NQ * 128 + 32 * k;
-            t_umma(tmem, a, t_desc(w), IDESC_256, (kb > 0 || k > 0) ? 1u : 0u);                    // columns 0..255
-            t_umma(tmem + 256, a, t_desc(w + 256 * 128), IDESC_128, (kb > 0 || k > 0) ? 1u : 0u);  // columns 256..383
+            umma_ss(tmem, a, smem_desc_sw128(w), IDESC_256, (kb > 0 || k > 0) ? 1u : 0u);                    // columns 0..255
+            umma_ss(tmem + 256, a, smem_desc_sw128(w + 256 * 128), IDESC_128, (kb > 0 || k > 0) ? 1u : 0u);  // columns 256..383
           }
-        t_commit(bars + B_ACCFULL);
+        umma_commit(bars + B_ACCFULL);
       }
       __syncwarp();
     }
@@ -156,7 +158,7 @@ ln_qkv_tc128_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     bool real = row_real32(g, row_base + (int)blockIdx.x * TM + r, rows);
     for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
       const int row0 = row_base + t * TM;
-      t_mbar_wait(g, bars + B_XFULL, i & 1);
+      mbar_wait(wc, bars + B_XFULL, i & 1);
       float v[D2];
       if (real) {
         load_row128(base + OFF_X, r, v);
@@ -166,15 +168,15 @@ ln_qkv_tc128_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       }
       t_bar_rows();  // every row is in registers: the normalised rows may overwrite the tile
       layernorm_row128_to_tiles(v, real, s_gamma, s_beta, eps, base + OFF_X, r);
-      t_fence_async();
+      fence_async_smem();
       __syncwarp();
-      if (lane == 0) t_mbar_arrive(bars + B_HREADY);
+      if (lane == 0) mbar_arrive(bars + B_HREADY);
       const bool real_next = row_real32(g, row_base + (t + (int)gridDim.x) * TM + r, rows);  // overlaps the MMA
 
-      t_mbar_wait(g, bars + B_ACCFULL, i & 1);
-      t_fence_after();
+      mbar_wait(wc, bars + B_ACCFULL, i & 1);
+      tc_fence_after();
       __syncwarp();
-      if (lane == 0) t_mbar_arrive(bars + B_XFREE);  // the MMA has read the normalised rows: the next tile may land
+      if (lane == 0) mbar_arrive(bars + B_XFREE);  // the MMA has read the normalised rows: the next tile may land
 #pragma unroll 1
       for (int pass = 0; pass < 2; ++pass) {
         if (i > 0 || pass > 0) {  // earlier stores must have finished reading the staging rows
@@ -194,24 +196,24 @@ ln_qkv_tc128_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
             float f0 = __uint_as_float(a[e]) + bb.x, f1 = __uint_as_float(a[e + 1]) + bb.y;
             float f2 = __uint_as_float(a[e + 2]) + bb.z, f3 = __uint_as_float(a[e + 3]) + bb.w;
             if (!real) { f0 = 0.f; f1 = 0.f; f2 = 0.f; f3 = 0.f; }
-            pk[e >> 1] = t_bf2(f0, f1);
-            pk[(e >> 1) + 1] = t_bf2(f2, f3);
+            pk[e >> 1] = pack_bf16(f0, f1);
+            pk[(e >> 1) + 1] = pack_bf16(f2, f3);
           }
           const uint32_t box = base + OFF_OUT + (c0 >> 6) * XBOX;
           const int ch0 = (c0 & 32) >> 3;
 #pragma unroll
-          for (int q = 0; q < 4; ++q) st_v4(sw128(box, r, ch0 + q), pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+          for (int q = 0; q < 4; ++q) st_shared_v4(sw128(box, r, ch0 + q), pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
         }
         if (pass == 1) {
-          t_fence_before();
+          tc_fence_before();
           __syncwarp();
-          if (lane == 0) t_mbar_arrive(bars + B_ACCFREE);
+          if (lane == 0) mbar_arrive(bars + B_ACCFREE);
         }
-        t_fence_async();
+        fence_async_smem();
         t_bar_rows();
         if (tid == 64) {
 #pragma unroll
-          for (int j = 0; j < 3; ++j) t_tma_store_2d(&tmOut, base + OFF_OUT + j * XBOX, pass * (NQ / 2) + 64 * j, row0);
+          for (int j = 0; j < 3; ++j) tma_store_2d(&tmOut, base + OFF_OUT + j * XBOX, pass * (NQ / 2) + 64 * j, row0);
           asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         }
       }
@@ -220,10 +222,10 @@ ln_qkv_tc128_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     if (tid == 64) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
 
-  t_fence_before();
+  tc_fence_before();
   __syncthreads();
   if (warp == 1) {
-    t_fence_after();
+    tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
   }
 }
@@ -257,6 +259,7 @@ proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_co
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t bars = base + OFF_BAR;
+  const WaitCtx wc{g.status, bars + SLOT + 4};
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int row_base = rows_begin(g), rows = rows_end(g);  // this problem's rows of the activation matrices
   const int ntiles = (rows - row_base + TM - 1) / TM;
@@ -269,120 +272,121 @@ proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_co
   stage_vector(prm + 3 * D2, b2, D2, 0.f, tid, T_THREADS);
   stage_vector(prm + 4 * D2, b1, d_ff, 0.f, tid, T_THREADS);
   if (tid == 0) {
-    t_mbar_init(bars + B_WO, 1);
-    t_mbar_init(bars + B_ATTFULL, 1);
-    t_mbar_init(bars + B_ATTFREE, 1);
-    t_mbar_init(bars + B_XFULL, 1);
-    t_mbar_init(bars + B_XFREE, 4);
-    t_mbar_init(bars + B_ACC1, 1);
-    t_mbar_init(bars + B_HREADY, 4);
+    asm volatile("st.shared.u32 [%0], %1;" ::"r"(bars + SLOT + 4), "r"(0u) : "memory");
+    mbar_init(bars + B_WO, 1);
+    mbar_init(bars + B_ATTFULL, 1);
+    mbar_init(bars + B_ATTFREE, 1);
+    mbar_init(bars + B_XFULL, 1);
+    mbar_init(bars + B_XFREE, 4);
+    mbar_init(bars + B_ACC1, 1);
+    mbar_init(bars + B_HREADY, 4);
     for (int i = 0; i < 2; ++i) {
-      t_mbar_init(bars + B_WCFULL + 8 * i, 1);
-      t_mbar_init(bars + B_WCFREE + 8 * i, 1);
-      t_mbar_init(bars + B_ACCF + 8 * i, 1);
+      mbar_init(bars + B_WCFULL + 8 * i, 1);
+      mbar_init(bars + B_WCFREE + 8 * i, 1);
+      mbar_init(bars + B_ACCF + 8 * i, 1);
     }
-    t_mbar_init(bars + B_FREADY, 4);
-    t_mbar_init(bars + B_FFREE, 1);
-    t_mbar_init(bars + B_ACCY, 1);
+    mbar_init(bars + B_FREADY, 4);
+    mbar_init(bars + B_FFREE, 1);
+    mbar_init(bars + B_ACCY, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    t_fence_async();
+    fence_async_smem();
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(bars + SLOT), "r"(TMEM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  t_fence_before();
+  tc_fence_before();
   __syncthreads();
-  t_fence_after();
+  tc_fence_after();
   uint32_t tmem;
   asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tmem) : "r"(bars + SLOT) : "memory");
 
   if (warp == 0) {
     // ================================ producer ================================
-    if (t_elect()) {
-      t_mbar_expect_tx(bars + B_WO, 2 * XBOX);
-      for (int kb = 0; kb < 2; ++kb) t_tma_2d(base + OFF_WO + kb * XBOX, &tmWo, 64 * kb, 0, bars + B_WO);
+    if (elect_one()) {
+      mbar_expect_tx(bars + B_WO, 2 * XBOX);
+      for (int kb = 0; kb < 2; ++kb) tma_load_2d(base + OFF_WO + kb * XBOX, &tmWo, 64 * kb, 0, bars + B_WO);
     }
     __syncwarp();
     int i = 0, n = 0;  // tiles, weight chunks requested so far
     for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
       const int row0 = row_base + t * TM;
       // the attention buffer also holds the LN2 rows of the previous tile until its last first-MLP product is done
-      if (i > 0) t_mbar_wait(g, bars + B_ATTFREE, (i - 1) & 1);
-      if (t_elect()) {
-        t_mbar_expect_tx(bars + B_ATTFULL, 2 * XBOX);
-        for (int kb = 0; kb < 2; ++kb) t_tma_2d(base + OFF_ATT + kb * XBOX, &tmAtt, 64 * kb, row0, bars + B_ATTFULL);
+      if (i > 0) mbar_wait(wc, bars + B_ATTFREE, (i - 1) & 1);
+      if (elect_one()) {
+        mbar_expect_tx(bars + B_ATTFULL, 2 * XBOX);
+        for (int kb = 0; kb < 2; ++kb) tma_load_2d(base + OFF_ATT + kb * XBOX, &tmAtt, 64 * kb, row0, bars + B_ATTFULL);
       }
       __syncwarp();
-      if (i > 0) t_mbar_wait(g, bars + B_XFREE, (i - 1) & 1);
-      if (t_elect()) {
-        t_mbar_expect_tx(bars + B_XFULL, 4 * XBOX);
-        for (int j = 0; j < 4; ++j) t_tma_2d(base + OFF_X + j * XBOX, &tmX, 32 * j, row0, bars + B_XFULL);
+      if (i > 0) mbar_wait(wc, bars + B_XFREE, (i - 1) & 1);
+      if (elect_one()) {
+        mbar_expect_tx(bars + B_XFULL, 4 * XBOX);
+        for (int j = 0; j < 4; ++j) tma_load_2d(base + OFF_X + j * XBOX, &tmX, 32 * j, row0, bars + B_XFULL);
       }
       __syncwarp();
       for (int c = 0; c < nc; ++c, ++n) {
         const int st = n & 1, use = n >> 1;
-        if (use > 0) t_mbar_wait(g, bars + B_WCFREE + 8 * st, (use - 1) & 1);
-        if (t_elect()) {
+        if (use > 0) mbar_wait(wc, bars + B_WCFREE + 8 * st, (use - 1) & 1);
+        if (elect_one()) {
           const uint32_t dst = base + OFF_WC + st * WC_STAGE;
-          t_mbar_expect_tx(bars + B_WCFULL + 8 * st, WC_STAGE);
-          t_tma_2d(dst, &tmW1, 0, 64 * c, bars + B_WCFULL + 8 * st);                // W_1[64c .. 64c+63, 0..63]
-          t_tma_2d(dst + 64 * 128, &tmW1, 64, 64 * c, bars + B_WCFULL + 8 * st);    // W_1[64c .. 64c+63, 64..127]
-          t_tma_2d(dst + 2 * 64 * 128, &tmW2, 64 * c, 0, bars + B_WCFULL + 8 * st); // W_2[0..127, 64c .. 64c+63]
+          mbar_expect_tx(bars + B_WCFULL + 8 * st, WC_STAGE);
+          tma_load_2d(dst, &tmW1, 0, 64 * c, bars + B_WCFULL + 8 * st);                // W_1[64c .. 64c+63, 0..63]
+          tma_load_2d(dst + 64 * 128, &tmW1, 64, 64 * c, bars + B_WCFULL + 8 * st);    // W_1[64c .. 64c+63, 64..127]
+          tma_load_2d(dst + 2 * 64 * 128, &tmW2, 64 * c, 0, bars + B_WCFULL + 8 * st); // W_2[0..127, 64c .. 64c+63]
         }
         __syncwarp();
       }
     }
   } else if (warp == 1) {
     // ================================ MMA issuer ================================
-    constexpr uint32_t IDESC_128 = t_idesc(128), IDESC_64 = t_idesc(64);
-    t_mbar_wait(g, bars + B_WO, 0);
+    constexpr uint32_t IDESC_128 = idesc_bf16(128, false), IDESC_64 = idesc_bf16(64, false);
+    mbar_wait(wc, bars + B_WO, 0);
     int i = 0, n = 0;  // tiles done, chunks whose first product has been issued
     for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
       // y1 accumulator = att W_o^T
-      t_mbar_wait(g, bars + B_ATTFULL, i & 1);
-      t_fence_after();
-      if (t_elect()) {
+      mbar_wait(wc, bars + B_ATTFULL, i & 1);
+      tc_fence_after();
+      if (elect_one()) {
 #pragma unroll
         for (int kb = 0; kb < 2; ++kb)
 #pragma unroll
           for (int k = 0; k < 4; ++k)
-            t_umma(tmem + COL_1, t_desc(base + OFF_ATT + kb * XBOX + 32 * k), t_desc(base + OFF_WO + kb * XBOX + 32 * k),
+            umma_ss(tmem + COL_1, smem_desc_sw128(base + OFF_ATT + kb * XBOX + 32 * k), smem_desc_sw128(base + OFF_WO + kb * XBOX + 32 * k),
                    IDESC_128, (kb > 0 || k > 0) ? 1u : 0u);
-        t_commit(bars + B_ACC1);
+        umma_commit(bars + B_ACC1);
       }
       __syncwarp();
-      t_mbar_wait(g, bars + B_HREADY, i & 1);
+      mbar_wait(wc, bars + B_HREADY, i & 1);
       // second product of chunk m (global index): accY += relu-hidden(m) W_2c^T
       auto second = [&](int m, bool first_of_tile, bool last_of_tile) {
-        t_mbar_wait(g, bars + B_FREADY, m & 1);
-        t_fence_after();
-        if (t_elect()) {
+        mbar_wait(wc, bars + B_FREADY, m & 1);
+        tc_fence_after();
+        if (elect_one()) {
           const uint32_t w2 = base + OFF_WC + (m & 1) * WC_STAGE + 2 * 64 * 128;
 #pragma unroll
           for (int k = 0; k < 4; ++k)
-            t_umma(tmem + COL_Y, t_desc(base + OFF_F + 32 * k), t_desc(w2 + 32 * k), IDESC_128, (!first_of_tile || k > 0) ? 1u : 0u);
-          t_commit(bars + B_WCFREE + 8 * (m & 1));
-          t_commit(bars + B_FFREE);
-          if (last_of_tile) t_commit(bars + B_ACCY);
+            umma_ss(tmem + COL_Y, smem_desc_sw128(base + OFF_F + 32 * k), smem_desc_sw128(w2 + 32 * k), IDESC_128, (!first_of_tile || k > 0) ? 1u : 0u);
+          umma_commit(bars + B_WCFREE + 8 * (m & 1));
+          umma_commit(bars + B_FFREE);
+          if (last_of_tile) umma_commit(bars + B_ACCY);
         }
         __syncwarp();
       };
       for (int c = 0; c < nc; ++c, ++n) {
         // first product of chunk n: hidden accumulator (n & 1) = LN2(y1) W_1c^T
         const int st = n & 1;
-        t_mbar_wait(g, bars + B_WCFULL + 8 * st, (n >> 1) & 1);
-        t_fence_after();
-        if (t_elect()) {
+        mbar_wait(wc, bars + B_WCFULL + 8 * st, (n >> 1) & 1);
+        tc_fence_after();
+        if (elect_one()) {
           const uint32_t w1 = base + OFF_WC + st * WC_STAGE;
 #pragma unroll
           for (int kb = 0; kb < 2; ++kb)
 #pragma unroll
             for (int k = 0; k < 4; ++k)
-              t_umma(tmem + COL_F + 64 * st, t_desc(base + OFF_ATT + kb * XBOX + 32 * k), t_desc(w1 + kb * 64 * 128 + 32 * k),
+              umma_ss(tmem + COL_F + 64 * st, smem_desc_sw128(base + OFF_ATT + kb * XBOX + 32 * k), smem_desc_sw128(w1 + kb * 64 * 128 + 32 * k),
                      IDESC_64, (kb > 0 || k > 0) ? 1u : 0u);
-          t_commit(bars + B_ACCF + 8 * st);
-          if (c + 1 == nc) t_commit(bars + B_ATTFREE);  // LN2 rows no longer needed: the next attention tile may land
+          umma_commit(bars + B_ACCF + 8 * st);
+          if (c + 1 == nc) umma_commit(bars + B_ATTFREE);  // LN2 rows no longer needed: the next attention tile may land
         }
         __syncwarp();
         if (c > 0) second(n - 1, c == 1, false);
@@ -400,7 +404,7 @@ proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_co
     for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
       const int row0 = row_base + t * TM;
       // ---- y1 = x + att W_o^T + b_o (registers) ----
-      t_mbar_wait(g, bars + B_XFULL, i & 1);
+      mbar_wait(wc, bars + B_XFULL, i & 1);
       float v[D2];
       if (real) {
         load_row128(base + OFF_X, r, v);
@@ -409,9 +413,9 @@ proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_co
         for (int e = 0; e < D2; ++e) v[e] = 0.f;
       }
       __syncwarp();
-      if (lane == 0) t_mbar_arrive(bars + B_XFREE);
-      t_mbar_wait(g, bars + B_ACC1, i & 1);
-      t_fence_after();
+      if (lane == 0) mbar_arrive(bars + B_XFREE);
+      mbar_wait(wc, bars + B_ACC1, i & 1);
+      tc_fence_after();
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         uint32_t a[32];
@@ -428,16 +432,16 @@ proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_co
       }
       // ---- h = LN2(y1) over the attention tile (its product has completed) ----
       layernorm_row128_to_tiles(v, real, s_gamma, s_beta, eps, base + OFF_ATT, r);
-      t_fence_async();
-      t_fence_before();
+      fence_async_smem();
+      tc_fence_before();
       __syncwarp();
-      if (lane == 0) t_mbar_arrive(bars + B_HREADY);
+      if (lane == 0) mbar_arrive(bars + B_HREADY);
       const bool real_next = row_real32(g, row_base + (t + (int)gridDim.x) * TM + r, rows);
       // ---- hidden chunks: f = relu(h W_1c^T + b_1c) -> A operand of the second product ----
 #pragma unroll 1
       for (int c = 0; c < nc; ++c, ++n) {
-        t_mbar_wait(g, bars + B_ACCF + 8 * (n & 1), (n >> 1) & 1);
-        t_fence_after();
+        mbar_wait(wc, bars + B_ACCF + 8 * (n & 1), (n >> 1) & 1);
+        tc_fence_after();
         uint32_t pk[32];
 #pragma unroll
         for (int hlf = 0; hlf < 2; ++hlf) {
@@ -447,21 +451,21 @@ proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_co
 #pragma unroll
           for (int e = 0; e < 32; e += 4) {
             const float4 bb = ld_v4f(s_b1 + (64 * c + 32 * hlf + e) * 4);
-            pk[16 * hlf + (e >> 1)] = t_bf2(fmaxf(__uint_as_float(a[e]) + bb.x, 0.f), fmaxf(__uint_as_float(a[e + 1]) + bb.y, 0.f));
-            pk[16 * hlf + (e >> 1) + 1] = t_bf2(fmaxf(__uint_as_float(a[e + 2]) + bb.z, 0.f), fmaxf(__uint_as_float(a[e + 3]) + bb.w, 0.f));
+            pk[16 * hlf + (e >> 1)] = pack_bf16(fmaxf(__uint_as_float(a[e]) + bb.x, 0.f), fmaxf(__uint_as_float(a[e + 1]) + bb.y, 0.f));
+            pk[16 * hlf + (e >> 1) + 1] = pack_bf16(fmaxf(__uint_as_float(a[e + 2]) + bb.z, 0.f), fmaxf(__uint_as_float(a[e + 3]) + bb.w, 0.f));
           }
         }
-        if (n > 0) t_mbar_wait(g, bars + B_FFREE, (n - 1) & 1);  // the previous second product has read the hidden chunk
+        if (n > 0) mbar_wait(wc, bars + B_FFREE, (n - 1) & 1);  // the previous second product has read the hidden chunk
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch) st_v4(sw128(base + OFF_F, r, ch), pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
-        t_fence_async();
-        t_fence_before();
+        for (int ch = 0; ch < 8; ++ch) st_shared_v4(sw128(base + OFF_F, r, ch), pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
+        fence_async_smem();
+        tc_fence_before();
         __syncwarp();
-        if (lane == 0) t_mbar_arrive(bars + B_FREADY);
+        if (lane == 0) mbar_arrive(bars + B_FREADY);
       }
       // ---- y = y1 + f W_2^T + b_2: each thread stores its own 512-byte row; padded rows +0 ----
-      t_mbar_wait(g, bars + B_ACCY, i & 1);
-      t_fence_after();
+      mbar_wait(wc, bars + B_ACCY, i & 1);
+      tc_fence_after();
       // The rows leave through a per-warp transpose in shared memory (this warp's 32 rows of the hidden-chunk buffer,
       // which nothing reads between the last second product and this warp's next chunk): a thread owns a row, but a
       // store instruction that writes 16 bytes to each of 32 rows wastes half of every sector, so 32 columns at a time
@@ -479,7 +483,7 @@ proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_co
           float4 o = make_float4(v[32 * c + e] + __uint_as_float(a[e]) + bb.x, v[32 * c + e + 1] + __uint_as_float(a[e + 1]) + bb.y,
                                  v[32 * c + e + 2] + __uint_as_float(a[e + 2]) + bb.z, v[32 * c + e + 3] + __uint_as_float(a[e + 3]) + bb.w);
           if (!real) o = make_float4(0.f, 0.f, 0.f, 0.f);
-          st_v4(scr + lane * 128 + ((((e >> 2)) ^ (lane & 7)) << 4), __float_as_uint(o.x), __float_as_uint(o.y), __float_as_uint(o.z),
+          st_shared_v4(scr + lane * 128 + ((((e >> 2)) ^ (lane & 7)) << 4), __float_as_uint(o.x), __float_as_uint(o.y), __float_as_uint(o.z),
                 __float_as_uint(o.w));
         }
         __syncwarp();
@@ -492,15 +496,15 @@ proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_co
         }
         __syncwarp();
       }
-      t_fence_before();  // orders these TMEM reads before the next tile's products (which wait for this thread's arrivals)
+      tc_fence_before();  // orders these TMEM reads before the next tile's products (which wait for this thread's arrivals)
       real = real_next;
     }
   }
 
-  t_fence_before();
+  tc_fence_before();
   __syncthreads();
   if (warp == 1) {
-    t_fence_after();
+    tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
   }
 }
@@ -519,11 +523,9 @@ cudaError_t launch_ln_qkv_tc128(const Geometry& g, const float* x, int64_t ldx, 
   if (!make_map(&tmW, w_qkv, 3 * D2, D2, D2, 64, 128) || !make_map_f32(&tmX, x, rows, D2, ldx, TM) ||
       !make_map(&tmOut, qkv, rows, 3 * D2, 3 * D2, 64, TM))
     return cudaErrorInvalidValue;
-  static bool done = false;
-  if (!done) {
-    cudaError_t e = cudaFuncSetAttribute(ln_qkv_tc128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, qk2::SMEM);
+  {
+    cudaError_t e = sm_count_and_smem_once(reinterpret_cast<const void*>(ln_qkv_tc128_kernel), qk2::SMEM, nullptr);
     if (e != cudaSuccess) return e;
-    done = true;
   }
   ln_qkv_tc128_kernel<<<min(ntiles, nsm), T_THREADS, qk2::SMEM, st>>>(tmW, tmX, tmOut, g, gamma, beta, eps, b_qkv);
   return cudaGetLastError();
@@ -542,11 +544,9 @@ cudaError_t launch_proj_mlp_tc128(const Geometry& g, const __nv_bfloat16* att, c
       !make_map(&tmWo, w_o, D2, D2, D2, 64, D2) || !make_map(&tmW1, w_1, d_ff, D2, D2, 64, 64) ||
       !make_map(&tmW2, w_2, D2, d_ff, d_ff, 64, D2))
     return cudaErrorInvalidValue;
-  static bool done = false;
-  if (!done) {
-    cudaError_t e = cudaFuncSetAttribute(proj_mlp_tc128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, pm2::SMEM);
+  {
+    cudaError_t e = sm_count_and_smem_once(reinterpret_cast<const void*>(proj_mlp_tc128_kernel), pm2::SMEM, nullptr);
     if (e != cudaSuccess) return e;
-    done = true;
   }
   proj_mlp_tc128_kernel<<<min(ntiles, nsm), T_THREADS, pm2::SMEM, st>>>(tmAtt, tmX, tmWo, tmW1, tmW2, g, b_o, gamma, beta, eps,
                                                                        b_1, b_2, d_ff, y, ldy);

@@ -17,78 +17,21 @@
 #include <cuda.h>
 
 #include "common.cuh"
+#include "ptx.cuh"
 #include "tensor_map.cuh"
 #include "tmem_ldst.cuh"
 
 namespace gsit {
 namespace {
 
+using namespace ptx;
+
 constexpr int GM = 128, GK = 64;          // rows per tile, k-block width
 constexpr int G_THREADS = 192;
 constexpr int A_STAGE = GM * GK * 2;      // 16 KB
-constexpr int G_SPIN = 1 << 16;
 constexpr int G_MAX_STAGES = 6;
 constexpr int G_BAR_BYTES = 256;
 constexpr int G_MIN_SMEM = 120 * 1024;    // more than half an SM's shared memory: one CTA per SM, so 512 TMEM columns fit
-
-__device__ __forceinline__ void g_mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void g_mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void g_mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void g_mbar_wait(const Geometry& g, uint32_t bar, uint32_t parity) {
-  for (int it = 0; it < G_SPIN; ++it) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    if (ok) return;
-    if ((it & 63) == 63 && (*reinterpret_cast<volatile unsigned int*>(g.status) & GSIT_DEVFLAG_TIMEOUT)) return;
-  }
-  raise_flag(g, GSIT_DEVFLAG_TIMEOUT);
-}
-__device__ __forceinline__ void g_tma_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(bar) : "memory");
-}
-__device__ __forceinline__ bool g_elect() {
-  uint32_t pred;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "elect.sync _|p, 0xffffffff;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(pred));
-  return pred != 0;
-}
-// K-major operand tile with 128-byte rows and 128-byte swizzle: 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t g_desc(uint32_t addr) {
-  return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) | (2ull << 61);
-}
-__device__ __forceinline__ void g_umma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
-}
-__device__ __forceinline__ void g_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void g_tma_store_2d(const CUtensorMap* tm, uint32_t src, int x, int y) {
-  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
-               ::"l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(src) : "memory");
-}
-__device__ __forceinline__ uint32_t g_bf2(float lo, float hi) {
-  uint32_t r;
-  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-  return r;
-}
 
 struct GemmParams {
   int M, N, K;
@@ -110,23 +53,21 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t bars = base + p.staging_off + (p.tma_store ? (p.bn / 64) * 16384 : 0);
   const uint32_t bar_full = bars, bar_empty = bars + 8 * G_MAX_STAGES, bar_accf = bars + 16 * G_MAX_STAGES,
-                 bar_acce = bar_accf + 16, slot = bar_acce + 16;
+                 bar_acce = bar_accf + 16, slot = bar_acce + 16, slot_gave_up = slot + 4;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const WaitCtx wc{g.status, slot_gave_up};
   const int kblocks = p.K / GK;
 
   if (tid == 0) {
-    for (int i = 0; i < p.stages; ++i) { g_mbar_init(bar_full + 8 * i, 1); g_mbar_init(bar_empty + 8 * i, 1); }
-    for (int i = 0; i < 2; ++i) { g_mbar_init(bar_accf + 8 * i, 1); g_mbar_init(bar_acce + 8 * i, 4); }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    for (int i = 0; i < p.stages; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_empty + 8 * i, 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_accf + 8 * i, 1); mbar_init(bar_acce + 8 * i, 4); }
+    asm volatile("st.shared.u32 [%0], %1;" ::"r"(slot_gave_up), "r"(0u) : "memory");
+    mbar_init_fence();
   }
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(512) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  if (warp == 1) tmem_alloc(slot, 512);
+  tc_fence_before();
   __syncthreads();
-  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  tc_fence_after();
   uint32_t tmem;
   asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tmem) : "r"(slot) : "memory");
 
@@ -137,12 +78,12 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       const int m0 = (t / p.tiles_n) * GM, n0 = (t % p.tiles_n) * p.bn;
       for (int kb = 0; kb < kblocks; ++kb, ++n) {
         const int st = n % p.stages, use = n / p.stages;
-        if (use > 0) g_mbar_wait(g, bar_empty + 8 * st, (use - 1) & 1);
-        if (g_elect()) {
+        if (use > 0) mbar_wait(wc, bar_empty + 8 * st, (use - 1) & 1);
+        if (elect_one()) {
           const uint32_t sA = base + st * p.stage_bytes;
-          g_mbar_expect_tx(bar_full + 8 * st, (uint32_t)(A_STAGE + p.bn * GK * 2));
-          g_tma_2d(sA, &tmA, kb * GK, m0, bar_full + 8 * st);
-          g_tma_2d(sA + A_STAGE, &tmW, kb * GK, n0, bar_full + 8 * st);
+          mbar_expect_tx(bar_full + 8 * st, (uint32_t)(A_STAGE + p.bn * GK * 2));
+          tma_load_2d(sA, &tmA, kb * GK, m0, bar_full + 8 * st);
+          tma_load_2d(sA + A_STAGE, &tmW, kb * GK, n0, bar_full + 8 * st);
         }
         __syncwarp();
       }
@@ -153,19 +94,19 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     int n = 0, i = 0;  // k-blocks consumed, tiles done by this CTA
     for (int t = blockIdx.x; t < p.n_tiles; t += gridDim.x, ++i) {
       const int ab = i & 1;
-      if (i >= 2) g_mbar_wait(g, bar_acce + 8 * ab, ((i >> 1) - 1) & 1);  // the epilogue has drained this accumulator
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      if (i >= 2) mbar_wait(wc, bar_acce + 8 * ab, ((i >> 1) - 1) & 1);  // the epilogue has drained this accumulator
+      tc_fence_after();
       for (int kb = 0; kb < kblocks; ++kb, ++n) {
         const int st = n % p.stages;
-        g_mbar_wait(g, bar_full + 8 * st, (n / p.stages) & 1);
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        if (g_elect()) {
+        mbar_wait(wc, bar_full + 8 * st, (n / p.stages) & 1);
+        tc_fence_after();
+        if (elect_one()) {
           const uint32_t sA = base + st * p.stage_bytes;
 #pragma unroll
           for (int k = 0; k < GK / 16; ++k)
-            g_umma(tmem + ab * 256, g_desc(sA + 32 * k), g_desc(sA + A_STAGE + 32 * k), idesc, (kb > 0 || k > 0) ? 1u : 0u);
-          g_commit(bar_empty + 8 * st);
-          if (kb + 1 == kblocks) g_commit(bar_accf + 8 * ab);
+            umma_ss(tmem + ab * 256, smem_desc_sw128(sA + 32 * k), smem_desc_sw128(sA + A_STAGE + 32 * k), idesc, (kb > 0 || k > 0) ? 1u : 0u);
+          umma_commit(bar_empty + 8 * st);
+          if (kb + 1 == kblocks) umma_commit(bar_accf + 8 * ab);
         }
         __syncwarp();
       }
@@ -181,8 +122,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       const int64_t row = (int64_t)m0 + quarter * 32 + lane;
       const bool in_m = row < p.M;
       const bool real = in_m && (!p.mask_rows || row_is_real(g, row));
-      g_mbar_wait(g, bar_accf + 8 * ab, (i >> 1) & 1);
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      mbar_wait(wc, bar_accf + 8 * ab, (i >> 1) & 1);
+      tc_fence_after();
       if (p.tma_store) {
         const uint32_t stg = base + p.staging_off;
         const int r = quarter * 32 + lane;
@@ -202,7 +143,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             if (p.bias != nullptr && col0 + e < p.N) { f0 += p.bias[col0 + e]; f1 += p.bias[col0 + e + 1]; }
             if (p.relu) { f0 = fmaxf(f0, 0.f); f1 = fmaxf(f1, 0.f); }
             if (!real) { f0 = 0.f; f1 = 0.f; }
-            pk[e >> 1] = g_bf2(f0, f1);
+            pk[e >> 1] = pack_bf16(f0, f1);
           }
           // box (c0 / 64), row r, 16-byte chunks (c0 % 64) / 8 .. +3, swizzled with the row
           const uint32_t rowp = stg + (c0 >> 6) * 16384 + r * 128;
@@ -212,14 +153,14 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(rowp + (((ch0 + q) ^ (r & 7)) << 4)), "r"(pk[4 * q]),
                          "r"(pk[4 * q + 1]), "r"(pk[4 * q + 2]), "r"(pk[4 * q + 3]) : "memory");
         }
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        tc_fence_before();
         __syncwarp();
-        if (lane == 0) g_mbar_arrive(bar_acce + 8 * ab);  // the accumulator is in shared memory: free it
+        if (lane == 0) mbar_arrive(bar_acce + 8 * ab);  // the accumulator is in shared memory: free it
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (tid == 64) {
           for (int j = 0; j < p.bn / 64; ++j)
-            if (n0 + 64 * j < p.N) g_tma_store_2d(&tmC, stg + j * 16384, n0 + 64 * j, m0);
+            if (n0 + 64 * j < p.N) tma_store_2d(&tmC, stg + j * 16384, n0 + 64 * j, m0);
           asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         }
         continue;
@@ -265,23 +206,23 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
             for (int e = 0; e < 32; e += 8)
               if (col0 + e < p.N)
-                *reinterpret_cast<uint4*>(dst + e) = make_uint4(g_bf2(f[e], f[e + 1]), g_bf2(f[e + 2], f[e + 3]),
-                                                                g_bf2(f[e + 4], f[e + 5]), g_bf2(f[e + 6], f[e + 7]));
+                *reinterpret_cast<uint4*>(dst + e) = make_uint4(pack_bf16(f[e], f[e + 1]), pack_bf16(f[e + 2], f[e + 3]),
+                                                                pack_bf16(f[e + 4], f[e + 5]), pack_bf16(f[e + 6], f[e + 7]));
           }
         }
       }
-      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      tc_fence_before();
       __syncwarp();
-      if (lane == 0) g_mbar_arrive(bar_acce + 8 * ab);
+      if (lane == 0) mbar_arrive(bar_acce + 8 * ab);
     }
   }
 
   if (tid == 64) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // outstanding TMA stores of this CTA
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  tc_fence_before();
   __syncthreads();
   if (warp == 1) {
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
   }
 }
 
@@ -324,13 +265,10 @@ cudaError_t launch_linear_tc_bf16(const Geometry& g, const LinearArgs& a, cudaSt
   } else {
     tmC = tmA;  // unused by the kernel on this path
   }
-  static int n_sm = 0;
-  if (n_sm == 0) {
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(linear_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-    if (e != cudaSuccess) { n_sm = 0; return e; }
+  int n_sm = 0;
+  {
+    cudaError_t e = sm_count_and_smem_once(reinterpret_cast<const void*>(linear_tc_kernel), 227 * 1024, &n_sm);
+    if (e != cudaSuccess) return e;
   }
   const unsigned grid = (unsigned)(p.n_tiles < n_sm ? p.n_tiles : n_sm);
   linear_tc_kernel<<<grid, G_THREADS, smem, st>>>(tmA, tmW, tmC, g, p);

@@ -10,6 +10,7 @@ from __future__ import annotations
 
 import torch
 
+from . import binding as B
 from .stack import GsitStack
 
 
@@ -68,6 +69,10 @@ class HostPipeline:
         self.n += 1
 
     def wait(self):
-        """Blocks until every queued step has delivered its result."""
+        """Blocks until every queued step has delivered its result, then reads the library's device status word: a
+        bounded device-side wait that ran out (the results are then invalid) raises GsitError instead of passing silently."""
         self.s_out.synchronize()
         torch.cuda.current_stream().synchronize()
+        code, flags = B.last_device_status()
+        if code != 0:
+            raise B.GsitError(code, f"HostPipeline: device status flags {flags:#x}")

@@ -186,15 +186,20 @@ class GsitStack:
         B.unpack_rows(res, y, self.seg_len, valid_len, plan)
         return y
 
-    def forward(self, x, valid_len=None, out=None):
+    def forward(self, x, valid_len=None, out=None, check=False):
         """x float32 [B, L, d] -> float32 [B, L, 2d].  The result lives in a buffer owned by this object, or in `out`
-        (float32 [B, L, 2d], contiguous) when one is given."""
+        (float32 [B, L, 2d], contiguous) when one is given.  check=True synchronises the stream afterwards and raises
+        GsitError if a kernel reported a timed-out device-side wait (not for use under stream capture)."""
         if out is not None:
             assert out.shape == (x.shape[0], x.shape[1], 2 * x.shape[2]) and out.dtype == torch.float32 and out.is_contiguous()
         res = self._forward(x, valid_len, out)
         if out is not None and res.data_ptr() != out.data_ptr():
             out.copy_(res)
             res = out
+        if check:
+            code, flags = B.last_device_status()
+            if code != 0:
+                raise B.GsitError(code, f"GsitStack.forward: device status flags {flags:#x}")
         return res
 
     def _forward(self, x, valid_len, out):

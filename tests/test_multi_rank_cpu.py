@@ -80,3 +80,71 @@ def test_stack_chunks_tile_the_batch():
             assert max(sizes) - min(sizes) <= 1 and min(sizes) >= 1
             st.concurrent_rings = False
             assert st._chunks(batch) == [slice(0, batch)]
+
+
+def _stub_rank(rank, tag, out, world, port):
+    """What bench.py's workers do around the step, with a stub step and gloo instead of NCCL."""
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world), MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        from paper_2505_01068_b200 import shard
+        dist.barrier()
+        total, t_max, per_s = shard.job_throughput(100 * (rank + 1), 1.0 + rank)
+        out[rank] = (tag, world, total, t_max)
+    finally:
+        dist.destroy_process_group()
+
+
+def test_spawn_ranks_starts_one_worker_per_rank_and_they_rendezvous():
+    """The launcher bench.py uses for --gpus N without torchrun: N workers, ranks 0..N-1, one rendezvous, job figures equal."""
+    from paper_2505_01068_b200 import shard
+
+    with mp.Manager() as mgr:
+        out = mgr.dict()
+        shard.spawn_ranks(2, _stub_rank, ("tag", out))
+        res = dict(out)
+    assert res == {0: ("tag", 2, 300.0, 2.0), 1: ("tag", 2, 300.0, 2.0)}
+
+
+def test_bench_selects_the_launcher_only_without_a_torchrun_environment(monkeypatch):
+    """`python bench.py --gpus 2` spawns its ranks; under torchrun (WORLD_SIZE set) the process is one of the ranks."""
+    import importlib.util
+    import sys
+    from pathlib import Path
+    from paper_2505_01068_b200 import shard
+
+    spec = importlib.util.spec_from_file_location("bench_under_test", Path(__file__).resolve().parent.parent / "bench.py")
+    bench = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(bench)
+    calls = []
+    monkeypatch.setattr(shard, "spawn_ranks", lambda world, fn, args=(): calls.append(("spawn", world, fn.__name__)))
+    monkeypatch.setattr(bench, "run_gpu", lambda args: calls.append(("run", args.gpus)))
+    monkeypatch.delenv("WORLD_SIZE", raising=False)
+    monkeypatch.setattr(sys, "argv", ["bench.py", "--gpus", "2", "--steps", "3"])
+    bench.main()
+    monkeypatch.setenv("WORLD_SIZE", "2")
+    bench.main()
+    monkeypatch.delenv("WORLD_SIZE")
+    monkeypatch.setattr(sys, "argv", ["bench.py", "--steps", "3"])
+    bench.main()
+    assert calls == [("spawn", 2, "_spawned_rank"), ("run", 2), ("run", 1)]
+
+
+def test_balanced_slices_follow_the_valid_tokens():
+    import workloads as wk
+    from paper_2505_01068_b200 import shard
+
+    wl = wk.WORKLOADS[4]
+    valid = wk.draw_valid_len(np.random.default_rng(wl.seed), wl)
+    cost = valid.sum(axis=1)
+    for world in (1, 2, 3, 8):
+        sl = shard.balanced_slices(cost, world)
+        assert [i for s in sl for i in range(wl.batch)[s]] == list(range(wl.batch))
+        shares = [int(cost[s].sum()) for s in sl]
+        assert max(shares) - min(shares) <= 2 * int(cost.max()) and min(shares) > 0
+    # a heavy sample at one end moves the cut, unlike a split by count
+    assert shard.balanced_slices([1000, 1, 1, 1], 2) == [slice(0, 1), slice(1, 4)]
+    assert shard.balanced_slices([1, 1, 1, 1000], 2) == [slice(0, 3), slice(3, 4)]
+    for n, world in ((0, 2), (1, 3), (2, 2), (5, 8)):
+        sl = shard.balanced_slices([7] * n, world)
+        assert len(sl) == world and [i for s in sl for i in range(n)[s]] == list(range(n))
