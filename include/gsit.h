@@ -136,6 +136,22 @@ gsit_status gsit_im_layer_fwd(const gsit_shape* shape, const gsit_layer_weights*
                               int64_t x_row_stride, float* y, int64_t y_row_stride, void* workspace,
                               size_t workspace_bytes, gsit_stream stream);
 
+/* Two IM encoder layers of the same geometry in one call (Eq. "All-Modal-In-One fusion": the forward-ring and the
+ * backward-ring fusion encoders have their own weights and share nothing until their outputs are put side by side, so
+ * their layers of equal depth are two independent problems of one shape).  Computes exactly what two gsit_im_layer_fwd
+ * calls compute, bit for bit; for bf16 at d_model 64 (d_ff <= 256) each of the layer's three kernels is launched once
+ * for both problems -- every SM works for one of the two, one launch tail is paid instead of two and the result does not
+ * depend on how two streams happen to interleave.  Other shapes run the two layers one after the other.
+ *   shape_a / shape_b  must agree in everything (sizes, dtype, valid_len and row_start pointers, scale) except phase and
+ *                      custom_mask; the two weight sets must have the same d_ff and ln_eps
+ *   x_*, y_*           as for gsit_im_layer_fwd, one pair per problem (x_a and x_b may be the same tensor); no y may
+ *                      overlap any x or the other y
+ *   workspace          2 * gsit_workspace_bytes(shape_a, GSIT_CALL_LAYER, d_ff) bytes, 256-byte aligned */
+gsit_status gsit_im_layer_pair_fwd(const gsit_shape* shape_a, const gsit_shape* shape_b, const gsit_layer_weights* weights_a,
+                                   const gsit_layer_weights* weights_b, const float* x_a, int64_t x_a_row_stride, const float* x_b,
+                                   int64_t x_b_row_stride, float* y_a, int64_t y_a_row_stride, float* y_b, int64_t y_b_row_stride,
+                                   void* workspace, size_t workspace_bytes, gsit_stream stream);
+
 /* Packed row layout, the three helpers (Section "Inner Decomposition for Efficiency": padded positions take no part in
  * the computation; here they take no memory either).  All run on the device, asynchronously on `stream`, and need no
  * host knowledge of the lengths, so a captured sequence of calls stays valid when valid_len changes.

@@ -42,7 +42,7 @@ class LayerWeights(ctypes.Structure):
 EXPORTS = ("gsit_im_qkv_proj", "gsit_im_attention_fwd", "gsit_im_layer_fwd", "gsit_workspace_bytes",
            "gsit_last_device_status", "gsit_status_string", "gsit_version", "gsit_trace_enable", "gsit_trace_read",
            "gsit_trace_launches", "gsit_trace_reset", "gsit_tune_attention", "gsit_test_expire_wait", "gsit_im_layer_fwd_static",
-           "gsit_stack_head_fwd",
+           "gsit_stack_head_fwd", "gsit_im_layer_pair_fwd",
            "gsit_plan_rows", "gsit_pack_rows", "gsit_unpack_rows")
 STATIC_SCRATCH_BYTES = 4 << 20
 KERNEL_ATTENTION, KERNEL_LINEAR, KERNEL_LAYERNORM = 0, 1, 2
@@ -66,6 +66,9 @@ def load():
     lib.gsit_im_attention_fwd.restype = ctypes.c_int
     lib.gsit_im_layer_fwd.argtypes = [sp, ctypes.POINTER(LayerWeights), vp, i64, vp, i64, vp, sz, vp]
     lib.gsit_im_layer_fwd.restype = ctypes.c_int
+    lib.gsit_im_layer_pair_fwd.argtypes = [sp, sp, ctypes.POINTER(LayerWeights), ctypes.POINTER(LayerWeights), vp, i64, vp, i64, vp, i64,
+                                           vp, i64, vp, sz, vp]
+    lib.gsit_im_layer_pair_fwd.restype = ctypes.c_int
     lib.gsit_im_layer_fwd_static.argtypes = [sp, ctypes.POINTER(LayerWeights), vp, i64, vp, i64, vp]
     lib.gsit_im_layer_fwd_static.restype = ctypes.c_int
     lib.gsit_stack_head_fwd.argtypes = [sp, vp, i64, ctypes.c_int32, vp, vp, vp, ctypes.c_int32, vp]
@@ -290,6 +293,39 @@ def im_layer_fwd(x, weights: dict, seg_len, heads, valid_len=None, phase=PHASE_I
     _check(load().gsit_im_layer_fwd(ctypes.byref(shape), ctypes.byref(lw), _ptr(x), x.stride(1), _ptr(out),
                                     out.stride(1), _ptr(workspace), workspace.numel(), _stream()), "gsit_im_layer_fwd")
     return out
+
+
+def im_layer_pair_fwd(x_a, x_b, weights_a: dict, weights_b: dict, seg_len, heads, valid_len=None, phase_a=PHASE_INTER_FWD,
+                      phase_b=PHASE_INTER_BWD, ln_eps=1e-5, out_a=None, out_b=None, workspace=None, row_start=None):
+    """Two layers of one geometry in one call (the two ring encoders' layers of equal depth): same results as two
+    im_layer_fwd calls.  x_* float32 [B, L, d] (or packed [capacity, d] with row_start), out_* likewise (required in the
+    packed layout); workspace: 2 x the layer's workspace bytes."""
+    code = _dtype_code(weights_a["w_qkv"].dtype)
+    lwa, lwb = make_layer_weights(weights_a, ln_eps), make_layer_weights(weights_b, ln_eps)
+    if row_start is not None:
+        cap, d = x_a.shape
+        Bn = valid_len.shape[0]
+        mk = lambda ph: make_shape(Bn, seg_len, d, heads, valid_len, code, ph, 0, 0.0, row_start, cap)
+        strides = lambda t: t.stride(0)
+        assert out_a is not None and out_b is not None
+    else:
+        Bn, L, d = x_a.shape
+        mk = lambda ph: make_shape(Bn, seg_len, d, heads, valid_len, code, ph)
+        strides = lambda t: t.stride(1)
+        if out_a is None:
+            out_a = torch.empty((Bn, L, d), dtype=torch.float32, device=x_a.device)
+        if out_b is None:
+            out_b = torch.empty((Bn, L, d), dtype=torch.float32, device=x_a.device)
+    for t in (x_a, x_b, out_a, out_b):
+        assert t.is_cuda and t.dtype == torch.float32 and t.stride(-1) == 1 and t.shape == x_a.shape
+    sha, shb = mk(phase_a), mk(phase_b)
+    need = 2 * workspace_bytes(sha, CALL_LAYER, lwa.d_ff)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=x_a.device)
+    _check(load().gsit_im_layer_pair_fwd(ctypes.byref(sha), ctypes.byref(shb), ctypes.byref(lwa), ctypes.byref(lwb), _ptr(x_a),
+                                         strides(x_a), _ptr(x_b), strides(x_b), _ptr(out_a), strides(out_a), _ptr(out_b),
+                                         strides(out_b), _ptr(workspace), workspace.numel(), _stream()), "gsit_im_layer_pair_fwd")
+    return out_a, out_b
 
 
 def im_layer_fwd_static(x, weights: dict, seg_len, heads, valid_len=None, phase=PHASE_INTER_FWD, custom_mask=0,

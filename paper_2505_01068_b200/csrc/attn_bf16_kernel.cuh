@@ -7,6 +7,16 @@ namespace {
 template <bool V> struct BoolTag { static constexpr bool value = V; };
 template <int V> struct IntTag { static constexpr int value = V; };
 
+// What distinguishes one attention problem of a launch from the other: its tensors, its block pattern and the order in
+// which its query segments are launched.
+struct AttnProblem {
+  CUtensorMap tmQ, tmK, tmV;
+  __nv_bfloat16* out;
+  float* lse;
+  uint32_t allowed;
+  int seg_order;
+};
+
 #ifndef GSIT_MS_POLY
 #define GSIT_MS_POLY 0
 #endif
@@ -14,9 +24,20 @@ constexpr unsigned MS_POLY = GSIT_MS_POLY;  // bit i: score n-tile i of a step t
 
 template <typename C>
 __global__ void __launch_bounds__(NTHREADS, C::MINB)
-attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                 const __grid_constant__ CUtensorMap tmV, const Geometry g, __nv_bfloat16* __restrict__ out,
-                 float* __restrict__ lse, const float sl2 /* scale * log2(e) */, const int seg_order) {
+attn_bf16_kernel(const __grid_constant__ AttnProblem prob0, const __grid_constant__ AttnProblem prob1, const Geometry g0,
+                 const float sl2 /* scale * log2(e) */, const int problems) {
+  // One launch can serve two problems of the same geometry that differ in their tensors and block pattern (the forward
+  // and the backward ring of one encoder depth); the problem index varies fastest over the grid, so both keep the
+  // longest-first launch order.
+  const int which = (problems == 2) ? (int)(blockIdx.x & 1u) : 0;
+  const int bx = (problems == 2) ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const AttnProblem& prob = which ? prob1 : prob0;
+  const CUtensorMap &tmQ = prob.tmQ, &tmK = prob.tmK, &tmV = prob.tmV;
+  __nv_bfloat16* __restrict__ out = prob.out;
+  float* __restrict__ lse = prob.lse;
+  const int seg_order = prob.seg_order;
+  Geometry g = g0;
+  g.allowed = prob.allowed;
   constexpr int HD = C::HD, CW = C::CW, G = C::G, R = C::R, QT = C::QT, PITCH = C::PITCH, SWZ = C::SWZ,
                 KSTEP = C::KSTEP, NT = C::NT, KSQ = C::KSQ, NTO = C::NTO, CPR = CW / 8 /* 16-byte chunks per row */;
   constexpr bool HOIST = (R > 1);  // several query slabs per warp reuse the K/V fragments of a step
@@ -37,8 +58,8 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   // ---- which tile of which block row.  blockIdx.x = (tile in cost order) * batch + sample: the query segments with
   // the most keys to walk are launched first (seg_order packs the three segment indices, two bits each), and CTAs that
   // run together work on the same tile of different samples, so the last wave is short and made of the cheapest tiles.
-  const int b = blockIdx.x % g.batch;
-  int tile = blockIdx.x / g.batch, s = seg_order & 3;
+  const int b = bx % g.batch;
+  int tile = bx / g.batch, s = seg_order & 3;
 #pragma unroll
   for (int rank = 0; rank < 2; ++rank) {
     const int nts = (g.seg_len[s] + QT - 1) / QT;

@@ -94,11 +94,21 @@ struct SItem {
   int grow0;                    // first row of the query tile in the activation matrices
 };
 
-__device__ __forceinline__ SItem decode_item(const Geometry& g, int w, int slices, int seg_order) {
+// What distinguishes one problem of a launch from the other (a launch serves one or two problems of the same geometry).
+struct SProblem {
+  CUtensorMap tmQ, tmK, tmV;
+  __nv_bfloat16* out;
+  float* lse;
+  uint32_t allowed;
+  int seg_order;
+};
+constexpr int WHICH_SHIFT = 30;  // the problem index rides in bit 30 of the item's slice field
+
+__device__ __forceinline__ SItem decode_item(const Geometry& g, int w, int slices, int seg_order, int which) {
   SItem it;
   it.b = w % g.batch;
   int t = w / g.batch;
-  it.c = t % slices;
+  it.c = (t % slices) | (which << WHICH_SHIFT);
   int tile = t / slices, s = seg_order & 3;
 #pragma unroll
   for (int rank = 0; rank < 2; ++rank) {
@@ -167,16 +177,16 @@ __device__ __forceinline__ SItem fetch_item(const WaitCtx& wc, uint32_t bars, in
 
 template <int HD>
 __global__ void __launch_bounds__(S_THREADS, S_CTAS_PER_SM)
-attn_tcs_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                const __grid_constant__ CUtensorMap tmV, const Geometry g, __nv_bfloat16* __restrict__ out,
-                float* __restrict__ lse, const float sl2 /* scale * log2(e) */, const int slices, const int seg_order,
-                const int n_items, int* __restrict__ next_item /* zeroed counter, or nullptr = static round robin */) {
+attn_tcs_kernel(const __grid_constant__ SProblem prob0, const __grid_constant__ SProblem prob1, const Geometry g0,
+                const float sl2 /* scale * log2(e) */, const int slices, const int n_items /* of all problems */,
+                const int problems, int* __restrict__ next_item /* zeroed counter, or nullptr = static round robin */) {
   using C = SCfg<HD>;
   constexpr int G = C::G, NPV = C::NPV, STAGES = C::STAGES, KVB = C::KV_BYTES, ROWB = C::ROWB;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t sQ = base, sK = base + C::OFF_K, sV = base + C::OFF_V, bars = base + C::OFF_BAR;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const Geometry& g = g0;
   const WaitCtx wc{g.status, bars + B_GAVE_UP};
 
   // ---- set-up, once per CTA: barriers, the zero blocks of the Q layout, tensor memory ----
@@ -234,9 +244,15 @@ attn_tcs_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         publish_item(bars, end, k, lane);
         break;
       }
-      const SItem it = decode_item(g, w, slices, seg_order);
+      const int which = (problems == 2) ? (w & 1) : 0;
+      const SProblem& prob = which ? prob1 : prob0;
+      Geometry g = g0;
+      g.allowed = prob.allowed;
+      SItem it = decode_item(g, (problems == 2) ? (w >> 1) : w, slices, prob.seg_order, which);
       publish_item(bars, it, k, lane);
       if (it.T == 0) continue;
+      it.c &= (1 << WHICH_SHIFT) - 1;
+      const CUtensorMap &tmQ = prob.tmQ, &tmK = prob.tmK, &tmV = prob.tmV;
       const int qb = n_q & 1;
       if (n_q >= 2) mbar_wait(wc, bars + B_QEMPTY + 8 * qb, ((n_q >> 1) - 1) & 1);
       if (elect_one()) {
@@ -354,8 +370,12 @@ attn_tcs_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       const SItem it = fetch_item(wc, bars, k, lane);
       if (it.T < 0) break;
       const int64_t grow = (int64_t)it.grow0 + r;
-      uint4* dst = reinterpret_cast<uint4*>(out + grow * g.d + it.c * C::SLW);
-      float* lse_row = (lse != nullptr) ? lse + ((int64_t)it.b * g.heads + it.c * G) * g.L + g.seg_off[it.s] + it.q0 + r : nullptr;
+      const SProblem& prob = (it.c >> WHICH_SHIFT) ? prob1 : prob0;
+      const int slice = it.c & ((1 << WHICH_SHIFT) - 1);
+      __nv_bfloat16* __restrict__ out = prob.out;
+      float* __restrict__ lse = prob.lse;
+      uint4* dst = reinterpret_cast<uint4*>(out + grow * g.d + slice * C::SLW);
+      float* lse_row = (lse != nullptr) ? lse + ((int64_t)it.b * g.heads + slice * G) * g.L + g.seg_off[it.s] + it.q0 + r : nullptr;
       const bool warp_active = (wq << 5) < it.q_real;  // some row of this warp receives a result
       if (it.T == 0 || !warp_active) {
         // nothing to compute for these rows (padding only, or an empty key set): exact zeros, lse = -inf
@@ -535,55 +555,50 @@ attn_tcs_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   }
 }
 
-constexpr int MAX_DEVICES = 64;
-
 template <int HD>
-cudaError_t launch_tcs(const Geometry& g, const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
-                       int64_t row_stride, __nv_bfloat16* out, float* lse, float scale, int* next_item, cudaStream_t st) {
+cudaError_t launch_tcs(const Geometry& g, const AttnOperands* ops, int n, int64_t row_stride, float scale, int* next_item,
+                       cudaStream_t st) {
   using C = SCfg<HD>;
   const int64_t rows = matrix_rows(g);
-  alignas(64) CUtensorMap tmQ, tmK, tmV;
-  const bool okq = (HD == 8) ? make_map(&tmQ, q, rows, g.d, row_stride, 8, SQ, true)
-                             : make_map(&tmQ, q, rows, g.d, row_stride, C::SLW, SQ);
-  if (!okq || !make_map(&tmK, k, rows, g.d, row_stride, C::SLW, SK) || !make_map(&tmV, v, rows, g.d, row_stride, C::SLW, SK))
-    return cudaErrorInvalidValue;
-  static int n_sm[MAX_DEVICES] = {};  // per device: SM count, and whether the kernel's shared-memory size has been set
-  int dev = 0;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e != cudaSuccess) return e;
-  if (dev < 0 || dev >= MAX_DEVICES) return cudaErrorInvalidDevice;
-  if (n_sm[dev] == 0) {
-    int n = 0;
-    e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(attn_tcs_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
-    if (e != cudaSuccess) return e;
-    n_sm[dev] = n;
+  alignas(64) SProblem pr[2];
+  for (int i = 0; i < n; ++i) {
+    const bool okq = (HD == 8) ? make_map(&pr[i].tmQ, ops[i].q, rows, g.d, row_stride, 8, SQ, true)
+                               : make_map(&pr[i].tmQ, ops[i].q, rows, g.d, row_stride, C::SLW, SQ);
+    if (!okq || !make_map(&pr[i].tmK, ops[i].k, rows, g.d, row_stride, C::SLW, SK) ||
+        !make_map(&pr[i].tmV, ops[i].v, rows, g.d, row_stride, C::SLW, SK))
+      return cudaErrorInvalidValue;
+    pr[i].out = ops[i].out;
+    pr[i].lse = ops[i].lse;
+    pr[i].allowed = ops[i].allowed;
+    // query segments in descending order of the keys their tiles walk (longest work first)
+    int cost[3], ord[3] = {0, 1, 2};
+    for (int s = 0; s < 3; ++s) {
+      cost[s] = 0;
+      for (int r = 0; r < 3; ++r)
+        if ((ops[i].allowed >> (3 * s + r)) & 1u) cost[s] += g.seg_len[r];
+    }
+    for (int a = 0; a < 3; ++a)
+      for (int b = a + 1; b < 3; ++b)
+        if (cost[ord[b]] > cost[ord[a]]) { const int t = ord[a]; ord[a] = ord[b]; ord[b] = t; }
+    pr[i].seg_order = ord[0] | (ord[1] << 2) | (ord[2] << 4);
   }
+  if (n == 1) pr[1] = pr[0];
+  int n_sm = 0;
+  cudaError_t e = sm_count_and_smem_once(reinterpret_cast<const void*>(attn_tcs_kernel<HD>), C::SMEM, &n_sm);
+  if (e != cudaSuccess) return e;
   int tiles = 0;
   for (int s = 0; s < 3; ++s) tiles += (g.seg_len[s] + SQ - 1) / SQ;
   const int slices = g.d / C::SLW;
-  const int64_t n_items = (int64_t)tiles * slices * g.batch;
-  if (n_items > 0x3fffffffLL) return cudaErrorNotSupported;
-  // query segments in descending order of the keys their tiles walk (longest work first)
-  int cost[3], ord[3] = {0, 1, 2};
-  for (int s = 0; s < 3; ++s) {
-    cost[s] = 0;
-    for (int r = 0; r < 3; ++r)
-      if ((g.allowed >> (3 * s + r)) & 1u) cost[s] += g.seg_len[r];
-  }
-  for (int i = 0; i < 3; ++i)
-    for (int j = i + 1; j < 3; ++j)
-      if (cost[ord[j]] > cost[ord[i]]) { const int t = ord[i]; ord[i] = ord[j]; ord[j] = t; }
-  const int seg_order = ord[0] | (ord[1] << 2) | (ord[2] << 4);
-  const int64_t resident = (int64_t)S_CTAS_PER_SM * n_sm[dev];
+  const int64_t n_items = (int64_t)tiles * slices * g.batch * n;
+  if (n_items > 0x3fffffffLL || slices >= (1 << WHICH_SHIFT)) return cudaErrorNotSupported;
+  const int64_t resident = (int64_t)S_CTAS_PER_SM * n_sm;
   const unsigned grid = (unsigned)((n_items < resident) ? n_items : resident);
   if (next_item != nullptr) {
     e = cudaMemsetAsync(next_item, 0, sizeof(int), st);
     if (e != cudaSuccess) return e;
   }
-  attn_tcs_kernel<HD><<<grid, S_THREADS, C::SMEM, st>>>(tmQ, tmK, tmV, g, out, lse, scale * 1.4426950408889634f, slices,
-                                                         seg_order, (int)n_items, next_item);
+  attn_tcs_kernel<HD><<<grid, S_THREADS, C::SMEM, st>>>(pr[0], pr[1], g, scale * 1.4426950408889634f, slices, (int)n_items, n,
+                                                         next_item);
   return cudaGetLastError();
 }
 
@@ -593,13 +608,12 @@ bool attn_tcs_supported(const Geometry& g) {
   return (g.hd == 8 || g.hd == 16) ? (g.d % 16 == 0) : (g.hd == 32 && g.d % 32 == 0);
 }
 
-cudaError_t launch_attn_tcs(const Geometry& g, const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
-                            int64_t row_stride, __nv_bfloat16* out, float* lse, float scale, int* next_item,
+cudaError_t launch_attn_tcs(const Geometry& g, const AttnOperands* ops, int n, int64_t row_stride, float scale, int* next_item,
                             cudaStream_t st) {
-  if (!attn_tcs_supported(g)) return cudaErrorNotSupported;
-  if (g.hd == 8) return launch_tcs<8>(g, q, k, v, row_stride, out, lse, scale, next_item, st);
-  if (g.hd == 16) return launch_tcs<16>(g, q, k, v, row_stride, out, lse, scale, next_item, st);
-  return launch_tcs<32>(g, q, k, v, row_stride, out, lse, scale, next_item, st);
+  if (!attn_tcs_supported(g) || n < 1 || n > 2) return cudaErrorNotSupported;
+  if (g.hd == 8) return launch_tcs<8>(g, ops, n, row_stride, scale, next_item, st);
+  if (g.hd == 16) return launch_tcs<16>(g, ops, n, row_stride, scale, next_item, st);
+  return launch_tcs<32>(g, ops, n, row_stride, scale, next_item, st);
 }
 
 }  // namespace gsit

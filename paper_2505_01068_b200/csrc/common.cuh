@@ -95,6 +95,16 @@ inline cudaError_t sm_count_and_smem_once(const void* func, int smem_bytes, int*
 // fp32 attention on CUDA cores (attn_f32.cu)
 cudaError_t launch_attn_f32(const Geometry& g, const float* q, const float* k, const float* v, int64_t row_stride,
                             float* out, float* lse, float scale, cudaStream_t st);
+// Operands of one bf16 attention problem; launch_attn_bf16_n serves one or two problems of the same geometry (same shape,
+// valid lengths and layout; own tensors and block pattern) with one launch where the kernel family allows it.
+struct AttnOperands {
+  const __nv_bfloat16 *q, *k, *v;
+  __nv_bfloat16* out;
+  float* lse;
+  uint32_t allowed;
+};
+cudaError_t launch_attn_bf16_n(const Geometry& g, const AttnOperands* ops, int n, int64_t row_stride, float scale, int* next_item,
+                               cudaStream_t st);
 // bf16 attention, mma.sync tiles fed by TMA (attn_bf16.cu); returns cudaErrorNotSupported for shapes it lacks
 cudaError_t launch_attn_bf16(const Geometry& g, const __nv_bfloat16* q, const __nv_bfloat16* k,
                              const __nv_bfloat16* v, int64_t row_stride, __nv_bfloat16* out, float* lse,
@@ -109,8 +119,8 @@ cudaError_t launch_attn_tc_hd64(const Geometry& g, const __nv_bfloat16* q, const
 // the call may use as its work counter (it is cleared on the stream before the launch), or nullptr for a fixed
 // assignment of work items to CTAs.
 bool attn_tcs_supported(const Geometry& g);
-cudaError_t launch_attn_tcs(const Geometry& g, const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
-                            int64_t row_stride, __nv_bfloat16* out, float* lse, float scale, int* next_item, cudaStream_t st);
+cudaError_t launch_attn_tcs(const Geometry& g, const AttnOperands* ops, int n, int64_t row_stride, float scale, int* next_item,
+                            cudaStream_t st);
 
 // Linear layers  C = act(A W^T + bias) (+ residual), rows that are padding written as zero when
 // `mask_rows` is set.  A [M,K] (lda), W [N,K], C [M,N] (ldc), residual float [M,N] (ldr) or nullptr.
@@ -150,6 +160,22 @@ cudaError_t launch_proj_mlp_tc(const Geometry& g, const __nv_bfloat16* att, cons
                                const __nv_bfloat16* w_o, const float* b_o, const float* gamma, const float* beta, float eps,
                                const __nv_bfloat16* w_1, const float* b_1, const __nv_bfloat16* w_2, const float* b_2, int d_ff,
                                float* y, int64_t ldy, cudaStream_t st);
+
+// Both halves for a pair of problems of one geometry in one launch each (d_model 64): pointers of one problem.
+struct FusedHalfArgs {
+  const float* x; int64_t ldx;
+  const float *ln1_gamma, *ln1_beta;
+  const __nv_bfloat16* w_qkv; const float* b_qkv;
+  __nv_bfloat16* qkv;            // written by the first half
+  const __nv_bfloat16* att;      // read by the second half
+  const __nv_bfloat16* w_o; const float* b_o;
+  const float *ln2_gamma, *ln2_beta;
+  const __nv_bfloat16* w_1; const float* b_1;
+  const __nv_bfloat16* w_2; const float* b_2;
+  float* y; int64_t ldy;
+};
+cudaError_t launch_ln_qkv_tc_pair(const Geometry& g, const FusedHalfArgs (&h)[2], float eps, cudaStream_t st);
+cudaError_t launch_proj_mlp_tc_pair(const Geometry& g, const FusedHalfArgs (&h)[2], float eps, int d_ff, cudaStream_t st);
 
 // ... and at d_model 128 (d_ff <= 512), with the MLP weights streamed in chunks (fused_layer_tc128.cu)
 bool fused_layer_tc128_supported(const Geometry& g, int d_ff);

@@ -76,11 +76,24 @@ constexpr int SMEM = OFF_BAR + 80 + 1024;
 constexpr int TMEM_COLS = 256;
 }  // namespace qk
 
+// Per-problem arguments of the LN1 + QKV kernel.  One launch can serve two problems of the same geometry (the forward-
+// ring and the backward-ring encoder layers of the same depth, Eq. "All-Modal-In-One fusion": they share nothing but
+// their shape): CTAs with an even index take the first, odd ones the second, each with its own weights resident.
+struct LnQkvArgs {
+  CUtensorMap tmW, tmX, tmOut;
+  const float *gamma, *beta, *bias;
+};
+
 __global__ void __launch_bounds__(T_THREADS, 1)
-ln_qkv_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
-                 const __grid_constant__ CUtensorMap tmOut, const Geometry g, const float* __restrict__ gamma,
-                 const float* __restrict__ beta, const float eps, const float* __restrict__ bias) {
+ln_qkv_tc_kernel(const __grid_constant__ LnQkvArgs arg0, const __grid_constant__ LnQkvArgs arg1, const Geometry g,
+                 const float eps, const int problems) {
   using namespace qk;
+  const int which = (problems == 2) ? (int)(blockIdx.x & 1u) : 0;
+  const int cta = (problems == 2) ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;       // index among the CTAs of this problem
+  const int ctas = (problems == 2) ? (int)((gridDim.x + 1 - which) >> 1) : (int)gridDim.x;
+  const LnQkvArgs& arg = which ? arg1 : arg0;
+  const CUtensorMap &tmW = arg.tmW, &tmX = arg.tmX, &tmOut = arg.tmOut;
+  const float *gamma = arg.gamma, *beta = arg.beta, *bias = arg.bias;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -122,7 +135,7 @@ ln_qkv_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
     }
     __syncwarp();
     int i = 0;
-    for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
+    for (int t = cta; t < ntiles; t += ctas, ++i) {
       const int xb = i & 1;
       if (i >= 2) mbar_wait(wc, bars + B_XFREE + 8 * xb, ((i >> 1) - 1) & 1);  // the row warps hold that tile in registers
       if (elect_one()) {
@@ -137,7 +150,7 @@ ln_qkv_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
     constexpr uint32_t IDESC = idesc_bf16(NQ, false);
     mbar_wait(wc, bars + B_W, 0);
     int i = 0;
-    for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
+    for (int t = cta; t < ntiles; t += ctas, ++i) {
       mbar_wait(wc, bars + B_HREADY, i & 1);
       if (i > 0) mbar_wait(wc, bars + B_ACCFREE, (i - 1) & 1);
       tc_fence_after();
@@ -155,8 +168,8 @@ ln_qkv_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
     const uint32_t tl = tmem + ((uint32_t)((warp & 3) << 5) << 16);
     const uint32_t s_gamma = base + OFF_P, s_beta = s_gamma + TD * 4, s_bias = s_beta + TD * 4;
     int i = 0;
-    bool real = row_real32(g, row_base + (int)blockIdx.x * TM + r, rows);
-    for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
+    bool real = row_real32(g, row_base + cta * TM + r, rows);
+    for (int t = cta; t < ntiles; t += ctas, ++i) {
       const int row0 = row_base + t * TM, xb = i & 1;
       mbar_wait(wc, bars + B_XFULL + 8 * xb, (i >> 1) & 1);
       float v[TD];
@@ -173,7 +186,7 @@ ln_qkv_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
       fence_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(bars + B_HREADY);
-      const bool real_next = row_real32(g, row_base + (t + (int)gridDim.x) * TM + r, rows);  // overlaps the MMA
+      const bool real_next = row_real32(g, row_base + (t + ctas) * TM + r, rows);  // overlaps the MMA
 
       mbar_wait(wc, bars + B_ACCFULL, i & 1);
       tc_fence_after();
@@ -242,13 +255,22 @@ constexpr int COL_1 = 0, COL_F = 64, COL_Y = 320, TMEM_COLS = 512;
 static_assert(SMEM <= 227 * 1024, "shared memory budget");
 }  // namespace pm
 
+// Per-problem arguments of the out-projection + MLP kernel (two problems per launch as for LnQkvArgs).
+struct ProjMlpArgs {
+  CUtensorMap tmAtt, tmX, tmWo, tmW1, tmW2, tmY;
+  const float *bo, *gamma, *beta, *b1, *b2;
+};
+
 __global__ void __launch_bounds__(T_THREADS, 1)
-proj_mlp_tc_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_constant__ CUtensorMap tmX,
-                   const __grid_constant__ CUtensorMap tmWo, const __grid_constant__ CUtensorMap tmW1,
-                   const __grid_constant__ CUtensorMap tmW2, const __grid_constant__ CUtensorMap tmY, const Geometry g,
-                   const float* __restrict__ bo, const float* __restrict__ gamma, const float* __restrict__ beta,
-                   const float eps, const float* __restrict__ b1, const float* __restrict__ b2, const int d_ff) {
+proj_mlp_tc_kernel(const __grid_constant__ ProjMlpArgs arg0, const __grid_constant__ ProjMlpArgs arg1, const Geometry g,
+                   const float eps, const int d_ff, const int problems) {
   using namespace pm;
+  const int which = (problems == 2) ? (int)(blockIdx.x & 1u) : 0;
+  const int cta = (problems == 2) ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int ctas = (problems == 2) ? (int)((gridDim.x + 1 - which) >> 1) : (int)gridDim.x;
+  const ProjMlpArgs& arg = which ? arg1 : arg0;
+  const CUtensorMap &tmAtt = arg.tmAtt, &tmX = arg.tmX, &tmWo = arg.tmWo, &tmW1 = arg.tmW1, &tmW2 = arg.tmW2, &tmY = arg.tmY;
+  const float *bo = arg.bo, *gamma = arg.gamma, *beta = arg.beta, *b1 = arg.b1, *b2 = arg.b2;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -299,7 +321,7 @@ proj_mlp_tc_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_const
     }
     __syncwarp();
     int i = 0;
-    for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
+    for (int t = cta; t < ntiles; t += ctas, ++i) {
       const int row0 = row_base + t * TM;
       const int b = i & 1;
       if (i >= 2) mbar_wait(wc, bars + B_ATTFREE + 8 * b, ((i >> 1) - 1) & 1);
@@ -322,7 +344,7 @@ proj_mlp_tc_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_const
     const uint32_t idesc_f = idesc_bf16(d_ff, false);
     mbar_wait(wc, bars + B_W, 0);
     int i = 0;
-    for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
+    for (int t = cta; t < ntiles; t += ctas, ++i) {
       const int b = i & 1;
       // y1 accumulator = att W_o^T
       mbar_wait(wc, bars + B_ATTFULL + 8 * b, (i >> 1) & 1);
@@ -365,8 +387,8 @@ proj_mlp_tc_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_const
     const uint32_t s_bo = base + OFF_P, s_gamma = s_bo + TD * 4, s_beta = s_gamma + TD * 4, s_b2 = s_beta + TD * 4,
                    s_b1 = s_b2 + TD * 4;
     int i = 0;
-    bool real = row_real32(g, row_base + (int)blockIdx.x * TM + r, rows);
-    for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
+    bool real = row_real32(g, row_base + cta * TM + r, rows);
+    for (int t = cta; t < ntiles; t += ctas, ++i) {
       const int row0 = row_base + t * TM;
       // ---- y1 = x + att W_o^T + b_o (registers) ----
       mbar_wait(wc, bars + B_XFULL, i & 1);
@@ -401,7 +423,7 @@ proj_mlp_tc_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_const
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bars + B_HREADY);
-      const bool real_next = row_real32(g, row_base + (t + (int)gridDim.x) * TM + r, rows);  // overlaps the MMA
+      const bool real_next = row_real32(g, row_base + (t + ctas) * TM + r, rows);  // overlaps the MMA
       // ---- f = relu(h W_1^T + b_1) -> A operand of the second MLP product ----
       mbar_wait(wc, bars + B_ACCF, i & 1);
       tc_fence_after();
@@ -474,21 +496,37 @@ proj_mlp_tc_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_const
 
 bool fused_layer_tc_supported(const Geometry& g, int d_ff) { return g.d == TD && d_ff >= 64 && d_ff <= 256 && d_ff % 64 == 0; }
 
+namespace {
+
+bool fill_ln_qkv(LnQkvArgs* a, int64_t rows, const float* x, int64_t ldx, const float* gamma, const float* beta,
+                 const __nv_bfloat16* w_qkv, const float* b_qkv, __nv_bfloat16* qkv) {
+  a->gamma = gamma; a->beta = beta; a->bias = b_qkv;
+  return make_map(&a->tmW, w_qkv, 3 * TD, TD, TD, 64, 3 * TD) && make_map_f32(&a->tmX, x, rows, TD, ldx, TM) &&
+         make_map(&a->tmOut, qkv, rows, 3 * TD, 3 * TD, 64, TM);
+}
+
+bool fill_proj_mlp(ProjMlpArgs* a, int64_t rows, const __nv_bfloat16* att, const float* x, int64_t ldx, const __nv_bfloat16* w_o,
+                   const float* b_o, const float* gamma, const float* beta, const __nv_bfloat16* w_1, const float* b_1,
+                   const __nv_bfloat16* w_2, const float* b_2, int d_ff, float* y, int64_t ldy) {
+  a->bo = b_o; a->gamma = gamma; a->beta = beta; a->b1 = b_1; a->b2 = b_2;
+  return make_map(&a->tmAtt, att, rows, TD, TD, 64, TM) && make_map_f32(&a->tmX, x, rows, TD, ldx, TM) &&
+         make_map(&a->tmWo, w_o, TD, TD, TD, 64, TD) && make_map(&a->tmW1, w_1, d_ff, TD, TD, 64, d_ff) &&
+         make_map(&a->tmW2, w_2, TD, d_ff, d_ff, 64, TD) && make_map_f32(&a->tmY, y, rows, TD, ldy, TM);
+}
+
+}  // namespace
+
 cudaError_t launch_ln_qkv_tc(const Geometry& g, const float* x, int64_t ldx, const float* gamma, const float* beta, float eps,
                              const __nv_bfloat16* w_qkv, const float* b_qkv, __nv_bfloat16* qkv, cudaStream_t st) {
   if (g.d != TD) return cudaErrorNotSupported;
   const int64_t rows = matrix_rows(g);  // bounds of the tensor maps; the kernel takes its own row range from the geometry
   const int ntiles = (int)((rows + TM - 1) / TM), nsm = t_sm_count();
   if (nsm == 0) return cudaErrorUnknown;
-  alignas(64) CUtensorMap tmW, tmX, tmOut;
-  if (!make_map(&tmW, w_qkv, 3 * TD, TD, TD, 64, 3 * TD) || !make_map_f32(&tmX, x, rows, TD, ldx, TM) ||
-      !make_map(&tmOut, qkv, rows, 3 * TD, 3 * TD, 64, TM))
-    return cudaErrorInvalidValue;
-  {
-    cudaError_t e = sm_count_and_smem_once(reinterpret_cast<const void*>(ln_qkv_tc_kernel), qk::SMEM, nullptr);
-    if (e != cudaSuccess) return e;
-  }
-  ln_qkv_tc_kernel<<<min(ntiles, nsm), T_THREADS, qk::SMEM, st>>>(tmW, tmX, tmOut, g, gamma, beta, eps, b_qkv);
+  alignas(64) LnQkvArgs a;
+  if (!fill_ln_qkv(&a, rows, x, ldx, gamma, beta, w_qkv, b_qkv, qkv)) return cudaErrorInvalidValue;
+  cudaError_t e = sm_count_and_smem_once(reinterpret_cast<const void*>(ln_qkv_tc_kernel), qk::SMEM, nullptr);
+  if (e != cudaSuccess) return e;
+  ln_qkv_tc_kernel<<<min(ntiles, nsm), T_THREADS, qk::SMEM, st>>>(a, a, g, eps, 1);
   return cudaGetLastError();
 }
 
@@ -500,17 +538,45 @@ cudaError_t launch_proj_mlp_tc(const Geometry& g, const __nv_bfloat16* att, cons
   const int64_t rows = matrix_rows(g);  // bounds of the tensor maps; the kernel takes its own row range from the geometry
   const int ntiles = (int)((rows + TM - 1) / TM), nsm = t_sm_count();
   if (nsm == 0) return cudaErrorUnknown;
-  alignas(64) CUtensorMap tmAtt, tmX, tmWo, tmW1, tmW2, tmY;
-  if (!make_map(&tmAtt, att, rows, TD, TD, 64, TM) || !make_map_f32(&tmX, x, rows, TD, ldx, TM) || !make_map(&tmWo, w_o, TD, TD, TD, 64, TD) ||
-      !make_map(&tmW1, w_1, d_ff, TD, TD, 64, d_ff) || !make_map(&tmW2, w_2, TD, d_ff, d_ff, 64, TD) ||
-      !make_map_f32(&tmY, y, rows, TD, ldy, TM))
-    return cudaErrorInvalidValue;
-  {
-    cudaError_t e = sm_count_and_smem_once(reinterpret_cast<const void*>(proj_mlp_tc_kernel), pm::SMEM, nullptr);
-    if (e != cudaSuccess) return e;
-  }
-  proj_mlp_tc_kernel<<<min(ntiles, nsm), T_THREADS, pm::SMEM, st>>>(tmAtt, tmX, tmWo, tmW1, tmW2, tmY, g, b_o, gamma, beta, eps,
-                                                                   b_1, b_2, d_ff);
+  alignas(64) ProjMlpArgs a;
+  if (!fill_proj_mlp(&a, rows, att, x, ldx, w_o, b_o, gamma, beta, w_1, b_1, w_2, b_2, d_ff, y, ldy)) return cudaErrorInvalidValue;
+  cudaError_t e = sm_count_and_smem_once(reinterpret_cast<const void*>(proj_mlp_tc_kernel), pm::SMEM, nullptr);
+  if (e != cudaSuccess) return e;
+  proj_mlp_tc_kernel<<<min(ntiles, nsm), T_THREADS, pm::SMEM, st>>>(a, a, g, eps, d_ff, 1);
+  return cudaGetLastError();
+}
+
+// The same two halves for a PAIR of problems of one geometry in one launch each (the two ring encoders' layers of equal
+// depth): CTAs alternate between the problems, so each problem has half the SMs for the whole launch and one tail is paid
+// instead of two.
+cudaError_t launch_ln_qkv_tc_pair(const Geometry& g, const FusedHalfArgs (&h)[2], float eps, cudaStream_t st) {
+  if (g.d != TD) return cudaErrorNotSupported;
+  const int64_t rows = matrix_rows(g);
+  const int ntiles = (int)((rows + TM - 1) / TM), nsm = t_sm_count();
+  if (nsm < 2) return cudaErrorUnknown;
+  alignas(64) LnQkvArgs a[2];
+  for (int i = 0; i < 2; ++i)
+    if (!fill_ln_qkv(&a[i], rows, h[i].x, h[i].ldx, h[i].ln1_gamma, h[i].ln1_beta, h[i].w_qkv, h[i].b_qkv, h[i].qkv))
+      return cudaErrorInvalidValue;
+  cudaError_t e = sm_count_and_smem_once(reinterpret_cast<const void*>(ln_qkv_tc_kernel), qk::SMEM, nullptr);
+  if (e != cudaSuccess) return e;
+  ln_qkv_tc_kernel<<<min(2 * ntiles, nsm & ~1), T_THREADS, qk::SMEM, st>>>(a[0], a[1], g, eps, 2);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_proj_mlp_tc_pair(const Geometry& g, const FusedHalfArgs (&h)[2], float eps, int d_ff, cudaStream_t st) {
+  if (!fused_layer_tc_supported(g, d_ff)) return cudaErrorNotSupported;
+  const int64_t rows = matrix_rows(g);
+  const int ntiles = (int)((rows + TM - 1) / TM), nsm = t_sm_count();
+  if (nsm < 2) return cudaErrorUnknown;
+  alignas(64) ProjMlpArgs a[2];
+  for (int i = 0; i < 2; ++i)
+    if (!fill_proj_mlp(&a[i], rows, h[i].att, h[i].x, h[i].ldx, h[i].w_o, h[i].b_o, h[i].ln2_gamma, h[i].ln2_beta, h[i].w_1, h[i].b_1,
+                       h[i].w_2, h[i].b_2, d_ff, h[i].y, h[i].ldy))
+      return cudaErrorInvalidValue;
+  cudaError_t e = sm_count_and_smem_once(reinterpret_cast<const void*>(proj_mlp_tc_kernel), pm::SMEM, nullptr);
+  if (e != cudaSuccess) return e;
+  proj_mlp_tc_kernel<<<min(2 * ntiles, nsm & ~1), T_THREADS, pm::SMEM, st>>>(a[0], a[1], g, eps, d_ff, 2);
   return cudaGetLastError();
 }
 

@@ -17,7 +17,7 @@ from . import binding as B
 class GsitStack:
     def __init__(self, fwd_layers, bwd_layers, intra_layers, seg_len, heads, intra_heads, ln_eps=1e-5, head=None,
                  concurrent_rings=True, batch_chunks=1, intra_halves=True,
-                 packed=True):
+                 packed=True, paired_rings=False):
         """head: optional (w_f, b_f) of the read-out X_m = f(|| Split(.)[-1]); see read_out().
         concurrent_rings: issue independent work on several streams (False: every launch on the caller's stream, whole
         batch per launch).  batch_chunks: with concurrent issue, the batch is cut into this many groups of samples, each
@@ -30,12 +30,16 @@ class GsitStack:
         stack works on the packed row layout: the real rows are gathered once, every layer runs on them only, and the
         result is scattered back with +0 in the padded positions.  The row-wise parts of the layers then do no work
         for padding (24 % of the rows at the benchmark's lengths).  The plan of where each segment starts is made on the
-        device, so a captured forward stays valid when the lengths change."""
+        device, so a captured forward stays valid when the lengths change.
+        paired_rings: (packed layout) the forward-ring and backward-ring layers of equal depth go through one
+        gsit_im_layer_pair_fwd call each -- three launches per depth for both rings, on one stream -- instead of two
+        streams of three launches."""
         self.head = head
         self.concurrent_rings = concurrent_rings
         self.batch_chunks = max(1, int(batch_chunks))
         self.intra_halves = bool(intra_halves)
         self.packed = bool(packed)
+        self.paired_rings = bool(paired_rings)
         self.fwd, self.bwd, self.intra = list(fwd_layers), list(bwd_layers), list(intra_layers)
         self.seg_len, self.heads, self.intra_heads, self.ln_eps = tuple(seg_len), heads, intra_heads, ln_eps
         self._bufs = None
@@ -108,7 +112,9 @@ class GsitStack:
                                    capacity=cap)
                 need = max(need, B.workspace_bytes(sh2, B.CALL_LAYER, self.intra[0]["w_1"].shape[0]))
             f32 = dict(dtype=torch.float32, device=x.device)
-            self._bufs[key] = (cap, plan, [torch.empty(need, dtype=torch.uint8, device=x.device) for _ in range(2)],
+            ws_all = torch.empty(2 * need, dtype=torch.uint8, device=x.device)   # one per ring, or both for a paired call
+            self._ws_pair = ws_all
+            self._bufs[key] = (cap, plan, [ws_all[:need], ws_all[need:]],
                                [torch.zeros((cap, d), **f32) for _ in range(5)],
                                torch.zeros((cap, 2 * d), **f32), torch.zeros((cap, 2 * d), **f32),
                                torch.empty((Bn, L, 2 * d), **f32))
@@ -142,7 +148,46 @@ class GsitStack:
                 cur = dst
             return cur
 
-        if not conc:
+        paired = self.paired_rings and len(self.fwd) == len(self.bwd) and len(self.fwd) > 0
+
+        def rings_paired():
+            cur_a = cur_b = xp
+            n = len(self.fwd)
+            for i in range(n):
+                last = i == n - 1
+                dst_a = c0[:, 0:d] if last else t[i % 2]
+                dst_b = c0[:, d:2 * d] if last else t[2 + i % 2]
+                B.im_layer_pair_fwd(cur_a, cur_b, self.fwd[i], self.bwd[i], self.seg_len, self.heads, valid_len, B.PHASE_INTER_FWD,
+                                    B.PHASE_INTER_BWD, ln_eps=self.ln_eps, out_a=dst_a, out_b=dst_b, workspace=self._ws_pair,
+                                    row_start=plan)
+                cur_a, cur_b = dst_a, dst_b
+
+        if paired and not (halves and self.intra):
+            rings_paired()
+            res = intra(0, Bn, ws[0]) if self.intra else c0
+        elif paired:
+            # both rings on the caller's stream, then the intra encoder on the two halves of the batch on two streams
+            rings_paired()
+            if self._lanes is None:
+                dev = x.device
+                self._lanes = ([torch.cuda.Stream(device=dev) for _ in range(2)], torch.cuda.Event(),
+                               [torch.cuda.Event() for _ in range(2)])
+                self._ring_done = [torch.cuda.Event()]
+            streams, fork, done = self._lanes
+            main = torch.cuda.current_stream(x.device)
+            fork.record(main)
+            for si, (lo, hi) in enumerate(((0, mid), (mid, Bn))):
+                streams[si].wait_event(fork)
+                with torch.cuda.stream(streams[si]):
+                    r_ = intra(lo, hi, ws[si])
+                    done[si].record(streams[si])
+                if si == 0:
+                    res = r_
+            for si in range(2):
+                main.wait_event(done[si])
+                x.record_stream(streams[si])
+                valid_len.record_stream(streams[si])
+        elif not conc:
             ring(self.fwd, B.PHASE_INTER_FWD, 0, ws[0], t[0:2])
             ring(self.bwd, B.PHASE_INTER_BWD, 1, ws[0], t[0:2])
             res = intra(0, Bn, ws[0]) if self.intra else c0
