@@ -1,35 +1,38 @@
 // bf16 IM attention for head_dim 8 / 16 / 32 on the 5th-generation tensor cores (tcgen05), scores and accumulators in
-// tensor memory (TMEM), operands fed by TMA.  One thread owns one query row, so the softmax needs no shuffles, no
-// fragment repacking and no shared-memory round trip: per score it costs a maximum, half a packed multiply-add, one
-// exponential, half a packed add and half a conversion.
+// tensor memory (TMEM), operands fed by TMA.  One thread owns one query row of one head, so the softmax needs no
+// shuffles, no fragment repacking and no shared-memory round trip: per score it costs a third of a three-way maximum,
+// half a packed multiply-add, one exponential, half a packed add and half a byte permute.
 //
 // Decomposition (paper, Section "Inner Decomposition for Efficiency"; Appendix A "From Set to Set Aggregation"): a work
-// item is 128 query rows of one modality segment of one sample and a narrow slice of features -- 32 bytes of every row
-// (a pair of heads of 8, or one head of 16), 64 bytes for one head of 32.  It walks only the key tiles (64 keys) of the
-// segment(s) the Interlaced Mask opens for that block row, up to the sample's valid length.  A (key tile, head) pair is a
-// "unit".  Items are small (at most 16 units at the MOSEI shape) and are handed out through an atomic counter, longest
-// first, so that all SMs finish together although the valid lengths differ from sample to sample.
+// item is 128 query rows of one modality segment of one sample and a PAIR OF HEADS (32, 64 or 128 bytes of every row for
+// head_dim 8, 16, 32).  It walks only the key tiles (64 keys) of the segment(s) the Interlaced Mask opens for that block
+// row, up to the sample's valid length.  Items are small (at most 16 head-tiles at the MOSEI shape) and are handed out
+// through an atomic counter, longest first, so that all SMs finish together although the valid lengths differ.
 //
-// The grid is persistent, FOUR light CTAs per SM (128 TMEM columns, at most 80 registers per thread, 32 to 48 KB of shared
-// memory each): a thread-per-row softmax is a long dependent chain per warp, and it is the number of softmax warps per
-// scheduler (four) that keeps the exponential unit and the issue slots busy, not a deep pipeline inside one CTA.
-// Roles inside a CTA of 6 warps:
+// The two heads of an item are two independent chains: each has its own score buffer, weight buffer and accumulator
+// in tensor memory and its own group of four softmax warps.  While one group waits for the round trip
+// weights -> P V and next Q K^T -> scores (some 450 clocks through the MMA warp), the other computes, and with two CTAs
+// per SM every scheduler holds four softmax warps: what keeps the exponential unit and the issue slots busy is the
+// number of independent softmax warps, not a deep pipeline behind one.
+//
+// The grid is persistent, two CTAs per SM.  Roles inside a CTA of 10 warps:
 //   warp 0      takes the next item from the counter, decodes it and hands it to the other warps through a ring of records;
-//               TMA producer: the Q tile of an item (two buffers), K and V tiles of 64 keys x 32 (64) bytes in rings
-//   warp 1      owns the TMEM columns and issues every tcgen05.mma:
-//                 S = Q_h K_h^T  M 128, N 64 (16 per 16-key group of a ragged tile), K 16 per step.  With head_dim 8 a
+//               TMA producer: the Q tile of an item (two buffers), K and V tiles of 64 keys in four-stage rings
+//   warp 1      owns 256 TMEM columns and issues every tcgen05.mma, alternating between the two heads:
+//                 S_h = Q_h K_h^T  M 128, N 64 (16 per 16-key group of a ragged tile), K 16 per step.  With head_dim 8 a
 //                   K step spans the pair of heads in the K tile; the A operand is then [q_h, 0] or [0, q_h]: the Q tile is
 //                   loaded head by head as 16-byte rows and the other core matrix of the step is a block of zeros,
 //                   reached through the descriptor's leading byte offset, so the neighbour head contributes nothing
-//                 O_h += P V     M 128, N 16 (32), K 16 per step; A = P from TMEM, B = the V tile as loaded
+//                 O_h += P_h V     M 128, N 16 (32), K 16 per step; A = P_h from TMEM, B = the V tile as loaded
 //                   (N-contiguous).  With head_dim 8, N = 16 covers the head pair; the neighbour's 8 columns of each
 //                   head's accumulator are never read
-//   warps 2..5  softmax: thread = query row = TMEM lane.  Two passes over the scores in groups of 16 columns (maximum,
-//               then weights), running maximum and sum in registers, O rescaled in TMEM only when the maximum has grown by
-//               more than 2^8.  Warps whose 32 rows hold no real query skip the arithmetic.
-// TMEM columns: [0,64) S fp32, [64,96) P bf16x2, [96,128) one accumulator of 16 (32) columns per head.  Every wait is
-// bounded; when one expires GSIT_DEVFLAG_TIMEOUT is raised, the CTA's other waits give up at once, and the CTA still
-// releases its TMEM and returns.
+//   warps 2..5  softmax of head 0, warps 6..9 of head 1: thread = query row = TMEM lane.  Two passes over the scores in
+//               groups of 16 columns (maximum, then weights), running maximum and sum in registers, O_h rescaled in TMEM
+//               only when the maximum has grown by more than 2^8.  Warps whose 32 rows hold no real query skip the
+//               arithmetic.
+// TMEM columns: [0,64) S_0, [64,128) S_1 fp32; [128,160) P_0, [160,192) P_1 bf16x2; [192,224) O_0, [224,256) O_1.
+// Every wait is bounded; when one expires GSIT_DEVFLAG_TIMEOUT is raised, the CTA's other waits give up at once, and the
+// CTA still releases its TMEM and returns.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -43,11 +46,11 @@ namespace {
 using namespace ptx;
 
 constexpr int SQ = 128, SK = 64;
-constexpr int S_THREADS = 192;
-constexpr int S_TMEM_COLS = 128, S_COL_P = 64, S_COL_O = 96;
-constexpr int S_CTAS_PER_SM = 4;
+constexpr int S_THREADS = 320;
+constexpr int S_TMEM_COLS = 256, S_COL_P = 128, S_COL_O = 192;
+constexpr int S_CTAS_PER_SM = 2;
 constexpr int S_ITEM_SLOTS = 4;
-constexpr int S_QBUF = 8192;  // bytes reserved per Q buffer
+constexpr int S_QBUF = 16384;  // bytes reserved per Q buffer
 #ifndef GSIT_POLY_PAIRS
 #define GSIT_POLY_PAIRS 0x52
 #endif
@@ -61,15 +64,14 @@ constexpr float TRUNC_LOG2 = 0.0020273f;  // log2(TRUNC_GAIN)
 constexpr unsigned POLY_PAIRS = GSIT_POLY_PAIRS;  // bit i: pair i of every 16-key group takes the polynomial 2^x
 // barriers (8 bytes each), relative to the barrier block
 constexpr int B_QFULL = 0, B_QEMPTY = 16, B_SFULL = 32, B_PFULL = 48, B_OFINAL = 64, B_TMEM_SLOT = 72, B_GAVE_UP = 76,
-              B_ITEMBAR = 80, B_ITEMS = 256, B_KFULL = 512, B_VFULL = 576, B_KEMPTY = 640, B_VEMPTY = 704, B_END = 768;
+              B_ITEMBAR = 80, B_ITEMS = 256, B_KFULL = 512, B_VFULL = 576, B_KVEMPTY = 640, B_END = 704;
 
 template <int HD>
 struct SCfg {
-  static constexpr int SLW = (HD == 32) ? 32 : 16;   // features per slice
-  static constexpr int ROWB = SLW * 2;               // bytes per tile row
-  static constexpr int G = SLW / HD;                 // heads per slice
-  static constexpr int NPV = SLW;                    // N of O_h += P V
-  static constexpr uint32_t SWZ = (ROWB == 32) ? 6u : 4u;   // descriptor code of the 32-byte / 64-byte swizzle
+  static constexpr int SLW = 2 * HD;                 // features per slice: a pair of heads
+  static constexpr int ROWB = SLW * 2;               // bytes per tile row: 32, 64, 128
+  static constexpr int NPV = (HD == 8) ? 16 : HD;    // N of O_h += P_h V
+  static constexpr uint32_t SWZ = (ROWB == 32) ? 6u : (ROWB == 64) ? 4u : 2u;  // descriptor code of the 32 / 64 / 128-byte swizzle
   static constexpr uint32_t SBO = 8 * ROWB;          // bytes between groups of 8 rows
   static constexpr int KV_BYTES = SK * ROWB;
   static constexpr int STAGES = 4;
@@ -78,7 +80,7 @@ struct SCfg {
   static constexpr int SMEM = OFF_BAR + B_END + 1024 /* alignment slack */;
 };
 
-// Descriptor of a swizzled tile as TMA wrote it (rows of 32 or 64 bytes): groups of 8 rows `sbo` bytes apart.
+// Descriptor of a swizzled tile as TMA wrote it (rows of 32, 64 or 128 bytes): groups of 8 rows `sbo` bytes apart.
 __device__ __forceinline__ uint64_t smem_desc_sw(uint32_t addr, uint32_t sbo, uint32_t code) {
   return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)(sbo >> 4) << 32) | (1ull << 46) | ((uint64_t)code << 61);
 }
@@ -181,7 +183,7 @@ attn_tcs_kernel(const __grid_constant__ SProblem prob0, const __grid_constant__ 
                 const float sl2 /* scale * log2(e) */, const int slices, const int n_items /* of all problems */,
                 const int problems, int* __restrict__ next_item /* zeroed counter, or nullptr = static round robin */) {
   using C = SCfg<HD>;
-  constexpr int G = C::G, NPV = C::NPV, STAGES = C::STAGES, KVB = C::KV_BYTES, ROWB = C::ROWB;
+  constexpr int NPV = C::NPV, STAGES = C::STAGES, KVB = C::KV_BYTES, ROWB = C::ROWB;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t sQ = base, sK = base + C::OFF_K, sV = base + C::OFF_V, bars = base + C::OFF_BAR;
@@ -196,19 +198,21 @@ attn_tcs_kernel(const __grid_constant__ SProblem prob0, const __grid_constant__ 
       mbar_init(bars + B_QFULL + 8 * i, 1);
       mbar_init(bars + B_QEMPTY + 8 * i, 1);
     }
-    mbar_init(bars + B_SFULL, 1);
-    mbar_init(bars + B_PFULL, 4);  // one arrival per softmax warp
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      mbar_init(bars + B_SFULL + 8 * h, 1);
+      mbar_init(bars + B_PFULL + 8 * h, 4);  // one arrival per softmax warp of the head
+    }
 #pragma unroll
     for (int i = 0; i < STAGES; ++i) {
       mbar_init(bars + B_KFULL + 8 * i, 1);
       mbar_init(bars + B_VFULL + 8 * i, 1);
-      mbar_init(bars + B_KEMPTY + 8 * i, 1);
-      mbar_init(bars + B_VEMPTY + 8 * i, 1);
+      mbar_init(bars + B_KVEMPTY + 8 * i, 1);
     }
     mbar_init(bars + B_OFINAL, 1);
     for (int i = 0; i < S_ITEM_SLOTS; ++i) {
       mbar_init(bars + B_ITEMBAR + 8 * i, 1);                     // record written (producer)
-      mbar_init(bars + B_ITEMBAR + 8 * S_ITEM_SLOTS + 8 * i, 5);  // record read (MMA warp + four softmax warps)
+      mbar_init(bars + B_ITEMBAR + 8 * S_ITEM_SLOTS + 8 * i, 9);  // record read (MMA warp + eight softmax warps)
     }
     asm volatile("st.shared.u32 [%0], %1;" ::"r"(bars + B_GAVE_UP), "r"(0u) : "memory");
     mbar_init_fence();
@@ -269,13 +273,10 @@ attn_tcs_kernel(const __grid_constant__ SProblem prob0, const __grid_constant__ 
         int krem, yrow;
         locate(it, i, krem, yrow);
         const int st = n_kv % STAGES, use = n_kv / STAGES;
-        if (use > 0) mbar_wait(wc, bars + B_KEMPTY + 8 * st, (use - 1) & 1);
+        if (use > 0) mbar_wait(wc, bars + B_KVEMPTY + 8 * st, (use - 1) & 1);
         if (elect_one()) {
           mbar_expect_tx(bars + B_KFULL + 8 * st, KVB);
           tma_load_2d(sK + st * KVB, &tmK, it.c * C::SLW, yrow, bars + B_KFULL + 8 * st);
-        }
-        if (use > 0) mbar_wait(wc, bars + B_VEMPTY + 8 * st, (use - 1) & 1);
-        if (elect_one()) {
           mbar_expect_tx(bars + B_VFULL + 8 * st, KVB);
           tma_load_2d(sV + st * KVB, &tmV, it.c * C::SLW, yrow, bars + B_VFULL + 8 * st);
         }
@@ -284,87 +285,77 @@ attn_tcs_kernel(const __grid_constant__ SProblem prob0, const __grid_constant__ 
   } else if (warp == 1) {
     // ================================ MMA issuer ================================
     constexpr uint32_t IDESC_PV = idesc_bf16(NPV, true);
-    int n_q = 0, n_kv = 0, n_u = 0;  // Q tiles, key tiles and units consumed so far
+    int n_q = 0, n_kv = 0;  // Q tiles and key tiles consumed so far; key tile n is also phase n of the heads' S / P barriers
     for (int k = 0;; ++k) {
-      SItem it;
-      {
-        const int slot = k % S_ITEM_SLOTS;
-        const bool ok = mbar_wait(wc, bars + B_ITEMBAR + 8 * slot, (k / S_ITEM_SLOTS) & 1);
-        it = read_item(bars, slot, lane);
-        if (!ok) it.T = -1;
-      }
+      const SItem it = fetch_item(wc, bars, k, lane);
       if (it.T < 0) break;
       if (it.T == 0) continue;
-      const int U = it.T * G, qb = n_q & 1;
+      const int qb = n_q & 1;
       const uint32_t sQb = sQ + qb * S_QBUF;
       mbar_wait(wc, bars + B_QFULL + 8 * qb, (n_q >> 1) & 1);
-      // Round u: the P V of unit u - 1 (once its weights are in TMEM), then the scores of unit u.  The softmax warps have
-      // finished reading S before they release P, so S may be overwritten then; and tcgen05.mma instructions of one
-      // thread execute in issue order, so P is read by the P V before the softmax of unit u (which waits for the scores
-      // issued after it) writes it again.
+      // Round (j, h): the P V of key tile j - 1 of head h (once its weights are in TMEM), then the scores of key tile j of
+      // head h.  The softmax warps of the head have finished reading S_h before they release P_h, so S_h may be
+      // overwritten then; tcgen05.mma instructions of one thread execute in issue order, so P_h is read by the P V
+      // before the head's next softmax (which waits for the scores issued after it) writes it again.  The other head's
+      // softmax runs meanwhile.
       int krem_prev = 0;
 #pragma unroll 1
-      for (int u = 0; u <= U; ++u) {
-        int krem = 0, st = 0, h = 0, j = 0;
-        if (u < U) {
-          j = u / G; h = u - j * G;
-          const int n = n_kv + j;
-          st = n % STAGES;
+      for (int j = 0; j <= it.T; ++j) {
+        const int n = n_kv + j, st = n % STAGES, pst = (n - 1) % STAGES;
+        int krem = 0;
+        if (j < it.T) {
           int yrow;
           locate(it, j, krem, yrow);
-          if (h == 0) mbar_wait(wc, bars + B_KFULL + 8 * st, (n / STAGES) & 1);
+          mbar_wait(wc, bars + B_KFULL + 8 * st, (n / STAGES) & 1);
         }
-        int pst = 0, ph = 0, pj = 0;
-        if (u > 0) {
-          const int v = u - 1, nu = n_u + v;
-          pj = v / G; ph = v - pj * G;
-          const int n = n_kv + pj;
-          pst = n % STAGES;
-          // P of unit v is in TMEM (and, for the first unit of an item, the previous item's O has been read)
-          mbar_wait(wc, bars + B_PFULL, nu & 1);
-          if (ph == 0) mbar_wait(wc, bars + B_VFULL + 8 * pst, (n / STAGES) & 1);
-        }
-        tc_fence_after();
-        if (elect_one()) {
-          if (u > 0) {
-            const int ksteps = (krem_prev >= SK) ? SK / 16 : (krem_prev + 15) >> 4;
-            const uint32_t vt = sV + pst * KVB;
-            for (int kk = 0; kk < ksteps; ++kk)  // 16 keys per step: two groups of 8 rows of the V tile
-              umma_ts(tmem + S_COL_O + NPV * ph, tmem + S_COL_P + 8 * kk, smem_desc_sw(vt + 2 * C::SBO * kk, C::SBO, C::SWZ),
-                      IDESC_PV, (pj > 0 || kk > 0) ? 1u : 0u);
-            if (ph == G - 1) umma_commit(bars + B_VEMPTY + 8 * pst);  // also: O holds key tiles 0..pj of every head
-            if (u == U) umma_commit(bars + B_OFINAL);
-          }
-          if (u < U) {
-            const int ncols = (krem >= SK) ? SK : ((krem + 15) >> 4) << 4;
-            const uint32_t idesc = idesc_bf16(ncols, false), kt = sK + st * KVB;
-            if constexpr (HD == 8) {
-              // [q_h, 0] for the even head, [0, q_h] for the odd one: start at q_even or at the zeros, 2 KB to the other half
-              umma_ss(tmem, smem_desc_plain(sQb + h * 2048, 2048, 128), smem_desc_sw(kt, C::SBO, C::SWZ), idesc, 0);
-            } else {
+        if (j > 0) mbar_wait(wc, bars + B_VFULL + 8 * pst, ((n - 1) / STAGES) & 1);
+        const int ncols = (krem >= SK) ? SK : ((krem + 15) >> 4) << 4;
+        const int ksteps = (krem_prev >= SK) ? SK / 16 : (krem_prev + 15) >> 4;
 #pragma unroll
-              for (int ks = 0; ks < HD / 16; ++ks)
-                umma_ss(tmem, smem_desc_sw(sQb + 32 * ks, C::SBO, C::SWZ), smem_desc_sw(kt + 32 * ks, C::SBO, C::SWZ), idesc, ks > 0);
+        for (int h = 0; h < 2; ++h) {
+          // P_h of key tile j - 1 is in TMEM (and, for the first tile of an item, the previous item's O_h has been read)
+          if (j > 0) mbar_wait(wc, bars + B_PFULL + 8 * h, (n - 1) & 1);
+          tc_fence_after();
+          if (elect_one()) {
+            if (j > 0) {
+              const uint32_t vt = sV + pst * KVB + ((HD == 8) ? 0 : 2 * HD * h);
+              for (int kk = 0; kk < ksteps; ++kk)  // 16 keys per step: two groups of 8 rows of the V tile
+                umma_ts(tmem + S_COL_O + 32 * h, tmem + S_COL_P + 32 * h + 8 * kk, smem_desc_sw(vt + 2 * C::SBO * kk, C::SBO, C::SWZ),
+                        IDESC_PV, (j > 1 || kk > 0) ? 1u : 0u);
+              if (h == 1) umma_commit(bars + B_KVEMPTY + 8 * pst);  // both tiles of the stage are read
+              if (j == it.T && h == 1) umma_commit(bars + B_OFINAL);
             }
-            if (h == G - 1) umma_commit(bars + B_KEMPTY + 8 * st);
-            if (u == U - 1) umma_commit(bars + B_QEMPTY + 8 * qb);
-            umma_commit(bars + B_SFULL);
+            if (j < it.T) {
+              const uint32_t idesc = idesc_bf16(ncols, false), kt = sK + st * KVB, d = tmem + 64 * h;
+              if constexpr (HD == 8) {
+                // [q_h, 0] for the even head, [0, q_h] for the odd one: start at q_even or at the zeros, 2 KB to the other half
+                umma_ss(d, smem_desc_plain(sQb + h * 2048, 2048, 128), smem_desc_sw(kt, C::SBO, C::SWZ), idesc, 0);
+              } else {
+#pragma unroll
+                for (int ks = 0; ks < HD / 16; ++ks)
+                  umma_ss(d, smem_desc_sw(sQb + 2 * HD * h + 32 * ks, C::SBO, C::SWZ), smem_desc_sw(kt + 2 * HD * h + 32 * ks, C::SBO, C::SWZ),
+                          idesc, ks > 0);
+              }
+              if (j == it.T - 1 && h == 1) umma_commit(bars + B_QEMPTY + 8 * qb);
+              umma_commit(bars + B_SFULL + 8 * h);
+            }
           }
+          __syncwarp();
         }
-        __syncwarp();
         krem_prev = krem;
       }
       n_kv += it.T;
-      n_u += U;
       ++n_q;
     }
   } else {
-    // ================================ softmax, one thread per query row ================================
+    // ================================ softmax: thread = (query row = TMEM lane, head of the pair) ================================
     const int wq = warp & 3;                               // TMEM lane quarter this warp may access
+    const int h = (warp - 2) >> 2;                         // head of the pair this warp group works for
     const int r = (wq << 5) + lane;                        // row in the tile = TMEM lane
     const uint32_t tl = tmem + ((uint32_t)(wq << 5) << 16);
+    const uint32_t tS = tl + 64 * h, tP = tl + S_COL_P + 32 * h, tO = tl + S_COL_O + 32 * h + ((HD == 8) ? 8 * h : 0);
     const float2 sl2v = make_float2(sl2, sl2);
-    int n_kv = 0, n_u = 0, n_items_done = 0;
+    int n_kv = 0, n_items_done = 0;
 
     for (int k = 0;; ++k) {
       const SItem it = fetch_item(wc, bars, k, lane);
@@ -374,33 +365,41 @@ attn_tcs_kernel(const __grid_constant__ SProblem prob0, const __grid_constant__ 
       const int slice = it.c & ((1 << WHICH_SHIFT) - 1);
       __nv_bfloat16* __restrict__ out = prob.out;
       float* __restrict__ lse = prob.lse;
-      uint4* dst = reinterpret_cast<uint4*>(out + grow * g.d + slice * C::SLW);
-      float* lse_row = (lse != nullptr) ? lse + ((int64_t)it.b * g.heads + slice * G) * g.L + g.seg_off[it.s] + it.q0 + r : nullptr;
+      uint4* dst = reinterpret_cast<uint4*>(out + grow * g.d + slice * C::SLW + h * HD);
+      float* lse_row = (lse != nullptr) ? lse + ((int64_t)it.b * g.heads + slice * 2 + h) * g.L + g.seg_off[it.s] + it.q0 + r : nullptr;
       const bool warp_active = (wq << 5) < it.q_real;  // some row of this warp receives a result
       if (it.T == 0 || !warp_active) {
-        // nothing to compute for these rows (padding only, or an empty key set): exact zeros, lse = -inf
+        // nothing to compute for these rows (padding only, or an empty key set): exact zeros, lse = -inf.  A warp without
+        // a real row leaves the item here: the head's first warp (rows 0..31, which always hold a real row when any does)
+        // arrives on the weights barrier for it as well, so it neither polls nor arrives during the key walk.
         if (r < it.rows_in_tile) {
 #pragma unroll
-          for (int c = 0; c < ROWB / 16; ++c) dst[c] = make_uint4(0, 0, 0, 0);
-          if (lse_row != nullptr)
-            for (int h = 0; h < G; ++h) lse_row[(int64_t)h * g.L] = -INFINITY;
+          for (int c = 0; c < HD / 8; ++c) dst[c] = make_uint4(0, 0, 0, 0);
+          if (lse_row != nullptr) *lse_row = -INFINITY;
         }
-        if (it.T == 0) continue;
+        if (it.T > 0) {
+          // ... but it may not run ahead into the next item: a barrier phase is told from the one two phases later only
+          // by the order of events, so every warp stays within one item of the others
+          mbar_wait(wc, bars + B_OFINAL, n_items_done & 1);
+          n_kv += it.T;
+          ++n_items_done;
+        }
+        continue;
       }
-      // running maximum (the one the weights are taken against) and sum, per head of the slice
-      float m0 = -INFINITY, l0 = 0.f, m1 = -INFINITY, l1 = 0.f;
-      const int U = it.T * G;
-      int krem = 0;
+      const uint32_t arrivals = (wq == 0) ? 1u + (uint32_t)(4 - min(4, (it.q_real + 31) >> 5)) : 1u;  // own + the idle warps' 
+      float mu = -INFINITY, lsum = 0.f;  // running maximum (the one the weights are taken against) and sum of this row and head
 #pragma unroll 1
-      for (int u = 0; u < U; ++u) {
-        const int j = u / G, h = u - j * G, n = n_kv + j, nu = n_u + u;
-        if (h == 0) { int yrow; locate(it, j, krem, yrow); }
-        mbar_wait(wc, bars + B_SFULL, nu & 1);
+      for (int j = 0; j < it.T; ++j) {
+        const int n = n_kv + j;
+        int krem, yrow;
+        locate(it, j, krem, yrow);
+        mbar_wait(wc, bars + B_SFULL + 8 * h, n & 1);
         tc_fence_after();
         if (krem < SK && h == 0) {
           // Rows of the V tile past the valid length hold whatever follows in memory; a zero weight times NaN or Inf
           // would still poison the accumulator, so clear them (up to the end of the last 16-key group that is
-          // multiplied) before the first P V of the tile reads them.
+          // multiplied) before the first P V of the tile reads them: the MMA warp issues head 0's product first, after
+          // this group's release of P_0.
           const int st = n % STAGES;
           mbar_wait(wc, bars + B_VFULL + 8 * st, (n / STAGES) & 1);
           const int row = krem + r;
@@ -412,10 +411,9 @@ attn_tcs_kernel(const __grid_constant__ SProblem prob0, const __grid_constant__ 
           fence_async_smem();
         }
         if (warp_active) {
-          // One unit, in four groups of 16 keys; groups without a real key are skipped (the branches are uniform over the
-          // CTA), the group that straddles the valid length is masked element by element.  Two register buffers of 16
-          // scores: a group is requested from TMEM while the one before it is being worked on.
-          float mu = (G == 2 && h == 1) ? m1 : m0, lsum = (G == 2 && h == 1) ? l1 : l0;
+          // One key tile of this head, in four groups of 16 keys; groups without a real key are skipped (the branches are
+          // uniform over the CTA), the group that straddles the valid length is masked element by element.  Two register
+          // buffers of 16 scores: a group is requested from TMEM while the one before it is being worked on.
           uint32_t sa[16], sb[16];
           auto fix = [&](uint32_t (&a)[16], const int c) {  // keys past the valid length get weight exactly zero
             if (krem < 16 * c + 16) {
@@ -433,15 +431,15 @@ attn_tcs_kernel(const __grid_constant__ SProblem prob0, const __grid_constant__ 
             for (int e = 0; e < 16; e += 2)
               mx4[(e >> 1) & 3] = fmax3(mx4[(e >> 1) & 3], __uint_as_float(a[e]), __uint_as_float(a[e + 1]));
           };
-          tmem_ld16(tl + 0, sa);
-          if (16 < krem) tmem_ld16(tl + 16, sb);
+          tmem_ld16(tS + 0, sa);
+          if (16 < krem) tmem_ld16(tS + 16, sb);
           tmem_wait_ld();
           fix(sa, 0);
           maxc(sa);
           if (16 < krem) { fix(sb, 1); maxc(sb); }
           if (32 < krem) {
-            tmem_ld16(tl + 32, sa);
-            if (48 < krem) tmem_ld16(tl + 48, sb);
+            tmem_ld16(tS + 32, sa);
+            if (48 < krem) tmem_ld16(tS + 48, sb);
             tmem_wait_ld();
             fix(sa, 2);
             maxc(sa);
@@ -453,10 +451,8 @@ attn_tcs_kernel(const __grid_constant__ SProblem prob0, const __grid_constant__ 
           if (j > 0 && __any_sync(0xffffffffu, grow_m)) {
             const float alpha = grow_m ? ex2((mu - mx) * sl2) : 1.f;
             lsum *= alpha;
-            // O_h must hold every earlier key tile before it is rescaled: wait for the last P V of key tile n - 1
-            mbar_wait(wc, bars + B_VEMPTY + 8 * ((n - 1) % STAGES), ((n - 1) / STAGES) & 1);
-            tc_fence_after();
-            const uint32_t tO = tl + S_COL_O + NPV * h + ((HD == 8) ? 8 * h : 0);
+            // O_h holds every earlier key tile: the P V of tile j - 1 was issued before the scores this thread has just
+            // waited for, and the tensor pipe runs in issue order
 #pragma unroll
             for (int c = 0; c < HD / 8; ++c) {
               uint32_t o[8];
@@ -482,15 +478,14 @@ attn_tcs_kernel(const __grid_constant__ SProblem prob0, const __grid_constant__ 
               sum[(e >> 1) & 1] = __fadd2_rn(sum[(e >> 1) & 1], p);
               pr[e >> 1] = __byte_perm(__float_as_uint(p.x), __float_as_uint(p.y), 0x7632);  // upper halves: bf16 pair
             }
-            tmem_st8(tl + S_COL_P + 8 * c, pr);
+            tmem_st8(tP + 8 * c, pr);
           };
           if (32 < krem) {
             weights(sa, 2);
-            tmem_ld16(tl + 0, sa);
+            tmem_ld16(tS + 0, sa);
             if (48 < krem) weights(sb, 3);
             tmem_wait_ld();
-            if (16 < krem) tmem_ld16(tl + 16, sb);
-            fix(sa, 0);  // never masks here (the tile has more than 32 keys); kept for symmetry, compiles to nothing taken
+            tmem_ld16(tS + 16, sb);
             weights(sa, 0);
             tmem_wait_ld();
             weights(sb, 1);
@@ -501,45 +496,38 @@ attn_tcs_kernel(const __grid_constant__ SProblem prob0, const __grid_constant__ 
           }
           const float2 s01 = __fadd2_rn(sum[0], sum[1]);
           lsum += s01.x + s01.y;
-          if (G == 2 && h == 1) { m1 = mu; l1 = lsum; } else { m0 = mu; l0 = lsum; }
           tmem_wait_st();
         }
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(bars + B_PFULL);
+        if (lane == 0) mbar_arrive_n(bars + B_PFULL + 8 * h, arrivals);
       }
       n_kv += it.T;
-      n_u += U;
 
-      // ---- epilogue: O_h / l_h -> bf16, each thread its own 32 (64) bytes of the row; padded rows +0 ----
+      // ---- epilogue: O_h / l -> bf16, each thread the 16 (32, 64) bytes of its row and head; padded rows +0 ----
       mbar_wait(wc, bars + B_OFINAL, n_items_done & 1);
       ++n_items_done;
       tc_fence_after();
       if (warp_active) {
         const bool real = r < it.q_real;
-        uint32_t orow[ROWB / 4];
+        const float inv = (lsum > 0.f) ? TRUNC_GAIN / lsum : 0.f;
+        uint32_t orow[HD / 2];
 #pragma unroll
-        for (int h = 0; h < G; ++h) {
-          const float lh = (h == 1) ? l1 : l0, mh = (h == 1) ? m1 : m0;
-          const float inv = (lh > 0.f) ? TRUNC_GAIN / lh : 0.f;
-          const uint32_t tO = tl + S_COL_O + NPV * h + ((HD == 8) ? 8 * h : 0);
+        for (int c = 0; c < HD / 8; ++c) {
+          uint32_t o[8];
+          tmem_ld8(tO + 8 * c, o);
+          tmem_wait_ld();
 #pragma unroll
-          for (int c = 0; c < HD / 8; ++c) {
-            uint32_t o[8];
-            tmem_ld8(tO + 8 * c, o);
-            tmem_wait_ld();
-#pragma unroll
-            for (int e = 0; e < 8; e += 2)
-              orow[(h * HD + c * 8 + e) >> 1] = pack_bf16(__uint_as_float(o[e]) * inv, __uint_as_float(o[e + 1]) * inv);
-          }
-          if (lse_row != nullptr && r < it.rows_in_tile) {
-            const float ln2 = 0.6931471805599453f;
-            lse_row[(int64_t)h * g.L] = (real && lh > 0.f) ? (mh * sl2 + log2f(lh) - TRUNC_LOG2) * ln2 : -INFINITY;
-          }
+          for (int e = 0; e < 8; e += 2)
+            orow[(c * 8 + e) >> 1] = pack_bf16(__uint_as_float(o[e]) * inv, __uint_as_float(o[e + 1]) * inv);
         }
         if (r < it.rows_in_tile) {
+          if (lse_row != nullptr) {
+            const float ln2 = 0.6931471805599453f;
+            *lse_row = (real && lsum > 0.f) ? (mu * sl2 + log2f(lsum) - TRUNC_LOG2) * ln2 : -INFINITY;
+          }
 #pragma unroll
-          for (int c = 0; c < ROWB / 16; ++c)
+          for (int c = 0; c < HD / 8; ++c)
             dst[c] = real ? make_uint4(orow[4 * c], orow[4 * c + 1], orow[4 * c + 2], orow[4 * c + 3]) : make_uint4(0, 0, 0, 0);
         }
       }
@@ -604,8 +592,8 @@ cudaError_t launch_tcs(const Geometry& g, const AttnOperands* ops, int n, int64_
 
 }  // namespace
 
-bool attn_tcs_supported(const Geometry& g) {
-  return (g.hd == 8 || g.hd == 16) ? (g.d % 16 == 0) : (g.hd == 32 && g.d % 32 == 0);
+bool attn_tcs_supported(const Geometry& g) {  // the kernel works on pairs of heads
+  return (g.hd == 8 || g.hd == 16 || g.hd == 32) && g.heads % 2 == 0;
 }
 
 cudaError_t launch_attn_tcs(const Geometry& g, const AttnOperands* ops, int n, int64_t row_stride, float scale, int* next_item,

@@ -99,7 +99,7 @@ __device__ __forceinline__ bool mbar_wait_parked(const WaitCtx& w, uint32_t bar,
 __device__ __forceinline__ bool mbar_wait_sleep(const WaitCtx& w, uint32_t bar, uint32_t parity, unsigned ns, int limit = 1 << 17) {
   for (int it = 0; it < limit; ++it) {
     if (mbar_test(bar, parity)) return true;
-    __nanosleep(ns);
+    if (ns) __nanosleep(ns);
     if ((it & 63) == 63 && cta_gave_up(w)) return false;
   }
   asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(w.gave_up), "r"(1u) : "memory");
@@ -107,6 +107,10 @@ __device__ __forceinline__ bool mbar_wait_sleep(const WaitCtx& w, uint32_t bar, 
   return false;
 }
 
+// Arrival that counts for `count` participants (a warp arriving on behalf of warps that have nothing to contribute).
+__device__ __forceinline__ void mbar_arrive_n(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
 // Bounded wait that spins on non-parking polls: the shortest hand-over latency, at the price of issue slots.
 __device__ __forceinline__ bool mbar_wait_spin(const WaitCtx& w, uint32_t bar, uint32_t parity, int limit = 1 << 22) {
   for (int it = 0; it < limit; ++it) {
