@@ -80,7 +80,7 @@ typedef struct gsit_shape {
    * either: activations are [packed_capacity, d] matrices of real rows, segment s of sample b at rows
    * row_start[3 b + s] .. + valid_len[b][s] - 1.  row_start is a DEVICE int32 array of 3 B + 1 entries written by
    * gsit_plan_rows (entry 3 B = the row after the last one); valid_len must be given.  Accepted by
-   * gsit_im_attention_fwd (bf16, head_dim 8 / 16 / 32) and gsit_im_layer_fwd (bf16, d_model 64 or 128); other
+   * gsit_im_attention_fwd (bf16, every head_dim) and gsit_im_layer_fwd (bf16, d_model 64 or 128); other
    * calls and shapes answer GSIT_ERR_UNSUPPORTED. */
   const int32_t* row_start;
   int32_t packed_capacity;  /* rows of the packed matrices (>= the plan's last entry rounded up to 128) */

@@ -58,6 +58,8 @@ struct Item {
   int q_real;        // rows that receive a computed result; the remaining rows_in_tile - q_real are written as +0
   int T;             // key tiles to walk
   int kn0, kn1, kn2, nk0, nk1;  // real keys per open key segment, key tiles of the first two
+  int kb0, kb1, kb2;            // first row of each key segment in the activation matrices (padded or packed layout)
+  int grow0;                    // first row of the query tile in the activation matrices
 };
 
 __device__ __forceinline__ Item decode_item(const Geometry& g, int w, int tiles_per_sample) {
@@ -74,8 +76,15 @@ __device__ __forceinline__ Item decode_item(const Geometry& g, int w, int tiles_
   }
   it.s = s;
   it.q0 = tile * TQ;
-  it.rows_in_tile = min(TQ, g.seg_len[s] - it.q0);
-  const int q_real_all = max(0, min(it.rows_in_tile, valid_rows(g, it.b, s) - it.q0));
+  const int in_seg = min(TQ, g.seg_len[s] - it.q0);
+  const int q_real_all = max(0, min(in_seg, valid_rows(g, it.b, s) - it.q0));
+  // rows of the tile this CTA writes: in the padded layout all that belong to the segment (padding as +0); in the packed
+  // layout only the real ones exist -- what follows them in memory is another segment
+  it.rows_in_tile = (g.row_start != nullptr) ? q_real_all : in_seg;
+  it.kb0 = seg_row0(g, it.b, 0);
+  it.kb1 = seg_row0(g, it.b, 1);
+  it.kb2 = seg_row0(g, it.b, 2);
+  it.grow0 = seg_row0(g, it.b, s) + it.q0;
   it.kn0 = ((g.allowed >> (3 * s + 0)) & 1u) ? valid_rows(g, it.b, 0) : 0;
   it.kn1 = ((g.allowed >> (3 * s + 1)) & 1u) ? valid_rows(g, it.b, 1) : 0;
   it.kn2 = ((g.allowed >> (3 * s + 2)) & 1u) ? valid_rows(g, it.b, 2) : 0;
@@ -93,7 +102,7 @@ __device__ __forceinline__ void locate(const Geometry& g, const Item& it, int i,
   if (t >= it.nk0) { t -= it.nk0; r = 1; if (t >= it.nk1) { t -= it.nk1; r = 2; } }
   const int kn = (r == 0) ? it.kn0 : (r == 1) ? it.kn1 : it.kn2;
   krem = kn - t * TK;
-  yrow = it.b * g.L + g.seg_off[r] + t * TK;
+  yrow = ((r == 0) ? it.kb0 : (r == 1) ? it.kb1 : it.kb2) + t * TK;
 }
 
 // Producer side: lane 0 writes record k of this CTA, then the slot's "written" barrier is released.
@@ -103,6 +112,7 @@ __device__ __forceinline__ void publish_item(uint32_t base, const Item& it, int 
     asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(it.b), "r"(it.h), "r"(it.s), "r"(it.q0) : "memory");
     asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(a + 16), "r"(it.rows_in_tile), "r"(it.q_real), "r"(it.T), "r"(it.kn0) : "memory");
     asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(a + 32), "r"(it.kn1), "r"(it.kn2), "r"(it.nk0), "r"(it.nk1) : "memory");
+    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(a + 48), "r"(it.kb0), "r"(it.kb1), "r"(it.kb2), "r"(it.grow0) : "memory");
     mbar_arrive(base + OFF_ITEMBAR + 8 * (k % ITEM_SLOTS));
   }
   __syncwarp();
@@ -116,6 +126,7 @@ __device__ __forceinline__ Item fetch_item(const WaitCtx& wc, uint32_t base, int
   asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(it.b), "=r"(it.h), "=r"(it.s), "=r"(it.q0) : "r"(a) : "memory");
   asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(it.rows_in_tile), "=r"(it.q_real), "=r"(it.T), "=r"(it.kn0) : "r"(a + 16) : "memory");
   asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(it.kn1), "=r"(it.kn2), "=r"(it.nk0), "=r"(it.nk1) : "r"(a + 32) : "memory");
+  asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(it.kb0), "=r"(it.kb1), "=r"(it.kb2), "=r"(it.grow0) : "r"(a + 48) : "memory");
   __syncwarp();
   if (lane == 0) mbar_arrive(base + OFF_ITEMBAR + 8 * ITEM_SLOTS + 8 * slot);
   return it;
@@ -177,7 +188,7 @@ attn_tc_hd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         if (quse > 0) mbar_wait(wc, bars + BAR_QEMPTY + 8 * qb, (quse - 1) & 1);
         if (elect_one()) {
           mbar_expect_tx(bars + BAR_QFULL + 8 * qb, Q_BYTES);
-          tma_load_2d(sQ + qb * Q_BYTES, &tmQ, it.h * HD64, it.b * g.L + g.seg_off[it.s] + it.q0, bars + BAR_QFULL + 8 * qb);
+          tma_load_2d(sQ + qb * Q_BYTES, &tmQ, it.h * HD64, it.grow0, bars + BAR_QFULL + 8 * qb);
         }
         ++n_q;
         for (int i = 0; i < it.T; ++i, ++n_kv) {
@@ -259,7 +270,7 @@ attn_tc_hd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     int k = 0;
     for (int w = blockIdx.x; w < n_items; w += gridDim.x, ++k) {
       const Item it = fetch_item(wc, base, k, lane);
-      const int64_t grow = (int64_t)it.b * g.L + g.seg_off[it.s] + it.q0 + r;
+      const int64_t grow = (int64_t)it.grow0 + r;
       uint4* dst = reinterpret_cast<uint4*>(out + grow * g.d + it.h * HD64);
       float* lse_row = (lse != nullptr) ? lse + ((int64_t)it.b * g.heads + it.h) * g.L + g.seg_off[it.s] + it.q0 + r : nullptr;
       if (it.T == 0) {  // nothing to attend (padding rows only, or an empty key set): exact zeros, lse = -inf
@@ -409,7 +420,7 @@ cudaError_t launch_attn_tc_hd64(const Geometry& g, const __nv_bfloat16* q, const
                                 const __nv_bfloat16* v, int64_t row_stride, __nv_bfloat16* out, float* lse,
                                 float scale, cudaStream_t st) {
   if (g.hd != HD64) return cudaErrorNotSupported;
-  const int64_t rows = (int64_t)g.batch * g.L;
+  const int64_t rows = matrix_rows(g);
   alignas(64) CUtensorMap tmQ, tmK, tmV;
   if (!make_map(&tmQ, q, rows, g.d, row_stride, HD64, TQ) || !make_map(&tmK, k, rows, g.d, row_stride, HD64, TK) ||
       !make_map(&tmV, v, rows, g.d, row_stride, HD64, TK))

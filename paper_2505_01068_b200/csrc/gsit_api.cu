@@ -220,7 +220,7 @@ gsit_status gsit_im_attention_fwd(const gsit_shape* shape, const void* q, const 
   if (!q || !k || !v || !out || row_stride < g.d) return GSIT_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return GSIT_ERR_INVALID_ARG;
   if (shape->dtype == GSIT_BF16 && row_stride % 8 != 0) return GSIT_ERR_INVALID_ARG;
-  if (g.row_start != nullptr && (shape->dtype != GSIT_BF16 || g.hd > 32)) return GSIT_ERR_UNSUPPORTED;
+  if (g.row_start != nullptr && shape->dtype != GSIT_BF16) return GSIT_ERR_UNSUPPORTED;  // every bf16 kernel takes the packed layout
   if (from_cuda(status_ptr(&g.status)) != GSIT_OK) return GSIT_ERR_CUDA;
   // optional scratch: with it the bf16 kernels hand out their work items through a counter instead of a fixed assignment
   void* scratch = (workspace != nullptr && workspace_bytes >= sizeof(int) && (reinterpret_cast<uintptr_t>(workspace) & 3u) == 0)

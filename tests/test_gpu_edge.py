@@ -143,6 +143,46 @@ def test_attention_with_and_without_scratch_gives_the_same_bits(g):
     assert g.last_device_status() == (0, 0)
 
 
+@pytest.mark.parametrize("H,hd", [(2, 64), (4, 16), (8, 8), (2, 32)])
+def test_attention_on_packed_rows_equals_padded_layout(g, H, hd):
+    """gsit_im_attention_fwd on the packed row layout (q, k, v and out hold real rows only) against the padded layout, for
+    every bf16 kernel family: the same bits in every real row, and nothing written outside them."""
+    rng = np.random.default_rng(900 + hd)
+    seg, B = (70, 200, 150), 4
+    d = H * hd
+    valid = np.array([[70, 200, 150], [33, 129, 65], [70, 0, 1], [0, 0, 0]], dtype=np.int32)
+    vl = torch.from_numpy(valid).cuda()
+    q, k, v = wk.draw_qkv(rng, B, sum(seg), H, hd, "bf16")
+    qkv = torch.stack([to_dev(a, "bf16") for a in (q, k, v)], dim=2).contiguous()          # [B, L, 3, H, hd]
+    want = g.im_attention_fwd(qkv[:, :, 0], qkv[:, :, 1], qkv[:, :, 2], seg, vl, oracle.PHASE_INTER_FWD)
+    L, cap = sum(seg), B * sum(seg) + 128
+    plan = g.plan_rows(vl, seg)
+    plan_h = plan.cpu().numpy()
+    packed = torch.full((cap, 3 * d), float("nan"), dtype=torch.bfloat16, device="cuda")
+    off = np.cumsum([0] + list(seg))
+    flat = qkv.reshape(B, L, 3 * d)
+    for b in range(B):
+        for s_ in range(3):
+            n = int(valid[b, s_])
+            packed[plan_h[3 * b + s_]:plan_h[3 * b + s_] + n] = flat[b, off[s_]:off[s_] + n]
+    out = torch.full((cap, d), 7.0, dtype=torch.bfloat16, device="cuda")
+    sh = g.make_shape(B, seg, d, H, vl, g.DTYPE_BF16, g.PHASE_INTER_FWD, row_start=plan, capacity=cap)
+    ws = torch.empty(256, dtype=torch.uint8, device="cuda")
+    lib = g.load()
+    es = 2
+    code = lib.gsit_im_attention_fwd(ctypes.byref(sh), packed.data_ptr(), packed.data_ptr() + d * es, packed.data_ptr() + 2 * d * es, 3 * d,
+                                     out.data_ptr(), None, ws.data_ptr(), ws.numel(), None)
+    assert code == 0
+    torch.cuda.synchronize()
+    used = int(plan_h[-1])
+    for b in range(B):
+        for s_ in range(3):
+            n = int(valid[b, s_])
+            assert torch.equal(out[plan_h[3 * b + s_]:plan_h[3 * b + s_] + n], want[b, off[s_]:off[s_] + n]), (b, s_)
+    assert bool((out[used:] == 7.0).all())
+    assert g.last_device_status() == (0, 0)
+
+
 def test_bounded_wait_runs_out_and_is_reported(g):
     """A device-side wait that nothing will ever satisfy gives up after its poll limit: the kernel returns, the status
     word carries the timeout flag exactly once, and the next ordinary call is clean."""
