@@ -43,8 +43,7 @@ cudaError_t launch_one(const Geometry& g, const AttnOperands* ops, int n, int64_
   if ((int64_t)tiles * g.batch * n > 0x7fffffffLL) return cudaErrorNotSupported;
   const dim3 grid((unsigned)(tiles * g.batch * n), (unsigned)(g.d / CW), 1u);
   const float sl2 = scale * 1.4426950408889634f;
-  attn_bf16_kernel<C><<<grid, NTHREADS, C::SMEM, st>>>(pr[0], pr[1], g, sl2, n);
-  return cudaGetLastError();
+  return launch_overlapped(attn_bf16_kernel<C>, grid, dim3(NTHREADS), C::SMEM, st, pr[0], pr[1], g, sl2, n);
 }
 
 }  // namespace
@@ -52,7 +51,7 @@ cudaError_t launch_one(const Geometry& g, const AttnOperands* ops, int n, int64_
 int g_attn_variant = 0;  // gsit_kernel_choice, or 1..7 = alternative tile configurations of the mma.sync attention
 
 cudaError_t launch_attn_bf16_n(const Geometry& g, const AttnOperands* ops, int n, int64_t row_stride, float scale, int* next_item,
-                               cudaStream_t st) {
+                               cudaStream_t st, bool counter_cleared) {
   if (n < 1 || n > 2) return cudaErrorInvalidValue;
   if (g.batch > 65535 || g.d % 16 != 0) return cudaErrorNotSupported;
   const int cw = (g.d % 64 == 0) ? 64 : (g.d % 32 == 0) ? 32 : 16;
@@ -71,7 +70,7 @@ cudaError_t launch_attn_bf16_n(const Geometry& g, const AttnOperands* ops, int n
   // mma.sync kernel below (61 against 46 us at the MOSEI cross shape: a tcgen05 hand-over per 64 keys of one head costs
   // more than the 8192 exponentials it feeds), so there it is selected by the knob only.
   if (attn_tcs_supported(g) && (var == GSIT_ATTN_TMEM || (var == 0 && g.hd >= 16)))
-    return launch_attn_tcs(g, ops, n, row_stride, scale, next_item, st);
+    return launch_attn_tcs(g, ops, n, row_stride, scale, next_item, st, counter_cleared);
 #define GSIT_CASE(VAR_, HD_, CW_, R_, KS_, MB_)         \
   if (g.hd == HD_ && cw == CW_ && (var == VAR_ || VAR_ == 0)) \
     return launch_one<Cfg<HD_, CW_, R_, KS_, MB_>>(g, ops, n, row_stride, scale, st);
@@ -90,9 +89,10 @@ cudaError_t launch_attn_bf16_n(const Geometry& g, const AttnOperands* ops, int n
 }
 
 cudaError_t launch_attn_bf16(const Geometry& g, const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
-                             int64_t row_stride, __nv_bfloat16* out, float* lse, float scale, int* next_item, cudaStream_t st) {
+                             int64_t row_stride, __nv_bfloat16* out, float* lse, float scale, int* next_item, cudaStream_t st,
+                             bool counter_cleared) {
   const AttnOperands op = {q, k, v, out, lse, g.allowed};
-  return launch_attn_bf16_n(g, &op, 1, row_stride, scale, next_item, st);
+  return launch_attn_bf16_n(g, &op, 1, row_stride, scale, next_item, st, counter_cleared);
 }
 
 }  // namespace gsit

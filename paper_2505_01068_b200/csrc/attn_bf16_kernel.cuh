@@ -53,6 +53,8 @@ attn_bf16_kernel(const __grid_constant__ AttnProblem prob0, const __grid_constan
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int head_in_slice = warp % G, sg = warp / G;
+  grid_dep_wait();  // q, k, v come from the kernel before this one
+  grid_dep_launch();
   const int cb = head_in_slice * (HD / 8);  // first 16-byte chunk of this warp's head inside a tile row
 
   // ---- which tile of which block row.  blockIdx.x = (tile in cost order) * batch + sample: the query segments with

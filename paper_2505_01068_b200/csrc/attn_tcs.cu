@@ -228,6 +228,8 @@ attn_tcs_kernel(const __grid_constant__ SProblem prob0, const __grid_constant__ 
   tc_fence_after();
   uint32_t tmem;
   asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tmem) : "r"(bars + B_TMEM_SLOT) : "memory");
+  grid_dep_wait();
+  grid_dep_launch();
 
   if (warp == 0) {
     // ================================ scheduler and TMA producer ================================
@@ -545,7 +547,7 @@ attn_tcs_kernel(const __grid_constant__ SProblem prob0, const __grid_constant__ 
 
 template <int HD>
 cudaError_t launch_tcs(const Geometry& g, const AttnOperands* ops, int n, int64_t row_stride, float scale, int* next_item,
-                       cudaStream_t st) {
+                       cudaStream_t st, bool counter_cleared) {
   using C = SCfg<HD>;
   const int64_t rows = matrix_rows(g);
   alignas(64) SProblem pr[2];
@@ -581,13 +583,12 @@ cudaError_t launch_tcs(const Geometry& g, const AttnOperands* ops, int n, int64_
   if (n_items > 0x3fffffffLL || slices >= (1 << WHICH_SHIFT)) return cudaErrorNotSupported;
   const int64_t resident = (int64_t)S_CTAS_PER_SM * n_sm;
   const unsigned grid = (unsigned)((n_items < resident) ? n_items : resident);
-  if (next_item != nullptr) {
+  if (next_item != nullptr && !counter_cleared) {
     e = cudaMemsetAsync(next_item, 0, sizeof(int), st);
     if (e != cudaSuccess) return e;
   }
-  attn_tcs_kernel<HD><<<grid, S_THREADS, C::SMEM, st>>>(pr[0], pr[1], g, scale * 1.4426950408889634f, slices, (int)n_items, n,
-                                                         next_item);
-  return cudaGetLastError();
+  return launch_overlapped(attn_tcs_kernel<HD>, dim3(grid), dim3(S_THREADS), C::SMEM, st, pr[0], pr[1], g,
+                           scale * 1.4426950408889634f, slices, (int)n_items, n, next_item);
 }
 
 }  // namespace
@@ -597,11 +598,11 @@ bool attn_tcs_supported(const Geometry& g) {  // the kernel works on pairs of he
 }
 
 cudaError_t launch_attn_tcs(const Geometry& g, const AttnOperands* ops, int n, int64_t row_stride, float scale, int* next_item,
-                            cudaStream_t st) {
+                            cudaStream_t st, bool counter_cleared) {
   if (!attn_tcs_supported(g) || n < 1 || n > 2) return cudaErrorNotSupported;
-  if (g.hd == 8) return launch_tcs<8>(g, ops, n, row_stride, scale, next_item, st);
-  if (g.hd == 16) return launch_tcs<16>(g, ops, n, row_stride, scale, next_item, st);
-  return launch_tcs<32>(g, ops, n, row_stride, scale, next_item, st);
+  if (g.hd == 8) return launch_tcs<8>(g, ops, n, row_stride, scale, next_item, st, counter_cleared);
+  if (g.hd == 16) return launch_tcs<16>(g, ops, n, row_stride, scale, next_item, st, counter_cleared);
+  return launch_tcs<32>(g, ops, n, row_stride, scale, next_item, st, counter_cleared);
 }
 
 }  // namespace gsit

@@ -89,6 +89,23 @@ inline cudaError_t sm_count_and_smem_once(const void* func, int smem_bytes, int*
   return cudaSuccess;
 }
 
+// Launches `kernel` so that it may begin before the previous kernel of the stream has ended (programmatic dependent
+// launch); the kernel itself waits for its predecessor with ptx::grid_dep_wait() before it touches dependent memory.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // ---- host-side launch entry points of the kernel files (all asynchronous on `st`) ----
 // Each returns cudaSuccess or the launch error.
 
@@ -104,11 +121,11 @@ struct AttnOperands {
   uint32_t allowed;
 };
 cudaError_t launch_attn_bf16_n(const Geometry& g, const AttnOperands* ops, int n, int64_t row_stride, float scale, int* next_item,
-                               cudaStream_t st);
+                               cudaStream_t st, bool counter_cleared = false);
 // bf16 attention, mma.sync tiles fed by TMA (attn_bf16.cu); returns cudaErrorNotSupported for shapes it lacks
 cudaError_t launch_attn_bf16(const Geometry& g, const __nv_bfloat16* q, const __nv_bfloat16* k,
                              const __nv_bfloat16* v, int64_t row_stride, __nv_bfloat16* out, float* lse,
-                             float scale, int* next_item, cudaStream_t st);
+                             float scale, int* next_item, cudaStream_t st, bool counter_cleared = false);
 
 // bf16 attention for head_dim 64 on tcgen05 tensor cores with TMEM accumulators (attn_tc.cu)
 cudaError_t launch_attn_tc_hd64(const Geometry& g, const __nv_bfloat16* q, const __nv_bfloat16* k,
@@ -116,11 +133,11 @@ cudaError_t launch_attn_tc_hd64(const Geometry& g, const __nv_bfloat16* q, const
                                 float scale, cudaStream_t st);
 
 // bf16 attention for head_dim 8 / 16 / 32 on tcgen05 with thread-per-row softmax (attn_tcs.cu).  next_item: a device int
-// the call may use as its work counter (it is cleared on the stream before the launch), or nullptr for a fixed
-// assignment of work items to CTAs.
+// the call may use as its work counter (cleared on the stream before the launch unless `counter_cleared` says that the
+// kernel before this one in the stream has done so), or nullptr for a fixed assignment of work items to CTAs.
 bool attn_tcs_supported(const Geometry& g);
 cudaError_t launch_attn_tcs(const Geometry& g, const AttnOperands* ops, int n, int64_t row_stride, float scale, int* next_item,
-                            cudaStream_t st);
+                            cudaStream_t st, bool counter_cleared = false);
 
 // Linear layers  C = act(A W^T + bias) (+ residual), rows that are padding written as zero when
 // `mask_rows` is set.  A [M,K] (lda), W [N,K], C [M,N] (ldc), residual float [M,N] (ldr) or nullptr.
@@ -152,10 +169,11 @@ cudaError_t launch_proj_mlp_bf16(const Geometry& g, const __nv_bfloat16* att, co
                                  const __nv_bfloat16* w_1, const float* b_1, const __nv_bfloat16* w_2, const float* b_2,
                                  int d_ff, float* y, int64_t ldy, cudaStream_t st);
 
-// The same two halves at d_model 64 (d_ff <= 256) on tcgen05 tensor cores with TMEM accumulators (fused_layer_tc.cu)
+// The same two halves at d_model 64 (d_ff <= 256) on tcgen05 tensor cores with TMEM accumulators (fused_layer_tc.cu).
+// zero_word: a device int the first half clears (the work counter of the attention kernel that follows), or nullptr.
 bool fused_layer_tc_supported(const Geometry& g, int d_ff);
 cudaError_t launch_ln_qkv_tc(const Geometry& g, const float* x, int64_t ldx, const float* gamma, const float* beta, float eps,
-                             const __nv_bfloat16* w_qkv, const float* b_qkv, __nv_bfloat16* qkv, cudaStream_t st);
+                             const __nv_bfloat16* w_qkv, const float* b_qkv, __nv_bfloat16* qkv, int* zero_word, cudaStream_t st);
 cudaError_t launch_proj_mlp_tc(const Geometry& g, const __nv_bfloat16* att, const float* x, int64_t ldx,
                                const __nv_bfloat16* w_o, const float* b_o, const float* gamma, const float* beta, float eps,
                                const __nv_bfloat16* w_1, const float* b_1, const __nv_bfloat16* w_2, const float* b_2, int d_ff,
@@ -174,13 +192,13 @@ struct FusedHalfArgs {
   const __nv_bfloat16* w_2; const float* b_2;
   float* y; int64_t ldy;
 };
-cudaError_t launch_ln_qkv_tc_pair(const Geometry& g, const FusedHalfArgs (&h)[2], float eps, cudaStream_t st);
+cudaError_t launch_ln_qkv_tc_pair(const Geometry& g, const FusedHalfArgs (&h)[2], float eps, int* zero_word, cudaStream_t st);
 cudaError_t launch_proj_mlp_tc_pair(const Geometry& g, const FusedHalfArgs (&h)[2], float eps, int d_ff, cudaStream_t st);
 
 // ... and at d_model 128 (d_ff <= 512), with the MLP weights streamed in chunks (fused_layer_tc128.cu)
 bool fused_layer_tc128_supported(const Geometry& g, int d_ff);
 cudaError_t launch_ln_qkv_tc128(const Geometry& g, const float* x, int64_t ldx, const float* gamma, const float* beta, float eps,
-                                const __nv_bfloat16* w_qkv, const float* b_qkv, __nv_bfloat16* qkv, cudaStream_t st);
+                                const __nv_bfloat16* w_qkv, const float* b_qkv, __nv_bfloat16* qkv, int* zero_word, cudaStream_t st);
 cudaError_t launch_proj_mlp_tc128(const Geometry& g, const __nv_bfloat16* att, const float* x, int64_t ldx,
                                   const __nv_bfloat16* w_o, const float* b_o, const float* gamma, const float* beta, float eps,
                                   const __nv_bfloat16* w_1, const float* b_1, const __nv_bfloat16* w_2, const float* b_2, int d_ff,

@@ -3,9 +3,9 @@
 //   ln_qkv_tc_kernel     qkv = LN1(x) W_qkv^T + b_qkv          (the shared projection of the concatenated sequence)
 //   proj_mlp_tc_kernel   y1 = x + att W_o^T + b_o ;  y = y1 + relu(LN2(y1) W_1^T + b_1) W_2^T + b_2   (d_ff <= 256)
 //
-// Persistent, one CTA per SM, tiles of 128 sequence rows, six warps:
+// Persistent (the first half two CTAs per SM, the second one), tiles of 128 sequence rows, six warps:
 //   warp 0      producer: weights once (TMA, 128-byte swizzle, resident for the whole kernel), then per tile the x rows
-//               (per-row bulk copies into padded float rows) and the attention tile (TMA)
+//               (TMA, two boxes of 32 floats) and the attention tile (TMA)
 //   warp 1      owns 512 TMEM columns and issues every tcgen05.mma (M 128, K 16, operands from shared memory)
 //   warps 2..5  thread = sequence row = TMEM lane.  LayerNorm needs no shuffles: a thread holds its whole row.  Rows
 //               are written back to shared memory as bf16 in the 128-byte swizzle the MMA expects (the A operand of the
@@ -66,14 +66,15 @@ __device__ __forceinline__ void layernorm_row_to_tile(const float (&v)[TD], bool
 namespace qk {
 constexpr int NQ = 3 * TD;                       // 192 output columns
 constexpr int OFF_W = 0;                         // W_qkv: 192 rows x 128 B, swizzled
-constexpr int OFF_H = OFF_W + NQ * 128;          // normalised rows (A operand)
-constexpr int OFF_OUT = OFF_H + TM * 128;        // 3 boxes of 64 columns x 128 rows
-constexpr int OFF_X = OFF_OUT + 3 * TM * 128;    // 2 float input tiles (2 boxes each)
-constexpr int OFF_P = OFF_X + 2 * 2 * XBOX;      // gamma[64], beta[64], bias[192] as floats
+constexpr int OFF_OUT = OFF_W + NQ * 128;        // 3 boxes of 64 columns x 128 rows
+constexpr int OFF_H = OFF_OUT;                   // normalised rows (A operand): the first box, free while the MMA runs
+constexpr int OFF_X = OFF_OUT + 3 * TM * 128;    // one float input tile (2 boxes), refilled as soon as it is in registers
+constexpr int OFF_P = OFF_X + 2 * XBOX;          // gamma[64], beta[64], bias[192] as floats
 constexpr int OFF_BAR = OFF_P + (2 * TD + NQ) * 4;
 constexpr int B_W = 0, B_XFULL = 8, B_XFREE = 24, B_HREADY = 40, B_ACCFULL = 48, B_ACCFREE = 56, SLOT = 64;
 constexpr int SMEM = OFF_BAR + 80 + 1024;
 constexpr int TMEM_COLS = 256;
+static_assert(2 * (SMEM + 1024) <= 227 * 1024, "two CTAs per SM");
 }  // namespace qk
 
 // Per-problem arguments of the LN1 + QKV kernel.  One launch can serve two problems of the same geometry (the forward-
@@ -84,9 +85,9 @@ struct LnQkvArgs {
   const float *gamma, *beta, *bias;
 };
 
-__global__ void __launch_bounds__(T_THREADS, 1)
+__global__ void __launch_bounds__(T_THREADS, 2)
 ln_qkv_tc_kernel(const __grid_constant__ LnQkvArgs arg0, const __grid_constant__ LnQkvArgs arg1, const Geometry g,
-                 const float eps, const int problems) {
+                 const float eps, const int problems, int* const zero_word) {
   using namespace qk;
   const int which = (problems == 2) ? (int)(blockIdx.x & 1u) : 0;
   const int cta = (problems == 2) ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;       // index among the CTAs of this problem
@@ -100,8 +101,6 @@ ln_qkv_tc_kernel(const __grid_constant__ LnQkvArgs arg0, const __grid_constant__
   const uint32_t bars = base + OFF_BAR;
   const WaitCtx wc{g.status, bars + SLOT + 4};
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int row_base = rows_begin(g), rows = rows_end(g);  // this problem's rows of the activation matrices
-  const int ntiles = (rows - row_base + TM - 1) / TM;
 
   float* prm = reinterpret_cast<float*>(base_ptr + OFF_P);
   stage_vector(prm, gamma, TD, 1.f, tid, T_THREADS);
@@ -110,7 +109,8 @@ ln_qkv_tc_kernel(const __grid_constant__ LnQkvArgs arg0, const __grid_constant__
   if (tid == 0) {
     asm volatile("st.shared.u32 [%0], %1;" ::"r"(bars + SLOT + 4), "r"(0u) : "memory");
     mbar_init(bars + B_W, 1);
-    for (int i = 0; i < 2; ++i) { mbar_init(bars + B_XFULL + 8 * i, 1); mbar_init(bars + B_XFREE + 8 * i, 4); }
+    mbar_init(bars + B_XFULL, 1);
+    mbar_init(bars + B_XFREE, 4);
     mbar_init(bars + B_HREADY, 4);
     mbar_init(bars + B_ACCFULL, 1);
     mbar_init(bars + B_ACCFREE, 4);
@@ -126,22 +126,28 @@ ln_qkv_tc_kernel(const __grid_constant__ LnQkvArgs arg0, const __grid_constant__
   tc_fence_after();
   uint32_t tmem;
   asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tmem) : "r"(bars + SLOT) : "memory");
-
-  if (warp == 0) {
-    // ================================ producer ================================
+  if (warp == 0) {  // the weights do not depend on the kernel before this one
     if (elect_one()) {
       mbar_expect_tx(bars + B_W, NQ * 128);
       tma_load_2d(base + OFF_W, &tmW, 0, 0, bars + B_W);
     }
     __syncwarp();
+  }
+  grid_dep_wait();
+  grid_dep_launch();
+  const int row_base = rows_begin(g), rows = rows_end(g);  // this problem's rows of the activation matrices
+  const int ntiles = (rows - row_base + TM - 1) / TM;
+  if (zero_word != nullptr && blockIdx.x == 0 && tid == 0) *zero_word = 0;  // work counter of the attention kernel that follows
+
+  if (warp == 0) {
+    // ================================ producer ================================
     int i = 0;
     for (int t = cta; t < ntiles; t += ctas, ++i) {
-      const int xb = i & 1;
-      if (i >= 2) mbar_wait(wc, bars + B_XFREE + 8 * xb, ((i >> 1) - 1) & 1);  // the row warps hold that tile in registers
+      if (i >= 1) mbar_wait(wc, bars + B_XFREE, (i - 1) & 1);  // the row warps hold the previous tile in registers
       if (elect_one()) {
-        mbar_expect_tx(bars + B_XFULL + 8 * xb, 2 * XBOX);
-        tma_load_2d(base + OFF_X + xb * 2 * XBOX, &tmX, 0, row_base + t * TM, bars + B_XFULL + 8 * xb);
-        tma_load_2d(base + OFF_X + xb * 2 * XBOX + XBOX, &tmX, 32, row_base + t * TM, bars + B_XFULL + 8 * xb);
+        mbar_expect_tx(bars + B_XFULL, 2 * XBOX);
+        tma_load_2d(base + OFF_X, &tmX, 0, row_base + t * TM, bars + B_XFULL);
+        tma_load_2d(base + OFF_X + XBOX, &tmX, 32, row_base + t * TM, bars + B_XFULL);
       }
       __syncwarp();
     }
@@ -170,30 +176,29 @@ ln_qkv_tc_kernel(const __grid_constant__ LnQkvArgs arg0, const __grid_constant__
     int i = 0;
     bool real = row_real32(g, row_base + cta * TM + r, rows);
     for (int t = cta; t < ntiles; t += ctas, ++i) {
-      const int row0 = row_base + t * TM, xb = i & 1;
-      mbar_wait(wc, bars + B_XFULL + 8 * xb, (i >> 1) & 1);
+      const int row0 = row_base + t * TM;
+      mbar_wait(wc, bars + B_XFULL, i & 1);
       float v[TD];
       if (real) {
-        load_row64(base + OFF_X + xb * 2 * XBOX, r, v);
+        load_row64(base + OFF_X, r, v);
       } else {  // padded input rows may hold anything (NaN included): never read them
 #pragma unroll
         for (int e = 0; e < TD; ++e) v[e] = 0.f;
       }
       __syncwarp();
-      if (lane == 0) mbar_arrive(bars + B_XFREE + 8 * xb);
-      // the MMA of the previous tile finished reading the normalised rows before its accumulator was handed over
+      if (lane == 0) mbar_arrive(bars + B_XFREE);
+      if (i > 0) {  // the previous tile's stores must have finished reading the staging rows (the normalised rows overlay them)
+        if (tid == 64) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        t_bar_rows();
+      }
       layernorm_row_to_tile(v, real, s_gamma, s_beta, eps, base + OFF_H, r);
       fence_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(bars + B_HREADY);
       const bool real_next = row_real32(g, row_base + (t + ctas) * TM + r, rows);  // overlaps the MMA
 
-      mbar_wait(wc, bars + B_ACCFULL, i & 1);
+      mbar_wait(wc, bars + B_ACCFULL, i & 1);  // the MMA has also finished reading the normalised rows
       tc_fence_after();
-      if (i > 0) {  // the previous tile's stores must have finished reading the staging rows
-        if (tid == 64) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-        t_bar_rows();
-      }
 #pragma unroll 1
       for (int c0 = 0; c0 < NQ; c0 += 32) {
         uint32_t a[32];
@@ -277,8 +282,6 @@ proj_mlp_tc_kernel(const __grid_constant__ ProjMlpArgs arg0, const __grid_consta
   const uint32_t bars = base + OFF_BAR;
   const WaitCtx wc{g.status, bars + SLOT + 4};
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int row_base = rows_begin(g), rows = rows_end(g);  // this problem's rows of the activation matrices
-  const int ntiles = (rows - row_base + TM - 1) / TM;
   const int nh = d_ff / 64;  // k-blocks of hidden units
 
   float* prm = reinterpret_cast<float*>(base_ptr + OFF_P);
@@ -310,9 +313,7 @@ proj_mlp_tc_kernel(const __grid_constant__ ProjMlpArgs arg0, const __grid_consta
   tc_fence_after();
   uint32_t tmem;
   asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tmem) : "r"(bars + SLOT) : "memory");
-
-  if (warp == 0) {
-    // ================================ producer ================================
+  if (warp == 0) {  // the weights do not depend on the kernel before this one
     if (elect_one()) {
       mbar_expect_tx(bars + B_W, (uint32_t)(TD * 128 + d_ff * 128 + nh * TD * 128));
       tma_load_2d(base + OFF_WO, &tmWo, 0, 0, bars + B_W);
@@ -320,6 +321,14 @@ proj_mlp_tc_kernel(const __grid_constant__ ProjMlpArgs arg0, const __grid_consta
       for (int kb = 0; kb < nh; ++kb) tma_load_2d(base + OFF_W2 + kb * TD * 128, &tmW2, 64 * kb, 0, bars + B_W);
     }
     __syncwarp();
+  }
+  grid_dep_wait();
+  grid_dep_launch();
+  const int row_base = rows_begin(g), rows = rows_end(g);  // this problem's rows of the activation matrices
+  const int ntiles = (rows - row_base + TM - 1) / TM;
+
+  if (warp == 0) {
+    // ================================ producer ================================
     int i = 0;
     for (int t = cta; t < ntiles; t += ctas, ++i) {
       const int row0 = row_base + t * TM;
@@ -517,7 +526,7 @@ bool fill_proj_mlp(ProjMlpArgs* a, int64_t rows, const __nv_bfloat16* att, const
 }  // namespace
 
 cudaError_t launch_ln_qkv_tc(const Geometry& g, const float* x, int64_t ldx, const float* gamma, const float* beta, float eps,
-                             const __nv_bfloat16* w_qkv, const float* b_qkv, __nv_bfloat16* qkv, cudaStream_t st) {
+                             const __nv_bfloat16* w_qkv, const float* b_qkv, __nv_bfloat16* qkv, int* zero_word, cudaStream_t st) {
   if (g.d != TD) return cudaErrorNotSupported;
   const int64_t rows = matrix_rows(g);  // bounds of the tensor maps; the kernel takes its own row range from the geometry
   const int ntiles = (int)((rows + TM - 1) / TM), nsm = t_sm_count();
@@ -526,8 +535,7 @@ cudaError_t launch_ln_qkv_tc(const Geometry& g, const float* x, int64_t ldx, con
   if (!fill_ln_qkv(&a, rows, x, ldx, gamma, beta, w_qkv, b_qkv, qkv)) return cudaErrorInvalidValue;
   cudaError_t e = sm_count_and_smem_once(reinterpret_cast<const void*>(ln_qkv_tc_kernel), qk::SMEM, nullptr);
   if (e != cudaSuccess) return e;
-  ln_qkv_tc_kernel<<<min(ntiles, nsm), T_THREADS, qk::SMEM, st>>>(a, a, g, eps, 1);
-  return cudaGetLastError();
+  return launch_overlapped(ln_qkv_tc_kernel, dim3(min(ntiles, 2 * nsm)), dim3(T_THREADS), qk::SMEM, st, a, a, g, eps, 1, zero_word);
 }
 
 cudaError_t launch_proj_mlp_tc(const Geometry& g, const __nv_bfloat16* att, const float* x, int64_t ldx,
@@ -542,14 +550,13 @@ cudaError_t launch_proj_mlp_tc(const Geometry& g, const __nv_bfloat16* att, cons
   if (!fill_proj_mlp(&a, rows, att, x, ldx, w_o, b_o, gamma, beta, w_1, b_1, w_2, b_2, d_ff, y, ldy)) return cudaErrorInvalidValue;
   cudaError_t e = sm_count_and_smem_once(reinterpret_cast<const void*>(proj_mlp_tc_kernel), pm::SMEM, nullptr);
   if (e != cudaSuccess) return e;
-  proj_mlp_tc_kernel<<<min(ntiles, nsm), T_THREADS, pm::SMEM, st>>>(a, a, g, eps, d_ff, 1);
-  return cudaGetLastError();
+  return launch_overlapped(proj_mlp_tc_kernel, dim3(min(ntiles, nsm)), dim3(T_THREADS), pm::SMEM, st, a, a, g, eps, d_ff, 1);
 }
 
 // The same two halves for a PAIR of problems of one geometry in one launch each (the two ring encoders' layers of equal
 // depth): CTAs alternate between the problems, so each problem has half the SMs for the whole launch and one tail is paid
 // instead of two.
-cudaError_t launch_ln_qkv_tc_pair(const Geometry& g, const FusedHalfArgs (&h)[2], float eps, cudaStream_t st) {
+cudaError_t launch_ln_qkv_tc_pair(const Geometry& g, const FusedHalfArgs (&h)[2], float eps, int* zero_word, cudaStream_t st) {
   if (g.d != TD) return cudaErrorNotSupported;
   const int64_t rows = matrix_rows(g);
   const int ntiles = (int)((rows + TM - 1) / TM), nsm = t_sm_count();
@@ -560,8 +567,7 @@ cudaError_t launch_ln_qkv_tc_pair(const Geometry& g, const FusedHalfArgs (&h)[2]
       return cudaErrorInvalidValue;
   cudaError_t e = sm_count_and_smem_once(reinterpret_cast<const void*>(ln_qkv_tc_kernel), qk::SMEM, nullptr);
   if (e != cudaSuccess) return e;
-  ln_qkv_tc_kernel<<<min(2 * ntiles, nsm & ~1), T_THREADS, qk::SMEM, st>>>(a[0], a[1], g, eps, 2);
-  return cudaGetLastError();
+  return launch_overlapped(ln_qkv_tc_kernel, dim3(min(2 * ntiles, 2 * nsm)), dim3(T_THREADS), qk::SMEM, st, a[0], a[1], g, eps, 2, zero_word);
 }
 
 cudaError_t launch_proj_mlp_tc_pair(const Geometry& g, const FusedHalfArgs (&h)[2], float eps, int d_ff, cudaStream_t st) {
@@ -576,8 +582,7 @@ cudaError_t launch_proj_mlp_tc_pair(const Geometry& g, const FusedHalfArgs (&h)[
       return cudaErrorInvalidValue;
   cudaError_t e = sm_count_and_smem_once(reinterpret_cast<const void*>(proj_mlp_tc_kernel), pm::SMEM, nullptr);
   if (e != cudaSuccess) return e;
-  proj_mlp_tc_kernel<<<min(2 * ntiles, nsm & ~1), T_THREADS, pm::SMEM, st>>>(a[0], a[1], g, eps, d_ff, 2);
-  return cudaGetLastError();
+  return launch_overlapped(proj_mlp_tc_kernel, dim3(min(2 * ntiles, nsm & ~1)), dim3(T_THREADS), pm::SMEM, st, a[0], a[1], g, eps, d_ff, 2);
 }
 
 }  // namespace gsit

@@ -71,7 +71,7 @@ static_assert(SMEM <= 227 * 1024, "shared memory budget");
 __global__ void __launch_bounds__(T_THREADS, 1)
 ln_qkv_tc128_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
                     const __grid_constant__ CUtensorMap tmOut, const Geometry g, const float* __restrict__ gamma,
-                    const float* __restrict__ beta, const float eps, const float* __restrict__ bias) {
+                    const float* __restrict__ beta, const float eps, const float* __restrict__ bias, int* const zero_word) {
   using namespace qk2;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -79,8 +79,6 @@ ln_qkv_tc128_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   const uint32_t bars = base + OFF_BAR;
   const WaitCtx wc{g.status, bars + SLOT + 4};
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int row_base = rows_begin(g), rows = rows_end(g);  // this problem's rows of the activation matrices
-  const int ntiles = (rows - row_base + TM - 1) / TM;
 
   float* prm = reinterpret_cast<float*>(base_ptr + OFF_P);
   stage_vector(prm, gamma, D2, 1.f, tid, T_THREADS);
@@ -106,9 +104,7 @@ ln_qkv_tc128_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   tc_fence_after();
   uint32_t tmem;
   asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tmem) : "r"(bars + SLOT) : "memory");
-
-  if (warp == 0) {
-    // ================================ producer ================================
+  if (warp == 0) {  // the weights do not depend on the kernel before this one
     if (elect_one()) {
       mbar_expect_tx(bars + B_W, 2 * NQ * 128);
       for (int kb = 0; kb < 2; ++kb)
@@ -116,6 +112,15 @@ ln_qkv_tc128_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
           tma_load_2d(base + OFF_W + kb * NQ * 128 + j * XBOX, &tmW, 64 * kb, 128 * j, bars + B_W);
     }
     __syncwarp();
+  }
+  grid_dep_wait();
+  grid_dep_launch();
+  const int row_base = rows_begin(g), rows = rows_end(g);  // this problem's rows of the activation matrices
+  const int ntiles = (rows - row_base + TM - 1) / TM;
+  if (zero_word != nullptr && blockIdx.x == 0 && tid == 0) *zero_word = 0;  // work counter of the attention kernel that follows
+
+  if (warp == 0) {
+    // ================================ producer ================================
     int i = 0;
     for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
       // the tile buffer also held the previous tile's normalised rows: wait until the MMA has consumed them
@@ -261,8 +266,6 @@ proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_co
   const uint32_t bars = base + OFF_BAR;
   const WaitCtx wc{g.status, bars + SLOT + 4};
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int row_base = rows_begin(g), rows = rows_end(g);  // this problem's rows of the activation matrices
-  const int ntiles = (rows - row_base + TM - 1) / TM;
   const int nc = d_ff / 64;  // chunks of 64 hidden units
 
   float* prm = reinterpret_cast<float*>(base_ptr + OFF_P);
@@ -300,14 +303,20 @@ proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_co
   tc_fence_after();
   uint32_t tmem;
   asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tmem) : "r"(bars + SLOT) : "memory");
-
-  if (warp == 0) {
-    // ================================ producer ================================
+  if (warp == 0) {  // the weights do not depend on the kernel before this one
     if (elect_one()) {
       mbar_expect_tx(bars + B_WO, 2 * XBOX);
       for (int kb = 0; kb < 2; ++kb) tma_load_2d(base + OFF_WO + kb * XBOX, &tmWo, 64 * kb, 0, bars + B_WO);
     }
     __syncwarp();
+  }
+  grid_dep_wait();
+  grid_dep_launch();
+  const int row_base = rows_begin(g), rows = rows_end(g);  // this problem's rows of the activation matrices
+  const int ntiles = (rows - row_base + TM - 1) / TM;
+
+  if (warp == 0) {
+    // ================================ producer ================================
     int i = 0, n = 0;  // tiles, weight chunks requested so far
     for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
       const int row0 = row_base + t * TM;
@@ -514,7 +523,7 @@ proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_co
 bool fused_layer_tc128_supported(const Geometry& g, int d_ff) { return g.d == D2 && d_ff >= 64 && d_ff <= 512 && d_ff % 64 == 0; }
 
 cudaError_t launch_ln_qkv_tc128(const Geometry& g, const float* x, int64_t ldx, const float* gamma, const float* beta, float eps,
-                                const __nv_bfloat16* w_qkv, const float* b_qkv, __nv_bfloat16* qkv, cudaStream_t st) {
+                                const __nv_bfloat16* w_qkv, const float* b_qkv, __nv_bfloat16* qkv, int* zero_word, cudaStream_t st) {
   if (g.d != D2) return cudaErrorNotSupported;
   const int64_t rows = matrix_rows(g);  // bounds of the tensor maps; the kernel takes its own row range from the geometry
   const int ntiles = (int)((rows + TM - 1) / TM), nsm = t_sm_count();
@@ -527,8 +536,8 @@ cudaError_t launch_ln_qkv_tc128(const Geometry& g, const float* x, int64_t ldx, 
     cudaError_t e = sm_count_and_smem_once(reinterpret_cast<const void*>(ln_qkv_tc128_kernel), qk2::SMEM, nullptr);
     if (e != cudaSuccess) return e;
   }
-  ln_qkv_tc128_kernel<<<min(ntiles, nsm), T_THREADS, qk2::SMEM, st>>>(tmW, tmX, tmOut, g, gamma, beta, eps, b_qkv);
-  return cudaGetLastError();
+  return launch_overlapped(ln_qkv_tc128_kernel, dim3(min(ntiles, nsm)), dim3(T_THREADS), qk2::SMEM, st, tmW, tmX, tmOut, g, gamma, beta,
+                           eps, b_qkv, zero_word);
 }
 
 cudaError_t launch_proj_mlp_tc128(const Geometry& g, const __nv_bfloat16* att, const float* x, int64_t ldx,
@@ -548,9 +557,8 @@ cudaError_t launch_proj_mlp_tc128(const Geometry& g, const __nv_bfloat16* att, c
     cudaError_t e = sm_count_and_smem_once(reinterpret_cast<const void*>(proj_mlp_tc128_kernel), pm2::SMEM, nullptr);
     if (e != cudaSuccess) return e;
   }
-  proj_mlp_tc128_kernel<<<min(ntiles, nsm), T_THREADS, pm2::SMEM, st>>>(tmAtt, tmX, tmWo, tmW1, tmW2, g, b_o, gamma, beta, eps,
-                                                                       b_1, b_2, d_ff, y, ldy);
-  return cudaGetLastError();
+  return launch_overlapped(proj_mlp_tc128_kernel, dim3(min(ntiles, nsm)), dim3(T_THREADS), pm2::SMEM, st, tmAtt, tmX, tmWo, tmW1, tmW2,
+                           g, b_o, gamma, beta, eps, b_1, b_2, d_ff, y, ldy);
 }
 
 }  // namespace gsit

@@ -156,12 +156,14 @@ gsit_status run_layernorm(const Geometry& g, const float* x, int64_t ldx, const 
 }
 
 gsit_status run_attention(const Geometry& g, int dtype, const void* q, const void* k, const void* v,
-                          int64_t row_stride, void* out, float* lse, float scale, void* scratch, cudaStream_t st) {
+                          int64_t row_stride, void* out, float* lse, float scale, void* scratch, cudaStream_t st,
+                          bool scratch_cleared = false) {
   TraceScope t(GSIT_KERNEL_ATTENTION, st);
   if (dtype == GSIT_BF16)
     return from_cuda(launch_attn_bf16(g, static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k),
                                       static_cast<const __nv_bfloat16*>(v), row_stride,
-                                      static_cast<__nv_bfloat16*>(out), lse, scale, static_cast<int*>(scratch), st));
+                                      static_cast<__nv_bfloat16*>(out), lse, scale, static_cast<int*>(scratch), st,
+                                      scratch_cleared));
   return from_cuda(launch_attn_f32(g, static_cast<const float*>(q), static_cast<const float*>(k),
                                    static_cast<const float*>(v), row_stride, static_cast<float*>(out), lse, scale, st));
 }
@@ -268,18 +270,19 @@ gsit_status gsit_im_layer_fwd(const gsit_shape* shape, const gsit_layer_weights*
       TraceScope t(GSIT_KERNEL_LINEAR, cs);
       st = from_cuda(tc ? launch_ln_qkv_tc(g, x, x_row_stride, w->ln1_gamma, w->ln1_beta, eps,
                                            static_cast<const __nv_bfloat16*>(w->w_qkv), w->b_qkv,
-                                           static_cast<__nv_bfloat16*>(qkv), cs)
+                                           static_cast<__nv_bfloat16*>(qkv), reinterpret_cast<int*>(ws + sc.sched), cs)
                      : tc128 ? launch_ln_qkv_tc128(g, x, x_row_stride, w->ln1_gamma, w->ln1_beta, eps,
                                                    static_cast<const __nv_bfloat16*>(w->w_qkv), w->b_qkv,
-                                                   static_cast<__nv_bfloat16*>(qkv), cs)
+                                                   static_cast<__nv_bfloat16*>(qkv), reinterpret_cast<int*>(ws + sc.sched), cs)
                         : launch_ln_qkv_bf16(g, x, x_row_stride, w->ln1_gamma, w->ln1_beta, eps,
                                              static_cast<const __nv_bfloat16*>(w->w_qkv), w->b_qkv,
                                              static_cast<__nv_bfloat16*>(qkv), cs));
     }
     if (st != GSIT_OK) return st;
     const uint8_t* qb = static_cast<const uint8_t*>(qkv);
+    // the tcgen05 first halves clear the attention kernel's work counter, so no memset separates the three kernels
     if ((st = run_attention(g, dtype, qb, qb + (size_t)d * es, qb + (size_t)2 * d * es, 3 * (int64_t)d, att, nullptr,
-                            pick_scale(shape, g), ws + sc.sched, cs)) != GSIT_OK) return st;
+                            pick_scale(shape, g), ws + sc.sched, cs, tc || tc128)) != GSIT_OK) return st;
     TraceScope t(GSIT_KERNEL_LINEAR, cs);
     if (tc)
       return from_cuda(launch_proj_mlp_tc(g, static_cast<const __nv_bfloat16*>(att), x, x_row_stride,
@@ -381,12 +384,12 @@ gsit_status gsit_im_layer_pair_fwd(const gsit_shape* shape_a, const gsit_shape* 
   }
   {
     TraceScope t(GSIT_KERNEL_LINEAR, cs);
-    if ((st = from_cuda(launch_ln_qkv_tc_pair(ga, h, eps_a, cs))) != GSIT_OK) return st;
+    if ((st = from_cuda(launch_ln_qkv_tc_pair(ga, h, eps_a, reinterpret_cast<int*>(ws + sc.sched), cs))) != GSIT_OK) return st;
   }
   {
     TraceScope t(GSIT_KERNEL_ATTENTION, cs);
     if ((st = from_cuda(launch_attn_bf16_n(ga, ops, 2, 3 * (int64_t)ga.d, pick_scale(shape_a, ga),
-                                           reinterpret_cast<int*>(ws + sc.sched), cs))) != GSIT_OK)
+                                           reinterpret_cast<int*>(ws + sc.sched), cs, true))) != GSIT_OK)
       return st;
   }
   TraceScope t(GSIT_KERNEL_LINEAR, cs);

@@ -136,6 +136,15 @@ __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.a
 
 // True in exactly one lane of a converged warp.  Whole warps run the producer / issuer loops so that addresses,
 // descriptors and barrier phases stay warp-uniform; only the asynchronous instruction itself is issued by one lane.
+// Programmatic dependent launch.  A kernel launched with the "programmatic stream serialization" attribute may start
+// while the kernel before it in the stream is still running; grid_dep_wait() blocks until that kernel has completed and
+// its writes are visible (a no-op for an ordinary launch), so everything above it -- barrier set-up, TMEM allocation,
+// loads of weights -- overlaps the predecessor's tail.  Every kernel launched that way calls it, in every thread, before
+// its first access to memory an earlier kernel of the stream wrote or read: completion then chains through the stream.
+// grid_dep_launch() lets the next kernel's CTAs be placed as soon as every CTA of this one has called it (or exited).
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ bool elect_one() {
   uint32_t pred;
   asm volatile(

@@ -2,6 +2,7 @@
 application's memory budget, inside a latency-critical loop, or after all pools were frozen).  It must give the
 same result as gsit_im_layer_fwd, whose workspace the caller provides, and keep doing so when called again while
 its built-in scratch still holds the previous call's intermediates.  Collected last on purpose."""
+import gc
 import numpy as np
 import pytest
 import torch
@@ -56,6 +57,7 @@ def test_static_scratch_layer_matches_workspace_layer_bit_for_bit(g):
         x, w, vl = _case(g, dtype, B, seg, d, heads, valid, 900 + call)
         want = g.im_layer_fwd(x, w, seg, heads, vl, phase)
         out = torch.full_like(want, float("nan"))
+        gc.collect()  # unreachable tensors of earlier tests go now, not when the collector happens to run below
         torch.cuda.synchronize()
         held, free = torch.cuda.memory_allocated(), _free_bytes()
         got = g.im_layer_fwd_static(x, w, seg, heads, vl, phase, out=out)
