@@ -3,14 +3,18 @@
 //   ln_qkv_tc_kernel     qkv = LN1(x) W_qkv^T + b_qkv          (the shared projection of the concatenated sequence)
 //   proj_mlp_tc_kernel   y1 = x + att W_o^T + b_o ;  y = y1 + relu(LN2(y1) W_1^T + b_1) W_2^T + b_2   (d_ff <= 256)
 //
-// Persistent (the first half two CTAs per SM, the second one), tiles of 128 sequence rows, six warps:
+// Persistent (the first half two CTAs per SM, the second one), tiles of 128 sequence rows:
 //   warp 0      producer: weights once (TMA, 128-byte swizzle, resident for the whole kernel), then per tile the x rows
 //               (TMA, two boxes of 32 floats) and the attention tile (TMA)
-//   warp 1      owns 512 TMEM columns and issues every tcgen05.mma (M 128, K 16, operands from shared memory)
-//   warps 2..5  thread = sequence row = TMEM lane.  LayerNorm needs no shuffles: a thread holds its whole row.  Rows
-//               are written back to shared memory as bf16 in the 128-byte swizzle the MMA expects (the A operand of the
-//               next product), so the normalised rows, the float residual y1 (registers) and the 256 hidden units per
-//               row never leave the SM.  Outputs leave through swizzled staging rows and TMA stores.
+//   warp 1      owns the TMEM columns and issues every tcgen05.mma (M 128, K 16, operands from shared memory)
+//   row warps   thread = sequence row = TMEM lane.  LayerNorm needs no shuffles.  Rows are written back to shared memory
+//               as bf16 in the 128-byte swizzle the MMA expects (the A operand of the next product), so the normalised
+//               rows, the float residual y1 (registers) and the 256 hidden units per row never leave the SM.  Outputs
+//               leave through swizzled staging rows and TMA stores.
+//               First half: four row warps, a thread holds its whole row.  Second half: eight row warps, two threads per
+//               row -- warps w and w + 4 own the same 32 lanes and half of the columns each (of the input row, and
+//               alternate groups of 32 accumulator columns); the pair exchanges a mean and a centred sum of squares
+//               through shared memory for LN2.
 // Every wait is bounded (GSIT_DEVFLAG_TIMEOUT instead of a hang) and TMEM is always released.
 #include "fused_tc_common.cuh"
 
@@ -18,6 +22,15 @@ namespace gsit {
 namespace {
 
 constexpr int TD = 64;            // d_model
+
+// Reads the thread's half of float row r (32 values: one box of a two-box swizzled float tile).
+__device__ __forceinline__ void load_half_row(uint32_t box, int r, float (&v)[32]) {
+#pragma unroll
+  for (int ch = 0; ch < 8; ++ch) {
+    const float4 t = ld_v4f(sw128(box, r, ch));
+    v[4 * ch] = t.x; v[4 * ch + 1] = t.y; v[4 * ch + 2] = t.z; v[4 * ch + 3] = t.w;
+  }
+}
 
 // Reads the thread's float row r (64 values) from a two-box swizzled float tile.
 __device__ __forceinline__ void load_row64(uint32_t tile, int r, float (&v)[TD]) {
@@ -252,7 +265,8 @@ constexpr int OFF_H = OFF_ATT + 2 * TM * 128;      // LN2 output
 constexpr int OFF_F = OFF_H + TM * 128;            // hidden units: up to 4 k-blocks of 128 rows x 128 B; later the y staging
 constexpr int OFF_X = OFF_F + 4 * TM * 128;        // float residual input tile (2 boxes)
 constexpr int OFF_P = OFF_X + 2 * XBOX;            // b_o[64], gamma[64], beta[64], b_2[64], b_1[256] as floats
-constexpr int OFF_BAR = OFF_P + (4 * TD + 256) * 4;
+constexpr int OFF_STAT = OFF_P + (4 * TD + 256) * 4;  // LayerNorm statistics exchanged by the two threads of a row
+constexpr int OFF_BAR = OFF_STAT + 2 * TM * 8;
 constexpr int B_W = 0, B_ATTFULL = 8, B_ATTFREE = 24, B_XFULL = 40, B_XFREE = 48, B_ACC1 = 56, B_HREADY = 64, B_ACCF = 72,
               B_FREADY = 80, B_ACCY = 88, SLOT = 96;
 constexpr int SMEM = OFF_BAR + 112 + 1024;
@@ -266,7 +280,7 @@ struct ProjMlpArgs {
   const float *bo, *gamma, *beta, *b1, *b2;
 };
 
-__global__ void __launch_bounds__(T_THREADS, 1)
+__global__ void __launch_bounds__(T_THREADS8, 1)
 proj_mlp_tc_kernel(const __grid_constant__ ProjMlpArgs arg0, const __grid_constant__ ProjMlpArgs arg1, const Geometry g,
                    const float eps, const int d_ff, const int problems) {
   using namespace pm;
@@ -285,21 +299,21 @@ proj_mlp_tc_kernel(const __grid_constant__ ProjMlpArgs arg0, const __grid_consta
   const int nh = d_ff / 64;  // k-blocks of hidden units
 
   float* prm = reinterpret_cast<float*>(base_ptr + OFF_P);
-  stage_vector(prm, bo, TD, 0.f, tid, T_THREADS);
-  stage_vector(prm + TD, gamma, TD, 1.f, tid, T_THREADS);
-  stage_vector(prm + 2 * TD, beta, TD, 0.f, tid, T_THREADS);
-  stage_vector(prm + 3 * TD, b2, TD, 0.f, tid, T_THREADS);
-  stage_vector(prm + 4 * TD, b1, d_ff, 0.f, tid, T_THREADS);
+  stage_vector(prm, bo, TD, 0.f, tid, T_THREADS8);
+  stage_vector(prm + TD, gamma, TD, 1.f, tid, T_THREADS8);
+  stage_vector(prm + 2 * TD, beta, TD, 0.f, tid, T_THREADS8);
+  stage_vector(prm + 3 * TD, b2, TD, 0.f, tid, T_THREADS8);
+  stage_vector(prm + 4 * TD, b1, d_ff, 0.f, tid, T_THREADS8);
   if (tid == 0) {
     asm volatile("st.shared.u32 [%0], %1;" ::"r"(bars + SLOT + 4), "r"(0u) : "memory");
     mbar_init(bars + B_W, 1);
     for (int i = 0; i < 2; ++i) { mbar_init(bars + B_ATTFULL + 8 * i, 1); mbar_init(bars + B_ATTFREE + 8 * i, 1); }
     mbar_init(bars + B_XFULL, 1);
-    mbar_init(bars + B_XFREE, 4);
+    mbar_init(bars + B_XFREE, 8);
     mbar_init(bars + B_ACC1, 1);
-    mbar_init(bars + B_HREADY, 4);
+    mbar_init(bars + B_HREADY, 8);
     mbar_init(bars + B_ACCF, 1);
-    mbar_init(bars + B_FREADY, 4);
+    mbar_init(bars + B_FREADY, 8);
     mbar_init(bars + B_ACCY, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
@@ -390,8 +404,8 @@ proj_mlp_tc_kernel(const __grid_constant__ ProjMlpArgs arg0, const __grid_consta
       __syncwarp();
     }
   } else {
-    // ================================ one thread per sequence row ================================
-    const int r = ((warp & 3) << 5) + lane;
+    // ================================ two threads per sequence row ================================
+    const int r = ((warp & 3) << 5) + lane, hf = (warp - 2) >> 2;  // row = TMEM lane; which half of the columns
     const uint32_t tl = tmem + ((uint32_t)((warp & 3) << 5) << 16);
     const uint32_t s_bo = base + OFF_P, s_gamma = s_bo + TD * 4, s_beta = s_gamma + TD * 4, s_b2 = s_beta + TD * 4,
                    s_b1 = s_b2 + TD * 4;
@@ -399,35 +413,36 @@ proj_mlp_tc_kernel(const __grid_constant__ ProjMlpArgs arg0, const __grid_consta
     bool real = row_real32(g, row_base + cta * TM + r, rows);
     for (int t = cta; t < ntiles; t += ctas, ++i) {
       const int row0 = row_base + t * TM;
-      // ---- y1 = x + att W_o^T + b_o (registers) ----
+      // ---- y1 = x + att W_o^T + b_o (this thread's 32 columns, in registers) ----
       mbar_wait(wc, bars + B_XFULL, i & 1);
-      float v[TD];
+      float v[32];
       if (real) {
-        load_row64(base + OFF_X, r, v);
+        load_half_row(base + OFF_X + hf * XBOX, r, v);
       } else {
 #pragma unroll
-        for (int e = 0; e < TD; ++e) v[e] = 0.f;
+        for (int e = 0; e < 32; ++e) v[e] = 0.f;
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(bars + B_XFREE);
       mbar_wait(wc, bars + B_ACC1, i & 1);
       tc_fence_after();
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
+      {
         uint32_t a[32];
-        tmem_ld32(tl + COL_1 + 32 * c, a);
+        tmem_ld32(tl + COL_1 + 32 * hf, a);
         tmem_wait_ld();
 #pragma unroll
         for (int e = 0; e < 32; e += 4) {
-          const float4 bb = ld_v4f(s_bo + (32 * c + e) * 4);
-          v[32 * c + e] += __uint_as_float(a[e]) + bb.x;
-          v[32 * c + e + 1] += __uint_as_float(a[e + 1]) + bb.y;
-          v[32 * c + e + 2] += __uint_as_float(a[e + 2]) + bb.z;
-          v[32 * c + e + 3] += __uint_as_float(a[e + 3]) + bb.w;
+          const float4 bb = ld_v4f(s_bo + (32 * hf + e) * 4);
+          v[e] += __uint_as_float(a[e]) + bb.x;
+          v[e + 1] += __uint_as_float(a[e + 1]) + bb.y;
+          v[e + 2] += __uint_as_float(a[e + 2]) + bb.z;
+          v[e + 3] += __uint_as_float(a[e + 3]) + bb.w;
         }
       }
       // ---- h = LN2(y1) -> A operand of the first MLP product ----
-      layernorm_row_to_tile(v, real, s_gamma, s_beta, eps, base + OFF_H, r);
+      float mean, rstd;
+      split_row_stats<32>(v, base + OFF_STAT, r, hf, eps, real, mean, rstd);
+      normalise_to_tile<32>(v, mean, rstd, real, s_gamma, s_beta, 32 * hf, base + OFF_H, r, 4 * hf);
       fence_async_smem();
       tc_fence_before();
       __syncwarp();
@@ -438,10 +453,10 @@ proj_mlp_tc_kernel(const __grid_constant__ ProjMlpArgs arg0, const __grid_consta
       tc_fence_after();
       if (i > 0) {  // the previous tile's output stores must have finished reading the staging rows (they overlay f)
         if (tid == 64) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-        t_bar_rows();
+        t_bar_rows8();
       }
 #pragma unroll 1
-      for (int c0 = 0; c0 < d_ff; c0 += 32) {
+      for (int c0 = 32 * hf; c0 < d_ff; c0 += 64) {  // alternate groups of 32 hidden units
         uint32_t a[32];
         tmem_ld32(tl + COL_F + c0, a);
         tmem_wait_ld();
@@ -461,28 +476,27 @@ proj_mlp_tc_kernel(const __grid_constant__ ProjMlpArgs arg0, const __grid_consta
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bars + B_FREADY);
-      // ---- y = y1 + f W_2^T + b_2 -> staging rows (two boxes of 32 floats) -> TMA stores; padded rows +0 ----
+      // ---- y = y1 + f W_2^T + b_2 -> staging rows (this thread's box of 32 floats) -> TMA stores; padded rows +0 ----
       mbar_wait(wc, bars + B_ACCY, i & 1);
       tc_fence_after();
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
+      {
         uint32_t a[32];
-        tmem_ld32(tl + COL_Y + 32 * c, a);
+        tmem_ld32(tl + COL_Y + 32 * hf, a);
         tmem_wait_ld();
-        const uint32_t box = base + OFF_F + c * (TM * 128);
+        const uint32_t box = base + OFF_F + hf * (TM * 128);
 #pragma unroll
         for (int ch = 0; ch < 8; ++ch) {
-          const int e = 32 * c + 4 * ch;
-          const float4 bb = ld_v4f(s_b2 + e * 4);
-          float o0 = v[e] + __uint_as_float(a[4 * ch]) + bb.x, o1 = v[e + 1] + __uint_as_float(a[4 * ch + 1]) + bb.y;
-          float o2 = v[e + 2] + __uint_as_float(a[4 * ch + 2]) + bb.z, o3 = v[e + 3] + __uint_as_float(a[4 * ch + 3]) + bb.w;
+          const int e = 4 * ch;
+          const float4 bb = ld_v4f(s_b2 + (32 * hf + e) * 4);
+          float o0 = v[e] + __uint_as_float(a[e]) + bb.x, o1 = v[e + 1] + __uint_as_float(a[e + 1]) + bb.y;
+          float o2 = v[e + 2] + __uint_as_float(a[e + 2]) + bb.z, o3 = v[e + 3] + __uint_as_float(a[e + 3]) + bb.w;
           if (!real) { o0 = 0.f; o1 = 0.f; o2 = 0.f; o3 = 0.f; }
           st_shared_v4(sw128(box, r, ch), __float_as_uint(o0), __float_as_uint(o1), __float_as_uint(o2), __float_as_uint(o3));
         }
       }
       tc_fence_before();
       fence_async_smem();
-      t_bar_rows();
+      t_bar_rows8();
       if (tid == 64) {
         tma_store_2d(&tmY, base + OFF_F, 0, row0);
         tma_store_2d(&tmY, base + OFF_F + TM * 128, 32, row0);
@@ -550,7 +564,7 @@ cudaError_t launch_proj_mlp_tc(const Geometry& g, const __nv_bfloat16* att, cons
   if (!fill_proj_mlp(&a, rows, att, x, ldx, w_o, b_o, gamma, beta, w_1, b_1, w_2, b_2, d_ff, y, ldy)) return cudaErrorInvalidValue;
   cudaError_t e = sm_count_and_smem_once(reinterpret_cast<const void*>(proj_mlp_tc_kernel), pm::SMEM, nullptr);
   if (e != cudaSuccess) return e;
-  return launch_overlapped(proj_mlp_tc_kernel, dim3(min(ntiles, nsm)), dim3(T_THREADS), pm::SMEM, st, a, a, g, eps, d_ff, 1);
+  return launch_overlapped(proj_mlp_tc_kernel, dim3(min(ntiles, nsm)), dim3(T_THREADS8), pm::SMEM, st, a, a, g, eps, d_ff, 1);
 }
 
 // The same two halves for a PAIR of problems of one geometry in one launch each (the two ring encoders' layers of equal
@@ -582,7 +596,7 @@ cudaError_t launch_proj_mlp_tc_pair(const Geometry& g, const FusedHalfArgs (&h)[
       return cudaErrorInvalidValue;
   cudaError_t e = sm_count_and_smem_once(reinterpret_cast<const void*>(proj_mlp_tc_kernel), pm::SMEM, nullptr);
   if (e != cudaSuccess) return e;
-  return launch_overlapped(proj_mlp_tc_kernel, dim3(min(2 * ntiles, nsm & ~1)), dim3(T_THREADS), pm::SMEM, st, a[0], a[1], g, eps, d_ff, 2);
+  return launch_overlapped(proj_mlp_tc_kernel, dim3(min(2 * ntiles, nsm & ~1)), dim3(T_THREADS8), pm::SMEM, st, a[0], a[1], g, eps, d_ff, 2);
 }
 
 }  // namespace gsit

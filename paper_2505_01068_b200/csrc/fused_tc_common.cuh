@@ -39,6 +39,62 @@ __device__ __forceinline__ bool row_real32(const Geometry& g, int row, int rows)
   return (p - g.seg_off[sgm]) < valid_rows(g, b, sgm);
 }
 
+// Kernels whose rows are split between two threads -- the same TMEM lane in warps w and w + 4, each owning half of the
+// columns -- have eight row warps.
+constexpr int T_THREADS8 = 320;
+__device__ __forceinline__ void t_bar_rows8() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
+// LayerNorm statistics of a row whose columns are split between two threads.  Each takes the mean and the centred sum
+// of squares of its own NC values; the pair exchanges them through `s_stat` (2 x 128 float pairs) and merges them with
+// the pairwise update of Chan, Golub and LeVeque, which is symmetric in the two halves, so both threads get the same
+// bits.  Every row thread calls it (it contains a barrier of the eight row warps).
+template <int NC>
+__device__ __forceinline__ void split_row_stats(const float (&v)[NC], uint32_t s_stat, int r, int hf, float eps, bool real,
+                                                float& mean, float& rstd) {
+  float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+  for (int e = 0; e < NC; e += 4) { s0 += v[e]; s1 += v[e + 1]; s2 += v[e + 2]; s3 += v[e + 3]; }
+  const float mean_h = ((s0 + s1) + (s2 + s3)) * (1.f / NC);
+  float q0 = 0.f, q1 = 0.f, q2 = 0.f, q3 = 0.f;
+#pragma unroll
+  for (int e = 0; e < NC; e += 4) {
+    const float a = v[e] - mean_h, b = v[e + 1] - mean_h, c = v[e + 2] - mean_h, d = v[e + 3] - mean_h;
+    q0 = fmaf(a, a, q0); q1 = fmaf(b, b, q1); q2 = fmaf(c, c, q2); q3 = fmaf(d, d, q3);
+  }
+  const float m2_h = (q0 + q1) + (q2 + q3);
+  asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(s_stat + (uint32_t)(hf * TM + r) * 8u), "f"(mean_h), "f"(m2_h) : "memory");
+  t_bar_rows8();
+  float mean_p, m2_p;
+  asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(mean_p), "=f"(m2_p) : "r"(s_stat + (uint32_t)((hf ^ 1) * TM + r) * 8u) : "memory");
+  const float delta = mean_p - mean_h;
+  mean = 0.5f * (mean_h + mean_p);
+  const float m2 = (m2_h + m2_p) + (delta * delta) * (0.5f * NC);
+  rstd = real ? rsqrtf(m2 * (1.f / (2 * NC)) + eps) : 0.f;
+}
+// Normalises the thread's NC columns (the row's columns col0 .. col0 + NC - 1) and writes them as bf16 into row r of a
+// tile of 128-byte rows in the 128-byte swizzle, 16-byte chunks chunk0 .. chunk0 + NC / 8 - 1 (zeros when !real).
+template <int NC>
+__device__ __forceinline__ void normalise_to_tile(const float (&v)[NC], float mean, float rstd, bool real, uint32_t s_gamma,
+                                                  uint32_t s_beta, int col0, uint32_t tile, int r, int chunk0) {
+#pragma unroll
+  for (int ch = 0; ch < NC / 8; ++ch) {
+    const uint32_t off = (uint32_t)(col0 + ch * 8) * 4u;
+    const float4 g0 = ld_v4f(s_gamma + off), g1 = ld_v4f(s_gamma + off + 16);
+    const float4 b0 = ld_v4f(s_beta + off), b1 = ld_v4f(s_beta + off + 16);
+    const float gm[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+    const float bt[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+    uint32_t pk[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int e = ch * 8 + 2 * k;
+      float a = fmaf((v[e] - mean) * rstd, gm[2 * k], bt[2 * k]), b = fmaf((v[e + 1] - mean) * rstd, gm[2 * k + 1], bt[2 * k + 1]);
+      if (!real) { a = 0.f; b = 0.f; }
+      pk[k] = pack_bf16(a, b);
+    }
+    st_shared_v4(sw128(tile, r, chunk0 + ch), pk[0], pk[1], pk[2], pk[3]);
+  }
+}
+
 // 2-D map over a [rows, cols] float view with row pitch `row_stride` elements; box = [32 columns, box_rows rows] (128
 // bytes wide), 128-byte swizzle.
 bool make_map_f32(CUtensorMap* tm, const void* basep, int64_t rows, int cols, int64_t row_stride, int box_rows) {
