@@ -1,6 +1,7 @@
 // The fused halves of the IM encoder layer at d_model 128 (the intra-modal encoder on the feature concat of the two
-// ring encoders) on tcgen05 / TMEM.  Same structure as fused_layer_tc.cu (one CTA per SM, 128-row tiles, thread = row
-// for LayerNorm and epilogues, operands in the 128-byte swizzle); what differs is the budget: rows are two k-blocks of
+// ring encoders) on tcgen05 / TMEM.  Same structure as fused_layer_tc.cu (one CTA per SM, 128-row tiles, two threads per
+// row for LayerNorm and epilogues -- warps w and w + 4 own the same TMEM lanes and half of the columns each --, operands
+// in the 128-byte swizzle); what differs is the budget: rows are two k-blocks of
 // 64 features wide, the 384 QKV columns need two MMA groups (N 256 + N 128), and the MLP weights (2 x 128 KB at
 // d_ff 512) no longer fit in shared memory, so W_1 / W_2 stream through a two-stage TMA ring in chunks of 64 hidden
 // units while the hidden accumulator is double-buffered in TMEM.
@@ -11,64 +12,35 @@ namespace {
 
 constexpr int D2 = 128;  // d_model
 
-// Reads the thread's float row r (128 values) from a four-box swizzled float tile.
-__device__ __forceinline__ void load_row128(uint32_t tile, int r, float (&v)[D2]) {
+// Reads the thread's half of float row r (64 values: two boxes of a four-box swizzled float tile).
+__device__ __forceinline__ void load_half_row128(uint32_t boxes, int r, float (&v)[64]) {
 #pragma unroll
-  for (int j = 0; j < 4; ++j)
+  for (int j = 0; j < 2; ++j)
 #pragma unroll
     for (int ch = 0; ch < 8; ++ch) {
-      const float4 t = ld_v4f(sw128(tile + j * XBOX, r, ch));
+      const float4 t = ld_v4f(sw128(boxes + j * XBOX, r, ch));
       const int e = 32 * j + 4 * ch;
       v[e] = t.x; v[e + 1] = t.y; v[e + 2] = t.z; v[e + 3] = t.w;
     }
-}
-// LayerNorm of one 128-feature row held by one thread -> bf16 row r of two swizzled k-block tiles (zeros when !real).
-__device__ __forceinline__ void layernorm_row128_to_tiles(const float (&v)[D2], bool real, uint32_t s_gamma, uint32_t s_beta,
-                                                          float eps, uint32_t tiles, int r) {
-  float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-#pragma unroll
-  for (int e = 0; e < D2; e += 4) { s0 += v[e]; s1 += v[e + 1]; s2 += v[e + 2]; s3 += v[e + 3]; }
-  const float mean = ((s0 + s1) + (s2 + s3)) * (1.f / D2);
-  float q0 = 0.f, q1 = 0.f, q2 = 0.f, q3 = 0.f;
-#pragma unroll
-  for (int e = 0; e < D2; e += 4) {
-    const float a = v[e] - mean, b = v[e + 1] - mean, c = v[e + 2] - mean, d = v[e + 3] - mean;
-    q0 = fmaf(a, a, q0); q1 = fmaf(b, b, q1); q2 = fmaf(c, c, q2); q3 = fmaf(d, d, q3);
-  }
-  const float rstd = real ? rsqrtf(((q0 + q1) + (q2 + q3)) * (1.f / D2) + eps) : 0.f;
-#pragma unroll
-  for (int c8 = 0; c8 < D2 / 8; ++c8) {  // 16 chunks of 8 features: k-block c8 / 8, chunk c8 % 8
-    const float4 g0 = ld_v4f(s_gamma + c8 * 32), g1 = ld_v4f(s_gamma + c8 * 32 + 16);
-    const float4 b0 = ld_v4f(s_beta + c8 * 32), b1 = ld_v4f(s_beta + c8 * 32 + 16);
-    const float gm[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
-    const float bt[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-    uint32_t pk[4];
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const int e = c8 * 8 + 2 * k;
-      float a = fmaf((v[e] - mean) * rstd, gm[2 * k], bt[2 * k]), b = fmaf((v[e + 1] - mean) * rstd, gm[2 * k + 1], bt[2 * k + 1]);
-      if (!real) { a = 0.f; b = 0.f; }
-      pk[k] = pack_bf16(a, b);
-    }
-    st_shared_v4(sw128(tiles + (c8 >> 3) * XBOX, r, c8 & 7), pk[0], pk[1], pk[2], pk[3]);
-  }
 }
 
 // ------------------------------------------------------------------------------------------------ LN1 + shared QKV
 namespace qk2 {
 constexpr int NQ = 3 * D2;                        // 384 output columns
 constexpr int OFF_W = 0;                          // W_qkv: 2 k-blocks x 384 rows x 128 B
-constexpr int OFF_X = OFF_W + 2 * NQ * 128;       // float input tile (4 boxes); the normalised rows (2 k-blocks) overlay it
+constexpr int OFF_X = OFF_W + 2 * NQ * 128;       // float input tile (4 boxes), refilled as soon as it is in registers
 constexpr int OFF_OUT = OFF_X + 4 * XBOX;         // 3 boxes of 64 columns: the output leaves in two passes
+constexpr int OFF_H = OFF_OUT;                    // normalised rows (2 k-blocks): the first two boxes, free while the MMA runs
 constexpr int OFF_P = OFF_OUT + 3 * XBOX;         // gamma[128], beta[128], bias[384]
-constexpr int OFF_BAR = OFF_P + (2 * D2 + NQ) * 4;
+constexpr int OFF_STAT = OFF_P + (2 * D2 + NQ) * 4;  // LayerNorm statistics exchanged by the two threads of a row
+constexpr int OFF_BAR = OFF_STAT + 2 * TM * 8;
 constexpr int B_W = 0, B_XFULL = 8, B_XFREE = 16, B_HREADY = 24, B_ACCFULL = 32, B_ACCFREE = 40, SLOT = 48;
 constexpr int SMEM = OFF_BAR + 64 + 1024;
 constexpr int TMEM_COLS = 512;
 static_assert(SMEM <= 227 * 1024, "shared memory budget");
 }  // namespace qk2
 
-__global__ void __launch_bounds__(T_THREADS, 1)
+__global__ void __launch_bounds__(T_THREADS8, 1)
 ln_qkv_tc128_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
                     const __grid_constant__ CUtensorMap tmOut, const Geometry g, const float* __restrict__ gamma,
                     const float* __restrict__ beta, const float eps, const float* __restrict__ bias, int* const zero_word) {
@@ -81,17 +53,17 @@ ln_qkv_tc128_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   float* prm = reinterpret_cast<float*>(base_ptr + OFF_P);
-  stage_vector(prm, gamma, D2, 1.f, tid, T_THREADS);
-  stage_vector(prm + D2, beta, D2, 0.f, tid, T_THREADS);
-  stage_vector(prm + 2 * D2, bias, NQ, 0.f, tid, T_THREADS);
+  stage_vector(prm, gamma, D2, 1.f, tid, T_THREADS8);
+  stage_vector(prm + D2, beta, D2, 0.f, tid, T_THREADS8);
+  stage_vector(prm + 2 * D2, bias, NQ, 0.f, tid, T_THREADS8);
   if (tid == 0) {
     asm volatile("st.shared.u32 [%0], %1;" ::"r"(bars + SLOT + 4), "r"(0u) : "memory");
     mbar_init(bars + B_W, 1);
     mbar_init(bars + B_XFULL, 1);
-    mbar_init(bars + B_XFREE, 4);
-    mbar_init(bars + B_HREADY, 4);
+    mbar_init(bars + B_XFREE, 8);
+    mbar_init(bars + B_HREADY, 8);
     mbar_init(bars + B_ACCFULL, 1);
-    mbar_init(bars + B_ACCFREE, 4);
+    mbar_init(bars + B_ACCFREE, 8);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
   }
@@ -123,8 +95,7 @@ ln_qkv_tc128_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     // ================================ producer ================================
     int i = 0;
     for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
-      // the tile buffer also held the previous tile's normalised rows: wait until the MMA has consumed them
-      if (i > 0) mbar_wait(wc, bars + B_XFREE, (i - 1) & 1);
+      if (i > 0) mbar_wait(wc, bars + B_XFREE, (i - 1) & 1);  // the row warps hold the previous tile in registers
       if (elect_one()) {
         mbar_expect_tx(bars + B_XFULL, 4 * XBOX);
         for (int j = 0; j < 4; ++j) tma_load_2d(base + OFF_X + j * XBOX, &tmX, 32 * j, row_base + t * TM, bars + B_XFULL);
@@ -145,7 +116,7 @@ ln_qkv_tc128_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         for (int kb = 0; kb < 2; ++kb)
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
-            const uint64_t a = smem_desc_sw128(base + OFF_X + kb * XBOX + 32 * k);
+            const uint64_t a = smem_desc_sw128(base + OFF_H + kb * XBOX + 32 * k);
             const uint32_t w = base + OFF_W + kb * NQ * 128 + 32 * k;
             umma_ss(tmem, a, smem_desc_sw128(w), IDESC_256, (kb > 0 || k > 0) ? 1u : 0u);                    // columns 0..255
             umma_ss(tmem + 256, a, smem_desc_sw128(w + 256 * 128), IDESC_128, (kb > 0 || k > 0) ? 1u : 0u);  // columns 256..383
@@ -155,8 +126,8 @@ ln_qkv_tc128_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       __syncwarp();
     }
   } else {
-    // ================================ one thread per sequence row ================================
-    const int r = ((warp & 3) << 5) + lane;
+    // ================================ two threads per sequence row ================================
+    const int r = ((warp & 3) << 5) + lane, hf = (warp - 2) >> 2;  // row = TMEM lane; which half of the columns
     const uint32_t tl = tmem + ((uint32_t)((warp & 3) << 5) << 16);
     const uint32_t s_gamma = base + OFF_P, s_beta = s_gamma + D2 * 4, s_bias = s_beta + D2 * 4;
     int i = 0;
@@ -164,32 +135,35 @@ ln_qkv_tc128_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
       const int row0 = row_base + t * TM;
       mbar_wait(wc, bars + B_XFULL, i & 1);
-      float v[D2];
+      float v[64];
       if (real) {
-        load_row128(base + OFF_X, r, v);
+        load_half_row128(base + OFF_X + 2 * hf * XBOX, r, v);
       } else {  // padded input rows may hold anything (NaN included): never read them
 #pragma unroll
-        for (int e = 0; e < D2; ++e) v[e] = 0.f;
+        for (int e = 0; e < 64; ++e) v[e] = 0.f;
       }
-      t_bar_rows();  // every row is in registers: the normalised rows may overwrite the tile
-      layernorm_row128_to_tiles(v, real, s_gamma, s_beta, eps, base + OFF_X, r);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bars + B_XFREE);
+      if (i > 0 && tid == 64) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+      // the barrier inside: the previous tile's stores have finished reading the staging rows the normalised rows overlay
+      float mean, rstd;
+      split_row_stats<64>(v, base + OFF_STAT, r, hf, eps, real, mean, rstd);
+      normalise_to_tile<64>(v, mean, rstd, real, s_gamma, s_beta, 64 * hf, base + OFF_H + hf * XBOX, r, 0);
       fence_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(bars + B_HREADY);
       const bool real_next = row_real32(g, row_base + (t + (int)gridDim.x) * TM + r, rows);  // overlaps the MMA
 
-      mbar_wait(wc, bars + B_ACCFULL, i & 1);
+      mbar_wait(wc, bars + B_ACCFULL, i & 1);  // the MMA has also finished reading the normalised rows
       tc_fence_after();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bars + B_XFREE);  // the MMA has read the normalised rows: the next tile may land
 #pragma unroll 1
       for (int pass = 0; pass < 2; ++pass) {
-        if (i > 0 || pass > 0) {  // earlier stores must have finished reading the staging rows
+        if (pass > 0) {  // the first pass's stores must have finished reading the staging rows
           if (tid == 64) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-          t_bar_rows();
+          t_bar_rows8();
         }
 #pragma unroll 1
-        for (int c0 = 0; c0 < NQ / 2; c0 += 32) {
+        for (int c0 = 32 * hf; c0 < NQ / 2; c0 += 64) {  // alternate groups of 32 output columns
           const int col = pass * (NQ / 2) + c0;
           uint32_t a[32];
           tmem_ld32(tl + col, a);
@@ -215,7 +189,7 @@ ln_qkv_tc128_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
           if (lane == 0) mbar_arrive(bars + B_ACCFREE);
         }
         fence_async_smem();
-        t_bar_rows();
+        t_bar_rows8();
         if (tid == 64) {
 #pragma unroll
           for (int j = 0; j < 3; ++j) tma_store_2d(&tmOut, base + OFF_OUT + j * XBOX, pass * (NQ / 2) + 64 * j, row0);
@@ -244,7 +218,8 @@ constexpr int WC_STAGE = 2 * 64 * 128 + XBOX;      // W_1 chunk: 2 k-blocks x 64
 constexpr int OFF_WC = OFF_X + 4 * XBOX;           // 2 stages
 constexpr int OFF_F = OFF_WC + 2 * WC_STAGE;       // hidden chunk: 128 rows x 64 units, bf16
 constexpr int OFF_P = OFF_F + XBOX;                // b_o[128], gamma[128], beta[128], b_2[128], b_1[512]
-constexpr int OFF_BAR = OFF_P + (4 * D2 + 512) * 4;
+constexpr int OFF_STAT = OFF_P + (4 * D2 + 512) * 4;  // LayerNorm statistics exchanged by the two threads of a row
+constexpr int OFF_BAR = OFF_STAT + 2 * TM * 8;
 constexpr int B_WO = 0, B_ATTFULL = 8, B_ATTFREE = 16, B_XFULL = 24, B_XFREE = 32, B_ACC1 = 40, B_HREADY = 48,
               B_WCFULL = 56, B_WCFREE = 72, B_ACCF = 88, B_FREADY = 104, B_FFREE = 112, B_ACCY = 120, SLOT = 128;
 constexpr int SMEM = OFF_BAR + 144 + 1024;
@@ -252,7 +227,7 @@ constexpr int COL_1 = 0, COL_F = 128, COL_Y = 256, TMEM_COLS = 512;
 static_assert(SMEM <= 227 * 1024, "shared memory budget");
 }  // namespace pm2
 
-__global__ void __launch_bounds__(T_THREADS, 1)
+__global__ void __launch_bounds__(T_THREADS8, 1)
 proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_constant__ CUtensorMap tmX,
                       const __grid_constant__ CUtensorMap tmWo, const __grid_constant__ CUtensorMap tmW1,
                       const __grid_constant__ CUtensorMap tmW2, const Geometry g, const float* __restrict__ bo,
@@ -269,26 +244,26 @@ proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_co
   const int nc = d_ff / 64;  // chunks of 64 hidden units
 
   float* prm = reinterpret_cast<float*>(base_ptr + OFF_P);
-  stage_vector(prm, bo, D2, 0.f, tid, T_THREADS);
-  stage_vector(prm + D2, gamma, D2, 1.f, tid, T_THREADS);
-  stage_vector(prm + 2 * D2, beta, D2, 0.f, tid, T_THREADS);
-  stage_vector(prm + 3 * D2, b2, D2, 0.f, tid, T_THREADS);
-  stage_vector(prm + 4 * D2, b1, d_ff, 0.f, tid, T_THREADS);
+  stage_vector(prm, bo, D2, 0.f, tid, T_THREADS8);
+  stage_vector(prm + D2, gamma, D2, 1.f, tid, T_THREADS8);
+  stage_vector(prm + 2 * D2, beta, D2, 0.f, tid, T_THREADS8);
+  stage_vector(prm + 3 * D2, b2, D2, 0.f, tid, T_THREADS8);
+  stage_vector(prm + 4 * D2, b1, d_ff, 0.f, tid, T_THREADS8);
   if (tid == 0) {
     asm volatile("st.shared.u32 [%0], %1;" ::"r"(bars + SLOT + 4), "r"(0u) : "memory");
     mbar_init(bars + B_WO, 1);
     mbar_init(bars + B_ATTFULL, 1);
     mbar_init(bars + B_ATTFREE, 1);
     mbar_init(bars + B_XFULL, 1);
-    mbar_init(bars + B_XFREE, 4);
+    mbar_init(bars + B_XFREE, 8);
     mbar_init(bars + B_ACC1, 1);
-    mbar_init(bars + B_HREADY, 4);
+    mbar_init(bars + B_HREADY, 8);
     for (int i = 0; i < 2; ++i) {
       mbar_init(bars + B_WCFULL + 8 * i, 1);
       mbar_init(bars + B_WCFREE + 8 * i, 1);
       mbar_init(bars + B_ACCF + 8 * i, 1);
     }
-    mbar_init(bars + B_FREADY, 4);
+    mbar_init(bars + B_FREADY, 8);
     mbar_init(bars + B_FFREE, 1);
     mbar_init(bars + B_ACCY, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -403,8 +378,8 @@ proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_co
       second(n - 1, nc == 1, true);
     }
   } else {
-    // ================================ one thread per sequence row ================================
-    const int r = ((warp & 3) << 5) + lane;
+    // ================================ two threads per sequence row ================================
+    const int r = ((warp & 3) << 5) + lane, hf = (warp - 2) >> 2;  // row = TMEM lane; which half of the columns
     const uint32_t tl = tmem + ((uint32_t)((warp & 3) << 5) << 16);
     const uint32_t s_bo = base + OFF_P, s_gamma = s_bo + D2 * 4, s_beta = s_gamma + D2 * 4, s_b2 = s_beta + D2 * 4,
                    s_b1 = s_b2 + D2 * 4;
@@ -412,98 +387,103 @@ proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_co
     bool real = row_real32(g, row_base + (int)blockIdx.x * TM + r, rows);
     for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
       const int row0 = row_base + t * TM;
-      // ---- y1 = x + att W_o^T + b_o (registers) ----
+      // ---- y1 = x + att W_o^T + b_o (this thread's 64 columns, in registers) ----
       mbar_wait(wc, bars + B_XFULL, i & 1);
-      float v[D2];
+      float v[64];
       if (real) {
-        load_row128(base + OFF_X, r, v);
+        load_half_row128(base + OFF_X + 2 * hf * XBOX, r, v);
       } else {
 #pragma unroll
-        for (int e = 0; e < D2; ++e) v[e] = 0.f;
+        for (int e = 0; e < 64; ++e) v[e] = 0.f;
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(bars + B_XFREE);
       mbar_wait(wc, bars + B_ACC1, i & 1);
       tc_fence_after();
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < 2; ++c) {
         uint32_t a[32];
-        tmem_ld32(tl + COL_1 + 32 * c, a);
+        tmem_ld32(tl + COL_1 + 64 * hf + 32 * c, a);
         tmem_wait_ld();
 #pragma unroll
         for (int e = 0; e < 32; e += 4) {
-          const float4 bb = ld_v4f(s_bo + (32 * c + e) * 4);
+          const float4 bb = ld_v4f(s_bo + (64 * hf + 32 * c + e) * 4);
           v[32 * c + e] += __uint_as_float(a[e]) + bb.x;
           v[32 * c + e + 1] += __uint_as_float(a[e + 1]) + bb.y;
           v[32 * c + e + 2] += __uint_as_float(a[e + 2]) + bb.z;
           v[32 * c + e + 3] += __uint_as_float(a[e + 3]) + bb.w;
         }
       }
-      // ---- h = LN2(y1) over the attention tile (its product has completed) ----
-      layernorm_row128_to_tiles(v, real, s_gamma, s_beta, eps, base + OFF_ATT, r);
+      // ---- h = LN2(y1) over the attention tile (its product has completed); this thread's columns are k-block hf ----
+      float mean, rstd;
+      split_row_stats<64>(v, base + OFF_STAT, r, hf, eps, real, mean, rstd);
+      normalise_to_tile<64>(v, mean, rstd, real, s_gamma, s_beta, 64 * hf, base + OFF_ATT + hf * XBOX, r, 0);
       fence_async_smem();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bars + B_HREADY);
       const bool real_next = row_real32(g, row_base + (t + (int)gridDim.x) * TM + r, rows);
-      // ---- hidden chunks: f = relu(h W_1c^T + b_1c) -> A operand of the second product ----
+      // ---- hidden chunks: f = relu(h W_1c^T + b_1c) -> A operand of the second product (32 of the 64 units each) ----
 #pragma unroll 1
       for (int c = 0; c < nc; ++c, ++n) {
         mbar_wait(wc, bars + B_ACCF + 8 * (n & 1), (n >> 1) & 1);
         tc_fence_after();
-        uint32_t pk[32];
-#pragma unroll
-        for (int hlf = 0; hlf < 2; ++hlf) {
+        uint32_t pk[16];
+        {
           uint32_t a[32];
-          tmem_ld32(tl + COL_F + 64 * (n & 1) + 32 * hlf, a);
+          tmem_ld32(tl + COL_F + 64 * (n & 1) + 32 * hf, a);
           tmem_wait_ld();
 #pragma unroll
           for (int e = 0; e < 32; e += 4) {
-            const float4 bb = ld_v4f(s_b1 + (64 * c + 32 * hlf + e) * 4);
-            pk[16 * hlf + (e >> 1)] = pack_bf16(fmaxf(__uint_as_float(a[e]) + bb.x, 0.f), fmaxf(__uint_as_float(a[e + 1]) + bb.y, 0.f));
-            pk[16 * hlf + (e >> 1) + 1] = pack_bf16(fmaxf(__uint_as_float(a[e + 2]) + bb.z, 0.f), fmaxf(__uint_as_float(a[e + 3]) + bb.w, 0.f));
+            const float4 bb = ld_v4f(s_b1 + (64 * c + 32 * hf + e) * 4);
+            pk[e >> 1] = pack_bf16(fmaxf(__uint_as_float(a[e]) + bb.x, 0.f), fmaxf(__uint_as_float(a[e + 1]) + bb.y, 0.f));
+            pk[(e >> 1) + 1] = pack_bf16(fmaxf(__uint_as_float(a[e + 2]) + bb.z, 0.f), fmaxf(__uint_as_float(a[e + 3]) + bb.w, 0.f));
           }
         }
         if (n > 0) mbar_wait(wc, bars + B_FFREE, (n - 1) & 1);  // the previous second product has read the hidden chunk
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch) st_shared_v4(sw128(base + OFF_F, r, ch), pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
+        for (int q = 0; q < 4; ++q) st_shared_v4(sw128(base + OFF_F, r, 4 * hf + q), pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
         fence_async_smem();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bars + B_FREADY);
       }
-      // ---- y = y1 + f W_2^T + b_2: each thread stores its own 512-byte row; padded rows +0 ----
+      // ---- y = y1 + f W_2^T + b_2; padded rows +0 ----
       mbar_wait(wc, bars + B_ACCY, i & 1);
       tc_fence_after();
-      // The rows leave through a per-warp transpose in shared memory (this warp's 32 rows of the hidden-chunk buffer,
-      // which nothing reads between the last second product and this warp's next chunk): a thread owns a row, but a
-      // store instruction that writes 16 bytes to each of 32 rows wastes half of every sector, so 32 columns at a time
-      // are written swizzled and read back with eight lanes per row -- each store then covers four full 128-byte lines.
-      const uint32_t scr = base + OFF_F + (warp & 3) * 4096;
-      const int rr0 = lane >> 3, jj = lane & 7;
+      // The rows leave through a per-warp transpose in shared memory (2 KB of the hidden-chunk buffer per warp, which
+      // nothing reads between the last second product and the next tile's first chunk): a thread owns a row, but a store
+      // instruction that writes 16 bytes to each of 32 rows touches half of 32 sectors, so 16 columns at a time are
+      // written swizzled and read back with four lanes per row -- each store then covers 8 rows x 64 contiguous bytes.
+      const uint32_t scr = base + OFF_F + (uint32_t)(warp - 2) * 2048u;
+      const int jj = lane & 3, rr0 = lane >> 2;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < 2; ++c) {
         uint32_t a[32];
-        tmem_ld32(tl + COL_Y + 32 * c, a);
+        tmem_ld32(tl + COL_Y + 64 * hf + 32 * c, a);
         tmem_wait_ld();
 #pragma unroll
-        for (int e = 0; e < 32; e += 4) {
-          const float4 bb = ld_v4f(s_b2 + (32 * c + e) * 4);
-          float4 o = make_float4(v[32 * c + e] + __uint_as_float(a[e]) + bb.x, v[32 * c + e + 1] + __uint_as_float(a[e + 1]) + bb.y,
-                                 v[32 * c + e + 2] + __uint_as_float(a[e + 2]) + bb.z, v[32 * c + e + 3] + __uint_as_float(a[e + 3]) + bb.w);
-          if (!real) o = make_float4(0.f, 0.f, 0.f, 0.f);
-          st_shared_v4(scr + lane * 128 + ((((e >> 2)) ^ (lane & 7)) << 4), __float_as_uint(o.x), __float_as_uint(o.y), __float_as_uint(o.z),
-                __float_as_uint(o.w));
-        }
-        __syncwarp();
+        for (int sub = 0; sub < 2; ++sub) {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const int rr = 4 * k + rr0;
-          const float4 o = ld_v4f(scr + rr * 128 + ((jj ^ (rr & 7)) << 4));
-          const int grow = row0 + ((warp & 3) << 5) + rr;
-          if (grow < rows) *reinterpret_cast<float4*>(y + (int64_t)grow * ldy + 32 * c + 4 * jj) = o;
+          for (int q = 0; q < 4; ++q) {
+            const int e = 16 * sub + 4 * q, ve = 32 * c + e;
+            const float4 bb = ld_v4f(s_b2 + (64 * hf + ve) * 4);
+            float4 o = make_float4(v[ve] + __uint_as_float(a[e]) + bb.x, v[ve + 1] + __uint_as_float(a[e + 1]) + bb.y,
+                                   v[ve + 2] + __uint_as_float(a[e + 2]) + bb.z, v[ve + 3] + __uint_as_float(a[e + 3]) + bb.w);
+            if (!real) o = make_float4(0.f, 0.f, 0.f, 0.f);
+            st_shared_v4(scr + lane * 64 + ((q ^ ((lane >> 1) & 3)) << 4), __float_as_uint(o.x), __float_as_uint(o.y), __float_as_uint(o.z),
+                         __float_as_uint(o.w));
+          }
+          __syncwarp();
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const int rr = 8 * k + rr0;
+            const float4 o = ld_v4f(scr + rr * 64 + ((jj ^ ((rr >> 1) & 3)) << 4));
+            const int grow = row0 + ((warp & 3) << 5) + rr;
+            if (grow < rows) *reinterpret_cast<float4*>(y + (int64_t)grow * ldy + 64 * hf + 32 * c + 16 * sub + 4 * jj) = o;
+          }
+          __syncwarp();
         }
-        __syncwarp();
       }
       tc_fence_before();  // orders these TMEM reads before the next tile's products (which wait for this thread's arrivals)
       real = real_next;
@@ -536,7 +516,7 @@ cudaError_t launch_ln_qkv_tc128(const Geometry& g, const float* x, int64_t ldx, 
     cudaError_t e = sm_count_and_smem_once(reinterpret_cast<const void*>(ln_qkv_tc128_kernel), qk2::SMEM, nullptr);
     if (e != cudaSuccess) return e;
   }
-  return launch_overlapped(ln_qkv_tc128_kernel, dim3(min(ntiles, nsm)), dim3(T_THREADS), qk2::SMEM, st, tmW, tmX, tmOut, g, gamma, beta,
+  return launch_overlapped(ln_qkv_tc128_kernel, dim3(min(ntiles, nsm)), dim3(T_THREADS8), qk2::SMEM, st, tmW, tmX, tmOut, g, gamma, beta,
                            eps, b_qkv, zero_word);
 }
 
@@ -557,7 +537,7 @@ cudaError_t launch_proj_mlp_tc128(const Geometry& g, const __nv_bfloat16* att, c
     cudaError_t e = sm_count_and_smem_once(reinterpret_cast<const void*>(proj_mlp_tc128_kernel), pm2::SMEM, nullptr);
     if (e != cudaSuccess) return e;
   }
-  return launch_overlapped(proj_mlp_tc128_kernel, dim3(min(ntiles, nsm)), dim3(T_THREADS), pm2::SMEM, st, tmAtt, tmX, tmWo, tmW1, tmW2,
+  return launch_overlapped(proj_mlp_tc128_kernel, dim3(min(ntiles, nsm)), dim3(T_THREADS8), pm2::SMEM, st, tmAtt, tmX, tmWo, tmW1, tmW2,
                            g, b_o, gamma, beta, eps, b_1, b_2, d_ff, y, ldy);
 }
 
