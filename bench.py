@@ -46,6 +46,12 @@ def recorded_traffic(kernel: str):
     return None if rec is None else float(rec["dram_bytes_per_launch"])
 
 
+def scaled_traffic(per_problem, problems: int):
+    """The capture is of a launch serving one problem; a launch serving two independent problems of the same shape moves
+    twice the bytes."""
+    return None if per_problem is None else per_problem * problems
+
+
 def peaks():
     p = ROOT / "MEASURED_PEAKS.json"
     if p.exists():
@@ -306,7 +312,8 @@ def run_gpu(args):
     nbuf = max(2, int(np.ceil(1.2 * L2_BYTES / x_host.numel() / 4)))
     xbufs = [x_host.cuda() for _ in range(nbuf)]
     # per layer: LN1+QKV, IM attention, out-proj+LN2+MLP (fused kernels); each intra layer once per half of the batch
-    launches_per_step = 3 * (n_f + n_b) + 3 * n_i * (2 if (stack.intra_halves and B >= 2) else 1)
+    paired = stack.paired_rings and n_f == n_b and n_f > 0   # one launch per kernel for both rings of a depth
+    launches_per_step = 3 * (n_f if paired else n_f + n_b) + 3 * n_i * (2 if (stack.intra_halves and B >= 2) else 1)
     if stack.packed:
         launches_per_step += 3   # row plan, gather of the real rows, scatter of the result
 
@@ -354,7 +361,8 @@ def run_gpu(args):
     y_host = y_hosts[0]
 
     # ---- per-kernel device times inside the step (eager, CUDA events around each launch) ----
-    # The two rings are issued one after the other here, so that every event pair brackets one kernel running alone.
+    # Everything is issued on one stream here (the intra encoder on the whole batch), so that every event pair brackets
+    # one kernel running alone; with paired rings a cross-modal launch serves both rings (two problems).
     trace_steps = max(1, min(args.steps, 10))
     stack.concurrent_rings = False
     g.trace_enable(True)
@@ -366,10 +374,13 @@ def run_gpu(args):
     lin_ms, lin_n = g.trace_read(g.KERNEL_LINEAR)
     ln_ms, ln_n = g.trace_read(g.KERNEL_LAYERNORM)
     g.trace_enable(False)
-    per_step = n_f + n_b + n_i
+    n_cross = n_f if paired else n_f + n_b
+    problems = 2 if paired else 1
+    per_step = n_cross + n_i
     att = np.asarray(att).reshape(trace_steps, per_step)
-    cross_s = float(att[:, : n_f + n_b].mean()) * 1e-3
-    intra_s = float(att[:, n_f + n_b:].mean()) * 1e-3 if n_i else None
+    cross_launch_s = float(att[:, :n_cross].mean()) * 1e-3
+    cross_s = cross_launch_s / problems          # per problem
+    intra_s = float(att[:, n_cross:].mean()) * 1e-3 if n_i else None
     pk, pk_kind = peaks()
 
     if rank != 0:
@@ -473,8 +484,9 @@ def run_gpu(args):
                    f"intra x{n_i} at d={2 * wl.d_model} (hd={2 * wl.d_model // ih})",
                    "valid_tokens_per_step": tokens, "padded_tokens_per_step": B * wl.L,
                    "l2": f"inputs rotate over {nbuf} device copies ({nbuf * x_host.numel() * 4 >> 20} MiB > 126 MiB L2); "
-                         "the step's scratch alone is larger than L2", "launch": "one CUDA graph per input buffer; inside it the forward and backward rings on two streams, then the "
-                             "intra encoder on the two halves of the batch on the same two streams; packed row layout (real rows only)"},
+                         "the step's scratch alone is larger than L2", "launch": "one CUDA graph per input buffer; inside it " + ("the forward and backward ring layers of each depth in one launch per kernel (two problems per launch), " if paired else "the forward and backward rings on two streams, ") +
+                             "then the intra encoder on the two halves of the batch on two streams; packed row layout (real rows only); "
+                             "kernels of a stream start under the tail of the one before (programmatic dependent launch)"},
         "clocks": clocks.summary(),
         "timed_regions": {"repeats": args.repeats, "steps_each": args.steps, "ms_per_step_median": ms_per_step,
                           "ms_per_step_min": min(regions) / args.steps, "ms_per_step_max": max(regions) / args.steps},
@@ -482,11 +494,12 @@ def run_gpu(args):
                 "d2h_bytes_per_step": int(y_host.numel() * 4) ,
                 "how": "HostPipeline, 2 steps in flight: copy-in, kernels and copy-out of neighbouring steps overlap"},
         "gpu_launches": launches_per_step * args.steps,
-        "roofline": {"kernel": "attn_bf16_kernel<8,64> (cross-modal IM attention inside the step)", "bound": "hbm",
-                     "achieved": cross["bytes"] / cross_s / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s",
-                     "frac": cross["bytes"] / cross_s / 1e9 / pk["hbm_gbs"], "traffic": recorded_traffic("attn_bf16_hd8_cfg4_cross"), "peak_kind": "of " + pk_kind,
-                     "launch_us": cross_s * 1e6, "algorithmic_bytes": cross["bytes"],
-                     "timed": "event pair around each launch, rings issued serially for this pass",
+        "roofline": {"kernel": "attn_bf16_kernel<8,64> (cross-modal IM attention inside the step" + (", both rings' layers of a depth in one launch)" if paired else ")"), "bound": "hbm",
+                     "achieved": problems * cross["bytes"] / cross_launch_s / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                     "frac": problems * cross["bytes"] / cross_launch_s / 1e9 / pk["hbm_gbs"],
+                     "traffic": scaled_traffic(recorded_traffic("attn_bf16_hd8_cfg4_cross"), problems), "peak_kind": "of " + pk_kind,
+                     "launch_us": cross_launch_s * 1e6, "algorithmic_bytes": problems * cross["bytes"], "problems_per_launch": problems,
+                     "timed": "event pair around each launch, everything on one stream for this pass; traffic = the one-problem capture x problems per launch",
                      # the same launch against the exponential unit: one ex2 per useful (query, key) pair per head
                      "alu": {"bound": "ex2 (special-function unit)", "achieved": wl.heads * cross["pairs"] / cross_s / 1e9,
                              "peak": ex2_rate / 1e9, "unit": "Gex2/s", "frac": wl.heads * cross["pairs"] / cross_s / ex2_rate,

@@ -17,23 +17,24 @@ from . import binding as B
 class GsitStack:
     def __init__(self, fwd_layers, bwd_layers, intra_layers, seg_len, heads, intra_heads, ln_eps=1e-5, head=None,
                  concurrent_rings=True, batch_chunks=1, intra_halves=True,
-                 packed=True, paired_rings=False):
+                 packed=True, paired_rings=True):
         """head: optional (w_f, b_f) of the read-out X_m = f(|| Split(.)[-1]); see read_out().
         concurrent_rings: issue independent work on several streams (False: every launch on the caller's stream, whole
         batch per launch).  batch_chunks: with concurrent issue, the batch is cut into this many groups of samples, each
         with its own pair of streams; samples never interact, so the result does not depend on it.  (At B = 64, L = 1050
         one chunk is fastest: the persistent fused kernels pay their per-CTA set-up once per launch.)
         intra_halves: with concurrent issue, the intra encoder runs on the two halves of the batch on the two streams, so
-        that the attention of one half overlaps the fused layer halves of the other (0.934 -> 0.914 ms at that shape;
-        three or four parts are slower again).
+        that the attention of one half overlaps the fused layer halves of the other (0.794 -> 0.784 ms at that shape
+        with paired rings; three or four parts are slower again).
         packed: when valid lengths are given (and the layers are bf16 at widths the tcgen05 fused kernels cover), the
         stack works on the packed row layout: the real rows are gathered once, every layer runs on them only, and the
         result is scattered back with +0 in the padded positions.  The row-wise parts of the layers then do no work
         for padding (24 % of the rows at the benchmark's lengths).  The plan of where each segment starts is made on the
         device, so a captured forward stays valid when the lengths change.
-        paired_rings: (packed layout) the forward-ring and backward-ring layers of equal depth go through one
-        gsit_im_layer_pair_fwd call each -- three launches per depth for both rings, on one stream -- instead of two
-        streams of three launches."""
+        paired_rings: (packed layout, rings of equal depth) the forward-ring and backward-ring layers of equal depth go
+        through one gsit_im_layer_pair_fwd call each -- three launches per depth for both rings, on one stream, each
+        starting under the tail of the one before it -- instead of two streams of three launches (0.784 against
+        0.789 ms at that shape).  False: one stream per ring."""
         self.head = head
         self.concurrent_rings = concurrent_rings
         self.batch_chunks = max(1, int(batch_chunks))

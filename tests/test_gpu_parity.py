@@ -334,7 +334,7 @@ def test_stack_rings_on_two_streams_match_serial_issue(g):
     mk = lambda conc, chunks=1: g.GsitStack([weights_to_dev(w, "bf16") for w in inp["fwd_layers"]],
                                             [weights_to_dev(w, "bf16") for w in inp["bwd_layers"]],
                                             [weights_to_dev(w, "bf16") for w in inp["intra_layers"]], wl.seg_len, wl.heads,
-                                            ih, concurrent_rings=conc, batch_chunks=chunks)
+                                            ih, concurrent_rings=conc, batch_chunks=chunks, paired_rings=False)
     x = to_dev(inp["x"])
     a = mk(True).forward(x, vl).clone()
     b = mk(False).forward(x, vl).clone()
@@ -342,8 +342,11 @@ def test_stack_rings_on_two_streams_match_serial_issue(g):
     st = mk(True)
     st.intra_halves = False                 # intra encoder on the whole batch instead of one half per stream
     d = st.forward(x, vl).clone()
+    st = mk(True)
+    st.paired_rings = True                  # both rings through the pair call on one stream (the default)
+    e = st.forward(x, vl).clone()
     torch.cuda.synchronize()
-    assert torch.equal(a, b) and torch.equal(a, c) and torch.equal(a, d)
+    assert torch.equal(a, b) and torch.equal(a, c) and torch.equal(a, d) and torch.equal(a, e)
     assert g.last_device_status() == (0, 0)
 
 
@@ -459,8 +462,8 @@ def test_packed_layout_gives_the_same_bits_as_the_padded_one(g):
                                   [weights_to_dev(w, "bf16") for w in inp["bwd_layers"]],
                                   [weights_to_dev(w, "bf16") for w in inp["intra_layers"]], wl.seg_len, wl.heads, ih, **kw)
     a = mk(packed=False).forward(x, vl).clone()
-    for kw in (dict(), dict(intra_halves=False), dict(concurrent_rings=False), dict(paired_rings=True),
-               dict(paired_rings=True, intra_halves=False)):
+    for kw in (dict(), dict(intra_halves=False), dict(concurrent_rings=False), dict(paired_rings=False),
+               dict(paired_rings=False, intra_halves=False), dict(paired_rings=False, concurrent_rings=False)):
         st = mk(**kw)
         b = st.forward(x, vl).clone()
         torch.cuda.synchronize()
