@@ -221,8 +221,9 @@ constexpr int OFF_P = OFF_F + XBOX;                // b_o[128], gamma[128], beta
 constexpr int OFF_STAT = OFF_P + (4 * D2 + 512) * 4;  // LayerNorm statistics exchanged by the two threads of a row
 constexpr int OFF_BAR = OFF_STAT + 2 * TM * 8;
 constexpr int B_WO = 0, B_ATTFULL = 8, B_ATTFREE = 16, B_XFULL = 24, B_XFREE = 32, B_ACC1 = 40, B_HREADY = 48,
-              B_WCFULL = 56, B_WCFREE = 72, B_ACCF = 88, B_FREADY = 104, B_FFREE = 112, B_ACCY = 120, SLOT = 128;
-constexpr int SMEM = OFF_BAR + 144 + 1024;
+              B_W1FULL = 56, B_W1FREE = 72, B_ACCF = 88, B_FREADY = 104, B_FFREE = 112, B_ACCY = 120, B_W2FULL = 128,
+              B_W2FREE = 144, SLOT = 160;
+constexpr int SMEM = OFF_BAR + 176 + 1024;
 constexpr int COL_1 = 0, COL_F = 128, COL_Y = 256, TMEM_COLS = 512;
 static_assert(SMEM <= 227 * 1024, "shared memory budget");
 }  // namespace pm2
@@ -259,8 +260,10 @@ proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_co
     mbar_init(bars + B_ACC1, 1);
     mbar_init(bars + B_HREADY, 8);
     for (int i = 0; i < 2; ++i) {
-      mbar_init(bars + B_WCFULL + 8 * i, 1);
-      mbar_init(bars + B_WCFREE + 8 * i, 1);
+      mbar_init(bars + B_W1FULL + 8 * i, 1);
+      mbar_init(bars + B_W1FREE + 8 * i, 1);
+      mbar_init(bars + B_W2FULL + 8 * i, 1);
+      mbar_init(bars + B_W2FREE + 8 * i, 1);
       mbar_init(bars + B_ACCF + 8 * i, 1);
     }
     mbar_init(bars + B_FREADY, 8);
@@ -292,35 +295,54 @@ proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_co
 
   if (warp == 0) {
     // ================================ producer ================================
-    int i = 0, n = 0;  // tiles, weight chunks requested so far
+    // The two halves of a weight chunk have their own rings: the W_1 half of a stage is free once the chunk's first product
+    // has completed, the W_2 half only after its second product, two hand-overs later.  Requests are made in the order in
+    // which their stages come free -- W_1(n), then W_2(n - 1) -- so that no wait holds back a load that could already go.
+    int i = 0, n = 0;  // tiles, weight chunks whose W_1 half has been requested
+    auto request_w1 = [&](int m) {
+      const int st = m & 1, use = m >> 1, c = m % nc;
+      if (use > 0) mbar_wait(wc, bars + B_W1FREE + 8 * st, (use - 1) & 1);
+      if (elect_one()) {
+        const uint32_t dst = base + OFF_WC + st * WC_STAGE;
+        mbar_expect_tx(bars + B_W1FULL + 8 * st, 2 * 64 * 128);
+        tma_load_2d(dst, &tmW1, 0, 64 * c, bars + B_W1FULL + 8 * st);              // W_1[64c .. 64c+63, 0..63]
+        tma_load_2d(dst + 64 * 128, &tmW1, 64, 64 * c, bars + B_W1FULL + 8 * st);  // W_1[64c .. 64c+63, 64..127]
+      }
+      __syncwarp();
+    };
+    auto request_w2 = [&](int m) {
+      const int st = m & 1, use = m >> 1, c = m % nc;
+      if (use > 0) mbar_wait(wc, bars + B_W2FREE + 8 * st, (use - 1) & 1);
+      if (elect_one()) {
+        const uint32_t dst = base + OFF_WC + st * WC_STAGE + 2 * 64 * 128;
+        mbar_expect_tx(bars + B_W2FULL + 8 * st, XBOX);
+        tma_load_2d(dst, &tmW2, 64 * c, 0, bars + B_W2FULL + 8 * st);              // W_2[0..127, 64c .. 64c+63]
+      }
+      __syncwarp();
+    };
     for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
       const int row0 = row_base + t * TM;
-      // the attention buffer also holds the LN2 rows of the previous tile until its last first-MLP product is done
-      if (i > 0) mbar_wait(wc, bars + B_ATTFREE, (i - 1) & 1);
-      if (elect_one()) {
-        mbar_expect_tx(bars + B_ATTFULL, 2 * XBOX);
-        for (int kb = 0; kb < 2; ++kb) tma_load_2d(base + OFF_ATT + kb * XBOX, &tmAtt, 64 * kb, row0, bars + B_ATTFULL);
-      }
-      __syncwarp();
-      if (i > 0) mbar_wait(wc, bars + B_XFREE, (i - 1) & 1);
-      if (elect_one()) {
-        mbar_expect_tx(bars + B_XFULL, 4 * XBOX);
-        for (int j = 0; j < 4; ++j) tma_load_2d(base + OFF_X + j * XBOX, &tmX, 32 * j, row0, bars + B_XFULL);
-      }
-      __syncwarp();
       for (int c = 0; c < nc; ++c, ++n) {
-        const int st = n & 1, use = n >> 1;
-        if (use > 0) mbar_wait(wc, bars + B_WCFREE + 8 * st, (use - 1) & 1);
-        if (elect_one()) {
-          const uint32_t dst = base + OFF_WC + st * WC_STAGE;
-          mbar_expect_tx(bars + B_WCFULL + 8 * st, WC_STAGE);
-          tma_load_2d(dst, &tmW1, 0, 64 * c, bars + B_WCFULL + 8 * st);                // W_1[64c .. 64c+63, 0..63]
-          tma_load_2d(dst + 64 * 128, &tmW1, 64, 64 * c, bars + B_WCFULL + 8 * st);    // W_1[64c .. 64c+63, 64..127]
-          tma_load_2d(dst + 2 * 64 * 128, &tmW2, 64 * c, 0, bars + B_WCFULL + 8 * st); // W_2[0..127, 64c .. 64c+63]
+        request_w1(n);
+        if (n > 0) request_w2(n - 1);
+        if (c == 0) {
+          // the attention buffer also holds the LN2 rows of the previous tile until its last first-MLP product is done
+          if (i > 0) mbar_wait(wc, bars + B_ATTFREE, (i - 1) & 1);
+          if (elect_one()) {
+            mbar_expect_tx(bars + B_ATTFULL, 2 * XBOX);
+            for (int kb = 0; kb < 2; ++kb) tma_load_2d(base + OFF_ATT + kb * XBOX, &tmAtt, 64 * kb, row0, bars + B_ATTFULL);
+          }
+          __syncwarp();
+          if (i > 0) mbar_wait(wc, bars + B_XFREE, (i - 1) & 1);
+          if (elect_one()) {
+            mbar_expect_tx(bars + B_XFULL, 4 * XBOX);
+            for (int j = 0; j < 4; ++j) tma_load_2d(base + OFF_X + j * XBOX, &tmX, 32 * j, row0, bars + B_XFULL);
+          }
+          __syncwarp();
         }
-        __syncwarp();
       }
     }
+    if (n > 0) request_w2(n - 1);
   } else if (warp == 1) {
     // ================================ MMA issuer ================================
     constexpr uint32_t IDESC_128 = idesc_bf16(128, false), IDESC_64 = idesc_bf16(64, false);
@@ -341,25 +363,10 @@ proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_co
       }
       __syncwarp();
       mbar_wait(wc, bars + B_HREADY, i & 1);
-      // second product of chunk m (global index): accY += relu-hidden(m) W_2c^T
-      auto second = [&](int m, bool first_of_tile, bool last_of_tile) {
-        mbar_wait(wc, bars + B_FREADY, m & 1);
-        tc_fence_after();
-        if (elect_one()) {
-          const uint32_t w2 = base + OFF_WC + (m & 1) * WC_STAGE + 2 * 64 * 128;
-#pragma unroll
-          for (int k = 0; k < 4; ++k)
-            umma_ss(tmem + COL_Y, smem_desc_sw128(base + OFF_F + 32 * k), smem_desc_sw128(w2 + 32 * k), IDESC_128, (!first_of_tile || k > 0) ? 1u : 0u);
-          umma_commit(bars + B_WCFREE + 8 * (m & 1));
-          umma_commit(bars + B_FFREE);
-          if (last_of_tile) umma_commit(bars + B_ACCY);
-        }
-        __syncwarp();
-      };
-      for (int c = 0; c < nc; ++c, ++n) {
-        // first product of chunk n: hidden accumulator (n & 1) = LN2(y1) W_1c^T
-        const int st = n & 1;
-        mbar_wait(wc, bars + B_WCFULL + 8 * st, (n >> 1) & 1);
+      // first product of chunk m (global index): hidden accumulator (m & 1) = LN2(y1) W_1c^T
+      auto first = [&](int m, bool last_of_tile) {
+        const int st = m & 1;
+        mbar_wait(wc, bars + B_W1FULL + 8 * st, (m >> 1) & 1);
         tc_fence_after();
         if (elect_one()) {
           const uint32_t w1 = base + OFF_WC + st * WC_STAGE;
@@ -370,12 +377,37 @@ proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_co
               umma_ss(tmem + COL_F + 64 * st, smem_desc_sw128(base + OFF_ATT + kb * XBOX + 32 * k), smem_desc_sw128(w1 + kb * 64 * 128 + 32 * k),
                      IDESC_64, (kb > 0 || k > 0) ? 1u : 0u);
           umma_commit(bars + B_ACCF + 8 * st);
-          if (c + 1 == nc) umma_commit(bars + B_ATTFREE);  // LN2 rows no longer needed: the next attention tile may land
+          umma_commit(bars + B_W1FREE + 8 * st);
+          if (last_of_tile) umma_commit(bars + B_ATTFREE);  // LN2 rows no longer needed: the next attention tile may land
         }
         __syncwarp();
-        if (c > 0) second(n - 1, c == 1, false);
+      };
+      // second product of chunk m: accY += relu-hidden(m) W_2c^T
+      auto second = [&](int m, bool first_of_tile, bool last_of_tile) {
+        mbar_wait(wc, bars + B_FREADY, m & 1);
+        mbar_wait(wc, bars + B_W2FULL + 8 * (m & 1), (m >> 1) & 1);
+        tc_fence_after();
+        if (elect_one()) {
+          const uint32_t w2 = base + OFF_WC + (m & 1) * WC_STAGE + 2 * 64 * 128;
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            umma_ss(tmem + COL_Y, smem_desc_sw128(base + OFF_F + 32 * k), smem_desc_sw128(w2 + 32 * k), IDESC_128, (!first_of_tile || k > 0) ? 1u : 0u);
+          umma_commit(bars + B_W2FREE + 8 * (m & 1));
+          umma_commit(bars + B_FFREE);
+          if (last_of_tile) umma_commit(bars + B_ACCY);
+        }
+        __syncwarp();
+      };
+      // The second product of chunk c sits on the critical chain (hidden buffer free -> next ReLU rows -> next second
+      // product); the first product of chunk c + 2 only has to be ready by the time the row warps come back for it.  So
+      // the first products run two chunks ahead and each is issued right behind a second product.
+      first(n, nc == 1);
+      if (nc > 1) first(n + 1, nc == 2);
+      for (int c = 0; c < nc; ++c) {
+        second(n + c, c == 0, c + 1 == nc);  // (its wait covers the rows' reads of hidden accumulator c & 1)
+        if (c + 2 < nc) first(n + c + 2, c + 3 == nc);
       }
-      second(n - 1, nc == 1, true);
+      n += nc;
     }
   } else {
     // ================================ two threads per sequence row ================================
