@@ -51,17 +51,23 @@ __device__ __forceinline__ void t_bar_rows8() { asm volatile("bar.sync 1, 256;" 
 template <int NC>
 __device__ __forceinline__ void split_row_stats(const float (&v)[NC], uint32_t s_stat, int r, int hf, float eps, bool real,
                                                 float& mean, float& rstd) {
-  float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-#pragma unroll
-  for (int e = 0; e < NC; e += 4) { s0 += v[e]; s1 += v[e + 1]; s2 += v[e + 2]; s3 += v[e + 3]; }
-  const float mean_h = ((s0 + s1) + (s2 + s3)) * (1.f / NC);
-  float q0 = 0.f, q1 = 0.f, q2 = 0.f, q3 = 0.f;
+  // packed f32x2 arithmetic: two columns per instruction
+  float2 s0 = make_float2(0.f, 0.f), s1 = s0;
 #pragma unroll
   for (int e = 0; e < NC; e += 4) {
-    const float a = v[e] - mean_h, b = v[e + 1] - mean_h, c = v[e + 2] - mean_h, d = v[e + 3] - mean_h;
-    q0 = fmaf(a, a, q0); q1 = fmaf(b, b, q1); q2 = fmaf(c, c, q2); q3 = fmaf(d, d, q3);
+    s0 = __fadd2_rn(s0, make_float2(v[e], v[e + 1]));
+    s1 = __fadd2_rn(s1, make_float2(v[e + 2], v[e + 3]));
   }
-  const float m2_h = (q0 + q1) + (q2 + q3);
+  const float mean_h = ((s0.x + s0.y) + (s1.x + s1.y)) * (1.f / NC);
+  const float2 nm = make_float2(-mean_h, -mean_h);
+  float2 q0 = make_float2(0.f, 0.f), q1 = q0;
+#pragma unroll
+  for (int e = 0; e < NC; e += 4) {
+    const float2 a = __fadd2_rn(make_float2(v[e], v[e + 1]), nm), b = __fadd2_rn(make_float2(v[e + 2], v[e + 3]), nm);
+    q0 = __ffma2_rn(a, a, q0);
+    q1 = __ffma2_rn(b, b, q1);
+  }
+  const float m2_h = (q0.x + q0.y) + (q1.x + q1.y);
   asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(s_stat + (uint32_t)(hf * TM + r) * 8u), "f"(mean_h), "f"(m2_h) : "memory");
   t_bar_rows8();
   float mean_p, m2_p;
@@ -73,23 +79,25 @@ __device__ __forceinline__ void split_row_stats(const float (&v)[NC], uint32_t s
 }
 // Normalises the thread's NC columns (the row's columns col0 .. col0 + NC - 1) and writes them as bf16 into row r of a
 // tile of 128-byte rows in the 128-byte swizzle, 16-byte chunks chunk0 .. chunk0 + NC / 8 - 1 (zeros when !real).
+// Per pair of columns: (v * rstd - mean * rstd) as one packed fused multiply-add, then * gamma + beta as another.
 template <int NC>
 __device__ __forceinline__ void normalise_to_tile(const float (&v)[NC], float mean, float rstd, bool real, uint32_t s_gamma,
                                                   uint32_t s_beta, int col0, uint32_t tile, int r, int chunk0) {
+  const float2 rs = make_float2(rstd, rstd), nmr = make_float2(-mean * rstd, -mean * rstd);
 #pragma unroll
   for (int ch = 0; ch < NC / 8; ++ch) {
     const uint32_t off = (uint32_t)(col0 + ch * 8) * 4u;
     const float4 g0 = ld_v4f(s_gamma + off), g1 = ld_v4f(s_gamma + off + 16);
     const float4 b0 = ld_v4f(s_beta + off), b1 = ld_v4f(s_beta + off + 16);
-    const float gm[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
-    const float bt[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+    const float2 gm[4] = {make_float2(g0.x, g0.y), make_float2(g0.z, g0.w), make_float2(g1.x, g1.y), make_float2(g1.z, g1.w)};
+    const float2 bt[4] = {make_float2(b0.x, b0.y), make_float2(b0.z, b0.w), make_float2(b1.x, b1.y), make_float2(b1.z, b1.w)};
     uint32_t pk[4];
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
       const int e = ch * 8 + 2 * k;
-      float a = fmaf((v[e] - mean) * rstd, gm[2 * k], bt[2 * k]), b = fmaf((v[e + 1] - mean) * rstd, gm[2 * k + 1], bt[2 * k + 1]);
-      if (!real) { a = 0.f; b = 0.f; }
-      pk[k] = pack_bf16(a, b);
+      const float2 t = __ffma2_rn(make_float2(v[e], v[e + 1]), rs, nmr);
+      const float2 y = __ffma2_rn(t, gm[k], bt[k]);
+      pk[k] = real ? pack_bf16(y.x, y.y) : 0u;
     }
     st_shared_v4(sw128(tile, r, chunk0 + ch), pk[0], pk[1], pk[2], pk[3]);
   }
