@@ -52,7 +52,7 @@ constexpr int S_CTAS_PER_SM = 2;
 constexpr int S_ITEM_SLOTS = 4;
 constexpr int S_QBUF = 16384;  // bytes reserved per Q buffer
 #ifndef GSIT_POLY_PAIRS
-#define GSIT_POLY_PAIRS 0x52
+#define GSIT_POLY_PAIRS 0x11
 #endif
 // The weights are cut to bf16 by dropping the low 16 bits (one byte permute on the integer pipe per pair; the rounding
 // conversion would occupy the special-function unit as long as an exponential).  Dropping bits loses on average
