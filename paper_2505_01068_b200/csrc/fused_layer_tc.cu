@@ -366,11 +366,10 @@ proj_mlp_tc_kernel(const __grid_constant__ ProjMlpArgs arg0, const __grid_consta
     constexpr uint32_t IDESC_D = idesc_bf16(TD, false);
     const uint32_t idesc_f = idesc_bf16(d_ff, false);
     mbar_wait(wc, bars + B_W, 0);
-    int i = 0;
-    for (int t = cta; t < ntiles; t += ctas, ++i) {
-      const int b = i & 1;
-      // y1 accumulator = att W_o^T
-      mbar_wait(wc, bars + B_ATTFULL + 8 * b, (i >> 1) & 1);
+    // y1 accumulator of tile number i_ = att W_o^T
+    auto out_proj = [&](int i_) {
+      const int b = i_ & 1;
+      mbar_wait(wc, bars + B_ATTFULL + 8 * b, (i_ >> 1) & 1);
       tc_fence_after();
       if (elect_one()) {
 #pragma unroll
@@ -380,8 +379,14 @@ proj_mlp_tc_kernel(const __grid_constant__ ProjMlpArgs arg0, const __grid_consta
         umma_commit(bars + B_ACC1);
       }
       __syncwarp();
+    };
+    // The row warps work one tile ahead with the first part of a tile (y1 and LN2) while the tensor core finishes the
+    // tile before it, so the products are issued in that order: W_1 of tile i, W_o of tile i + 1, W_2 of tile i.
+    int i = 0;
+    if (cta < ntiles) out_proj(0);
+    for (int t = cta; t < ntiles; t += ctas, ++i) {
       // hidden accumulator = LN2(y1) W_1^T
-      mbar_wait(wc, bars + B_HREADY, i & 1);
+      mbar_wait(wc, bars + B_HREADY, i & 1);  // (the rows have also read the y1 accumulator of this tile)
       tc_fence_after();
       if (elect_one()) {
 #pragma unroll
@@ -390,6 +395,7 @@ proj_mlp_tc_kernel(const __grid_constant__ ProjMlpArgs arg0, const __grid_consta
         umma_commit(bars + B_ACCF);
       }
       __syncwarp();
+      if (t + ctas < ntiles) out_proj(i + 1);
       // output accumulator = relu(hidden) W_2^T
       mbar_wait(wc, bars + B_FREADY, i & 1);
       tc_fence_after();
@@ -409,22 +415,20 @@ proj_mlp_tc_kernel(const __grid_constant__ ProjMlpArgs arg0, const __grid_consta
     const uint32_t tl = tmem + ((uint32_t)((warp & 3) << 5) << 16);
     const uint32_t s_bo = base + OFF_P, s_gamma = s_bo + TD * 4, s_beta = s_gamma + TD * 4, s_b2 = s_beta + TD * 4,
                    s_b1 = s_b2 + TD * 4;
-    int i = 0;
-    bool real = row_real32(g, row_base + cta * TM + r, rows);
-    for (int t = cta; t < ntiles; t += ctas, ++i) {
-      const int row0 = row_base + t * TM;
-      // ---- y1 = x + att W_o^T + b_o (this thread's 32 columns, in registers) ----
-      mbar_wait(wc, bars + B_XFULL, i & 1);
-      float v[32];
-      if (real) {
-        load_half_row(base + OFF_X + hf * XBOX, r, v);
+    // First part of tile number i_: y1 = x + att W_o^T + b_o (this thread's 32 columns, kept in v_) and h = LN2(y1), the
+    // A operand of the first MLP product.  It runs one tile ahead of the rest, while the tensor core is still busy with
+    // the tile before (whose first MLP product has completed, so the LN2 buffer is free).
+    auto first_part = [&](int i_, bool real_, float (&v_)[32]) {
+      mbar_wait(wc, bars + B_XFULL, i_ & 1);
+      if (real_) {
+        load_half_row(base + OFF_X + hf * XBOX, r, v_);
       } else {
 #pragma unroll
-        for (int e = 0; e < 32; ++e) v[e] = 0.f;
+        for (int e = 0; e < 32; ++e) v_[e] = 0.f;
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(bars + B_XFREE);
-      mbar_wait(wc, bars + B_ACC1, i & 1);
+      mbar_wait(wc, bars + B_ACC1, i_ & 1);
       tc_fence_after();
       {
         uint32_t a[32];
@@ -433,21 +437,28 @@ proj_mlp_tc_kernel(const __grid_constant__ ProjMlpArgs arg0, const __grid_consta
 #pragma unroll
         for (int e = 0; e < 32; e += 4) {
           const float4 bb = ld_v4f(s_bo + (32 * hf + e) * 4);
-          v[e] += __uint_as_float(a[e]) + bb.x;
-          v[e + 1] += __uint_as_float(a[e + 1]) + bb.y;
-          v[e + 2] += __uint_as_float(a[e + 2]) + bb.z;
-          v[e + 3] += __uint_as_float(a[e + 3]) + bb.w;
+          v_[e] += __uint_as_float(a[e]) + bb.x;
+          v_[e + 1] += __uint_as_float(a[e + 1]) + bb.y;
+          v_[e + 2] += __uint_as_float(a[e + 2]) + bb.z;
+          v_[e + 3] += __uint_as_float(a[e + 3]) + bb.w;
         }
       }
-      // ---- h = LN2(y1) -> A operand of the first MLP product ----
       float mean, rstd;
-      split_row_stats<32>(v, base + OFF_STAT, r, hf, eps, real, mean, rstd);
-      normalise_to_tile<32>(v, mean, rstd, real, s_gamma, s_beta, 32 * hf, base + OFF_H, r, 4 * hf);
+      split_row_stats<32>(v_, base + OFF_STAT, r, hf, eps, real_, mean, rstd);
+      normalise_to_tile<32>(v_, mean, rstd, real_, s_gamma, s_beta, 32 * hf, base + OFF_H, r, 4 * hf);
       fence_async_smem();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bars + B_HREADY);
-      const bool real_next = row_real32(g, row_base + (t + ctas) * TM + r, rows);  // overlaps the MMA
+    };
+    int i = 0;
+    bool real = row_real32(g, row_base + cta * TM + r, rows);
+    float v[32];
+    if (cta < ntiles) first_part(0, real, v);
+    for (int t = cta; t < ntiles; t += ctas, ++i) {
+      const int row0 = row_base + t * TM;
+      const bool has_next = t + ctas < ntiles;
+      const bool real_next = row_real32(g, row_base + (t + ctas) * TM + r, rows);
       // ---- f = relu(h W_1^T + b_1) -> A operand of the second MLP product ----
       mbar_wait(wc, bars + B_ACCF, i & 1);
       tc_fence_after();
@@ -476,6 +487,9 @@ proj_mlp_tc_kernel(const __grid_constant__ ProjMlpArgs arg0, const __grid_consta
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bars + B_FREADY);
+      // ---- the next tile's first part, while the second MLP product of this one runs ----
+      float vn[32];
+      if (has_next) first_part(i + 1, real_next, vn);
       // ---- y = y1 + f W_2^T + b_2 -> staging rows (this thread's box of 32 floats) -> TMA stores; padded rows +0 ----
       mbar_wait(wc, bars + B_ACCY, i & 1);
       tc_fence_after();
@@ -503,6 +517,10 @@ proj_mlp_tc_kernel(const __grid_constant__ ProjMlpArgs arg0, const __grid_consta
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
       }
       real = real_next;
+      if (has_next) {
+#pragma unroll
+        for (int e = 0; e < 32; ++e) v[e] = vn[e];
+      }
     }
     if (tid == 64) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
