@@ -168,15 +168,15 @@ ln_qkv_tc128_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
           uint32_t a[32];
           tmem_ld32(tl + col, a);
           tmem_wait_ld();
+          tmem_regs_ready(a);
           uint32_t pk[16];
 #pragma unroll
           for (int e = 0; e < 32; e += 4) {
             const float4 bb = ld_v4f(s_bias + (col + e) * 4);
-            float f0 = __uint_as_float(a[e]) + bb.x, f1 = __uint_as_float(a[e + 1]) + bb.y;
-            float f2 = __uint_as_float(a[e + 2]) + bb.z, f3 = __uint_as_float(a[e + 3]) + bb.w;
-            if (!real) { f0 = 0.f; f1 = 0.f; f2 = 0.f; f3 = 0.f; }
-            pk[e >> 1] = pack_bf16(f0, f1);
-            pk[(e >> 1) + 1] = pack_bf16(f2, f3);
+            const float2 h0 = __fadd2_rn(make_float2(__uint_as_float(a[e]), __uint_as_float(a[e + 1])), make_float2(bb.x, bb.y));
+            const float2 h1 = __fadd2_rn(make_float2(__uint_as_float(a[e + 2]), __uint_as_float(a[e + 3])), make_float2(bb.z, bb.w));
+            pk[e >> 1] = real ? pack_bf16(h0.x, h0.y) : 0u;
+            pk[(e >> 1) + 1] = real ? pack_bf16(h1.x, h1.y) : 0u;
           }
           const uint32_t box = base + OFF_OUT + (c0 >> 6) * XBOX;
           const int ch0 = (c0 & 32) >> 3;
@@ -437,6 +437,7 @@ proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_co
         uint32_t a[32];
         tmem_ld32(tl + COL_1 + 64 * hf + 32 * c, a);
         tmem_wait_ld();
+        tmem_regs_ready(a);
 #pragma unroll
         for (int e = 0; e < 32; e += 4) {
           const float4 bb = ld_v4f(s_bo + (64 * hf + 32 * c + e) * 4);
@@ -465,11 +466,14 @@ proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_co
           uint32_t a[32];
           tmem_ld32(tl + COL_F + 64 * (n & 1) + 32 * hf, a);
           tmem_wait_ld();
+          tmem_regs_ready(a);
 #pragma unroll
           for (int e = 0; e < 32; e += 4) {
             const float4 bb = ld_v4f(s_b1 + (64 * c + 32 * hf + e) * 4);
-            pk[e >> 1] = pack_bf16(fmaxf(__uint_as_float(a[e]) + bb.x, 0.f), fmaxf(__uint_as_float(a[e + 1]) + bb.y, 0.f));
-            pk[(e >> 1) + 1] = pack_bf16(fmaxf(__uint_as_float(a[e + 2]) + bb.z, 0.f), fmaxf(__uint_as_float(a[e + 3]) + bb.w, 0.f));
+            const float2 h0 = __fadd2_rn(make_float2(__uint_as_float(a[e]), __uint_as_float(a[e + 1])), make_float2(bb.x, bb.y));
+            const float2 h1 = __fadd2_rn(make_float2(__uint_as_float(a[e + 2]), __uint_as_float(a[e + 3])), make_float2(bb.z, bb.w));
+            pk[e >> 1] = pack_bf16(fmaxf(h0.x, 0.f), fmaxf(h0.y, 0.f));
+            pk[(e >> 1) + 1] = pack_bf16(fmaxf(h1.x, 0.f), fmaxf(h1.y, 0.f));
           }
         }
         if (n > 0) mbar_wait(wc, bars + B_FFREE, (n - 1) & 1);  // the previous second product has read the hidden chunk
@@ -494,6 +498,7 @@ proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_co
         uint32_t a[32];
         tmem_ld32(tl + COL_Y + 64 * hf + 32 * c, a);
         tmem_wait_ld();
+        tmem_regs_ready(a);
 #pragma unroll
         for (int sub = 0; sub < 2; ++sub) {
 #pragma unroll

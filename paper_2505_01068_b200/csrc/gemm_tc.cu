@@ -135,6 +135,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           uint32_t v[32];
           tmem_ld32(tl + ab * 256 + c0, v);
           tmem_wait_ld();
+          tmem_regs_ready(v);
           const int col0 = n0 + c0;
           uint32_t pk[16];
 #pragma unroll
@@ -169,6 +170,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         uint32_t v[32];
         tmem_ld32(tl + ab * 256 + c0, v);
         tmem_wait_ld();
+        tmem_regs_ready(v);
         const int col0 = n0 + c0;
         if (in_m && col0 < p.N) {
           float f[32];

@@ -50,6 +50,67 @@ def test_cfg4_full_batch_stack_sampled_samples(g):
     assert code == 0 and flags == 0
 
 
+@pytest.mark.parametrize("which", ["cross_d64", "intra_d128"])
+def test_full_batch_layer_repeats_bit_for_bit(g, which):
+    """The same layer call on the same inputs, many times, at the full batch (several tiles per persistent CTA, every
+    prefetch and hand-over of the fused kernels in play): every run must give the bits of the first.  A buffer that is
+    refilled or an accumulator that is overwritten a moment too early shows up here as a handful of changed rows in a
+    few runs out of a hundred, which a single comparison with the oracle would mostly miss."""
+    inp = wk.make_inputs(4)
+    wl = inp["workload"]
+    n_f, n_b, n_i, ih = wl.stack
+    valid = inp["valid_len"]
+    vl = torch.from_numpy(valid).cuda()
+    d, heads, w, phase = ((wl.d_model, wl.heads, inp["fwd_layers"][0], oracle.PHASE_INTER_FWD) if which == "cross_d64"
+                          else (2 * wl.d_model, ih, inp["intra_layers"][0], oracle.PHASE_INTRA))
+    rng = np.random.default_rng(31)
+    x = to_dev(wk.fill_padding(rng.standard_normal((wl.batch, wl.L, d)).astype(np.float32), wl.seg_len, valid, np.nan))
+    wd = weights_to_dev(w, "bf16")
+    first = g.im_layer_fwd(x, wd, wl.seg_len, heads, vl, phase).clone()
+    torch.cuda.synchronize()
+    assert torch.isfinite(first).all()
+    for run in range(120):
+        y = g.im_layer_fwd(x, wd, wl.seg_len, heads, vl, phase)
+        torch.cuda.synchronize()
+        assert torch.equal(y, first), (which, run)
+    # the packed row layout through the same kernels
+    cap = wl.batch * wl.L + 128
+    plan = g.plan_rows(vl, wl.seg_len)
+    xp = torch.zeros((cap, d), device="cuda")
+    g.pack_rows(x, xp, wl.seg_len, vl, plan)
+    used = int(plan[-1])
+    firstp = None
+    for run in range(60):
+        yp = torch.zeros((cap, d), device="cuda")
+        g.im_layer_fwd(xp, wd, wl.seg_len, heads, vl, phase, out=yp, row_start=plan)
+        torch.cuda.synchronize()
+        if firstp is None:
+            firstp = yp.clone()
+        assert torch.equal(yp[:used], firstp[:used]), (which, "packed", run)
+    assert g.last_device_status() == (0, 0)
+
+
+def test_cfg4_stack_repeats_bit_for_bit(g):
+    """The whole stack, eager, repeated on NaN-padded input in each way of issuing it."""
+    inp = wk.make_inputs(4)
+    wl = inp["workload"]
+    n_f, n_b, n_i, ih = wl.stack
+    valid = inp["valid_len"]
+    vl = torch.from_numpy(valid).cuda()
+    x_dev = to_dev(wk.fill_padding(inp["x"], wl.seg_len, valid, np.nan))
+    for kw in (dict(), dict(paired_rings=False), dict(packed=False)):
+        stack = g.GsitStack([weights_to_dev(w, "bf16") for w in inp["fwd_layers"]],
+                            [weights_to_dev(w, "bf16") for w in inp["bwd_layers"]],
+                            [weights_to_dev(w, "bf16") for w in inp["intra_layers"]], wl.seg_len, wl.heads, ih, **kw)
+        first = stack.forward(x_dev, vl).clone()
+        torch.cuda.synchronize()
+        for run in range(12):
+            y = stack.forward(x_dev, vl)
+            torch.cuda.synchronize()
+            assert torch.equal(y, first), (kw, run)
+    assert g.last_device_status() == (0, 0)
+
+
 def test_cfg5_full_batch_attention_and_projection_sampled_samples(g):
     """The scaled shape at B = 128: tcgen05 attention (all three patterns) and the tcgen05 QKV projection."""
     wl = wk.WORKLOADS[5]
