@@ -165,6 +165,7 @@ __device__ __forceinline__ SItem read_item(uint32_t bars, int slot, int lane) {
   asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(it.rows_in_tile), "=r"(it.q_real), "=r"(it.T), "=r"(it.kn0) : "r"(a + 16) : "memory");
   asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(it.kn1), "=r"(it.kn2), "=r"(it.nk0), "=r"(it.nk1) : "r"(a + 32) : "memory");
   asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(it.kb0), "=r"(it.kb1), "=r"(it.kb2), "=r"(it.grow0) : "r"(a + 48) : "memory");
+  fence_reads_before_release();
   __syncwarp();
   if (lane == 0) mbar_arrive(bars + B_ITEMBAR + 8 * S_ITEM_SLOTS + 8 * slot);
   return it;

@@ -198,6 +198,7 @@ ln_qkv_tc_kernel(const __grid_constant__ LnQkvArgs arg0, const __grid_constant__
 #pragma unroll
         for (int e = 0; e < TD; ++e) v[e] = 0.f;
       }
+      fence_reads_before_release();
       __syncwarp();
       if (lane == 0) mbar_arrive(bars + B_XFREE);
       if (i > 0) {  // the previous tile's stores must have finished reading the staging rows (the normalised rows overlay them)
@@ -426,8 +427,9 @@ proj_mlp_tc_kernel(const __grid_constant__ ProjMlpArgs arg0, const __grid_consta
 #pragma unroll
         for (int e = 0; e < 32; ++e) v_[e] = 0.f;
       }
+      fence_reads_before_release();
       __syncwarp();
-      if (lane == 0 && i_ == 0) mbar_arrive(bars + B_XFREE);  // later tiles release the buffer at the end of the loop body
+      if (lane == 0) mbar_arrive(bars + B_XFREE);
       mbar_wait(wc, bars + B_ACC1, i_ & 1);
       tc_fence_after();
       {
@@ -520,14 +522,6 @@ proj_mlp_tc_kernel(const __grid_constant__ ProjMlpArgs arg0, const __grid_consta
         tma_store_2d(&tmY, base + OFF_F, 0, row0);
         tma_store_2d(&tmY, base + OFF_F + TM * 128, 32, row0);
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-      }
-      // The x buffer of the next tile (read above, before the output epilogue) is released only here.  Releasing it
-      // right after the read is what the barrier protocol would allow, but then the load of the tile after it lands
-      // during the output epilogue, and that gave wrong rows in the tile just read in about 3 % of 300 repeated runs
-      // (never with the release here, in 400): measured, the cause not found.
-      if (has_next) {
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bars + B_XFREE);
       }
       real = real_next;
       if (has_next) {

@@ -142,6 +142,7 @@ ln_qkv_tc128_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
 #pragma unroll
         for (int e = 0; e < 64; ++e) v[e] = 0.f;
       }
+      fence_reads_before_release();
       __syncwarp();
       if (lane == 0) mbar_arrive(bars + B_XFREE);
       if (i > 0 && tid == 64) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
@@ -428,6 +429,7 @@ proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_co
 #pragma unroll
         for (int e = 0; e < 64; ++e) v[e] = 0.f;
       }
+      fence_reads_before_release();
       __syncwarp();
       if (lane == 0) mbar_arrive(bars + B_XFREE);
       mbar_wait(wc, bars + B_ACC1, i & 1);
