@@ -481,8 +481,8 @@ proj_mlp_tc_kernel(const __grid_constant__ ProjMlpArgs arg0, const __grid_consta
           const float4 bb = ld_v4f(s_b1 + (c0 + e) * 4);
           const float2 h0 = __fadd2_rn(make_float2(__uint_as_float(a[e]), __uint_as_float(a[e + 1])), make_float2(bb.x, bb.y));
           const float2 h1 = __fadd2_rn(make_float2(__uint_as_float(a[e + 2]), __uint_as_float(a[e + 3])), make_float2(bb.z, bb.w));
-          pk[e >> 1] = pack_bf16(fmaxf(h0.x, 0.f), fmaxf(h0.y, 0.f));
-          pk[(e >> 1) + 1] = pack_bf16(fmaxf(h1.x, 0.f), fmaxf(h1.y, 0.f));
+          pk[e >> 1] = pack_bf16_relu(h0.x, h0.y);
+          pk[(e >> 1) + 1] = pack_bf16_relu(h1.x, h1.y);
         }
         const uint32_t blk = base + OFF_F + (c0 >> 6) * (TM * 128);
         const int ch0 = (c0 & 32) >> 3;

@@ -474,8 +474,8 @@ proj_mlp_tc128_kernel(const __grid_constant__ CUtensorMap tmAtt, const __grid_co
             const float4 bb = ld_v4f(s_b1 + (64 * c + 32 * hf + e) * 4);
             const float2 h0 = __fadd2_rn(make_float2(__uint_as_float(a[e]), __uint_as_float(a[e + 1])), make_float2(bb.x, bb.y));
             const float2 h1 = __fadd2_rn(make_float2(__uint_as_float(a[e + 2]), __uint_as_float(a[e + 3])), make_float2(bb.z, bb.w));
-            pk[e >> 1] = pack_bf16(fmaxf(h0.x, 0.f), fmaxf(h0.y, 0.f));
-            pk[(e >> 1) + 1] = pack_bf16(fmaxf(h1.x, 0.f), fmaxf(h1.y, 0.f));
+            pk[e >> 1] = pack_bf16_relu(h0.x, h0.y);
+            pk[(e >> 1) + 1] = pack_bf16_relu(h1.x, h1.y);
           }
         }
         if (n > 0) mbar_wait(wc, bars + B_FFREE, (n - 1) & 1);  // the previous second product has read the hidden chunk
