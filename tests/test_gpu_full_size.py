@@ -139,5 +139,10 @@ def test_cfg5_full_batch_attention_and_projection_sampled_samples(g):
             q64 = to_np64(qkv[b:b + 1])
             ref = oracle.im_attention_dense(q64[:, :, 0], q64[:, :, 1], q64[:, :, 2], wl.seg_len, valid[b:b + 1], ph)
             check_close(to_np64(out[b:b + 1]), ref, "bf16", pm[b:b + 1], f"full-batch attention phase {ph}, sample {b}")
+        for run in range(10):  # the same launch again: the same bits, whichever CTA takes which work item
+            again = g.im_attention_fwd(qkv[:, :, 0], qkv[:, :, 1], qkv[:, :, 2], wl.seg_len, vl, ph)
+            assert torch.equal(again, out), (ph, run)
+    for run in range(10):
+        assert torch.equal(g.im_qkv_proj(x, w, None, wl.seg_len, wl.heads, vl), qkv), run
     code, flags = g.last_device_status()
     assert code == 0 and flags == 0
