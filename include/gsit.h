@@ -80,8 +80,10 @@ typedef struct gsit_shape {
    * either: activations are [packed_capacity, d] matrices of real rows, segment s of sample b at rows
    * row_start[3 b + s] .. + valid_len[b][s] - 1.  row_start is a DEVICE int32 array of 3 B + 1 entries written by
    * gsit_plan_rows (entry 3 B = the row after the last one); valid_len must be given.  Accepted by
-   * gsit_im_attention_fwd (bf16, every head_dim) and gsit_im_layer_fwd (bf16, d_model 64 or 128); other
-   * calls and shapes answer GSIT_ERR_UNSUPPORTED. */
+   * gsit_im_attention_fwd (bf16, every head_dim), gsit_im_layer_fwd (bf16, d_model 64 or 128) and gsit_im_qkv_proj
+   * (bf16, d_model a multiple of 64); other calls and shapes answer GSIT_ERR_UNSUPPORTED.  A call on samples
+   * b0 .. b1 - 1 passes valid_len + 3 b0 and row_start + 3 b0 with the same matrices (rows are absolute) and reads
+   * and writes the rows of those samples only. */
   const int32_t* row_start;
   int32_t packed_capacity;  /* rows of the packed matrices (>= the plan's last entry rounded up to 128) */
 } gsit_shape;

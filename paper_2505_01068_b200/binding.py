@@ -179,8 +179,19 @@ def trace_launches(kind: int, capacity: int = 8192) -> list[float]:
     return [float(buf[i]) for i in range(n.value)]
 
 
-def im_qkv_proj(x, w_qkv, b_qkv, seg_len, heads, valid_len=None, out=None):
-    """x [B, L, d] (last dim contiguous) -> qkv [B, L, 3, H, hd]."""
+def im_qkv_proj(x, w_qkv, b_qkv, seg_len, heads, valid_len=None, out=None, row_start=None):
+    """x [B, L, d] (last dim contiguous) -> qkv [B, L, 3, H, hd].
+    With row_start (from plan_rows; bf16, d a multiple of 64) x is the packed matrix [capacity, d] and qkv
+    [capacity, 3, H, hd]; valid_len gives the batch size, and only the rows of these samples are computed and written."""
+    if row_start is not None:
+        cap, d = x.shape
+        assert x.is_cuda and x.stride(1) == 1 and w_qkv.is_contiguous() and valid_len is not None
+        shape = make_shape(valid_len.shape[0], seg_len, d, heads, valid_len, _dtype_code(x.dtype), PHASE_INTRA, 0, 0.0, row_start, cap)
+        if out is None:
+            out = torch.zeros((cap, 3, heads, d // heads), dtype=x.dtype, device=x.device)
+        _check(load().gsit_im_qkv_proj(ctypes.byref(shape), _ptr(x), x.stride(0), _ptr(w_qkv), _ptr(b_qkv), _ptr(out),
+                                       _stream()), "gsit_im_qkv_proj")
+        return out
     B, L, d = x.shape
     assert x.is_cuda and x.stride(2) == 1 and x.stride(0) == L * x.stride(1) and w_qkv.is_contiguous()
     shape = make_shape(B, seg_len, d, heads, valid_len, _dtype_code(x.dtype), PHASE_INTRA)

@@ -42,6 +42,8 @@ struct GemmParams {
   const float* residual; int64_t ldr;
   void* C; int64_t ldc;
   int relu, out_f32, mask_rows;
+  int packed;        // rows are the packed layout's: only rows_begin(g) .. rows_end(g) - 1 (read on the device) are computed
+                     // and written, all of them real; everything outside that range is left untouched
   int tma_store;     // bf16 output through the shared-memory staging area and TMA stores
   int staging_off;   // offset of the staging area from the aligned base
 };
@@ -70,12 +72,16 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   tc_fence_after();
   uint32_t tmem;
   asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tmem) : "r"(slot) : "memory");
+  // rows this call computes; a row tile wholly outside them is skipped by every role alike
+  const int row_lo = p.packed ? rows_begin(g) : 0, row_hi = p.packed ? rows_end(g) : p.M;
+  auto tile_outside = [&](int m0) { return m0 + GM <= row_lo || m0 >= row_hi; };
 
   if (warp == 0) {
     // ================================ TMA producer ================================
     int n = 0;  // k-blocks requested so far
     for (int t = blockIdx.x; t < p.n_tiles; t += gridDim.x) {
       const int m0 = (t / p.tiles_n) * GM, n0 = (t % p.tiles_n) * p.bn;
+      if (tile_outside(m0)) continue;
       for (int kb = 0; kb < kblocks; ++kb, ++n) {
         const int st = n % p.stages, use = n / p.stages;
         if (use > 0) mbar_wait(wc, bar_empty + 8 * st, (use - 1) & 1);
@@ -92,7 +98,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     // ================================ MMA issuer ================================
     const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.bn >> 3) << 17) | ((uint32_t)(GM >> 4) << 24);
     int n = 0, i = 0;  // k-blocks consumed, tiles done by this CTA
-    for (int t = blockIdx.x; t < p.n_tiles; t += gridDim.x, ++i) {
+    for (int t = blockIdx.x; t < p.n_tiles; t += gridDim.x) {
+      if (tile_outside((t / p.tiles_n) * GM)) continue;
       const int ab = i & 1;
       if (i >= 2) mbar_wait(wc, bar_acce + 8 * ab, ((i >> 1) - 1) & 1);  // the epilogue has drained this accumulator
       tc_fence_after();
@@ -110,18 +117,20 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
         __syncwarp();
       }
+      ++i;
     }
   } else {
     // ================================ epilogue: one thread per output row ================================
     const int quarter = warp & 3;
     const uint32_t tl = tmem + ((uint32_t)(quarter << 5) << 16);
     int i = 0;
-    for (int t = blockIdx.x; t < p.n_tiles; t += gridDim.x, ++i) {
-      const int ab = i & 1;
+    for (int t = blockIdx.x; t < p.n_tiles; t += gridDim.x) {
       const int m0 = (t / p.tiles_n) * GM, n0 = (t % p.tiles_n) * p.bn;
+      if (tile_outside(m0)) continue;
+      const int ab = i & 1;
       const int64_t row = (int64_t)m0 + quarter * 32 + lane;
-      const bool in_m = row < p.M;
-      const bool real = in_m && (!p.mask_rows || row_is_real(g, row));
+      const bool in_m = row >= row_lo && row < row_hi;
+      const bool real = in_m && (!p.mask_rows || p.packed || row_is_real(g, row));
       mbar_wait(wc, bar_accf + 8 * ab, (i >> 1) & 1);
       tc_fence_after();
       if (p.tma_store) {
@@ -164,6 +173,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             if (n0 + 64 * j < p.N) tma_store_2d(&tmC, stg + j * 16384, n0 + 64 * j, m0);
           asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         }
+        ++i;
         continue;
       }
       for (int c0 = 0; c0 < p.bn; c0 += 32) {
@@ -216,6 +226,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_acce + 8 * ab);
+      ++i;
     }
   }
 
@@ -249,7 +260,10 @@ cudaError_t launch_linear_tc_bf16(const Geometry& g, const LinearArgs& a, cudaSt
   p.stage_bytes = A_STAGE + ((p.bn * GK * 2 + 1023) & ~1023);
   p.bias = a.bias; p.residual = a.residual; p.ldr = a.ldr; p.C = a.C; p.ldc = a.ldc;
   p.relu = a.relu; p.out_f32 = a.out_f32; p.mask_rows = a.mask_rows;
-  p.tma_store = (!a.out_f32 && a.residual == nullptr && p.bn % 64 == 0 && a.N % 8 == 0 &&
+  p.packed = (g.row_start != nullptr) ? 1 : 0;
+  // TMA stores write whole tiles; in the packed layout the rows of a boundary tile that lie outside this call's range
+  // belong to other samples, so there every thread stores its own row
+  p.tma_store = (!p.packed && !a.out_f32 && a.residual == nullptr && p.bn % 64 == 0 && a.N % 8 == 0 &&
                  (reinterpret_cast<uintptr_t>(a.C) & 15u) == 0) ? 1 : 0;
   const int staging = p.tma_store ? (p.bn / 64) * 16384 : 0;
   const int budget = 227 * 1024 - 1024 - G_BAR_BYTES - staging;

@@ -200,7 +200,6 @@ gsit_status gsit_im_qkv_proj(const gsit_shape* shape, const void* x, int64_t x_r
   Geometry g;
   gsit_status st = make_geometry(shape, &g);
   if (st != GSIT_OK) return st;
-  if (g.row_start != nullptr) return GSIT_ERR_UNSUPPORTED;  // the packed layout reaches this projection through the layer call
   if (!x || !w_qkv || !qkv || x_row_stride < g.d) return GSIT_ERR_INVALID_ARG;
   if (!aligned16(x) || !aligned16(w_qkv) || !aligned16(qkv)) return GSIT_ERR_INVALID_ARG;
   if (shape->dtype == GSIT_BF16 && x_row_stride % 8 != 0) return GSIT_ERR_INVALID_ARG;
@@ -208,8 +207,14 @@ gsit_status gsit_im_qkv_proj(const gsit_shape* shape, const void* x, int64_t x_r
   LinearArgs a = {};
   a.A = x; a.lda = x_row_stride; a.W = w_qkv; a.bias = b_qkv;
   a.C = qkv; a.ldc = 3 * (int64_t)g.d;
-  a.M = g.batch * g.L; a.N = 3 * g.d; a.K = g.d;
+  a.M = (int)matrix_rows(g); a.N = 3 * g.d; a.K = g.d;
   a.mask_rows = 1;
+  if (g.row_start != nullptr) {
+    // packed rows: the tcgen05 kernel computes and writes this call's row range only (widths it covers: multiples of 64)
+    if (shape->dtype != GSIT_BF16 || !linear_tc_supported(a)) return GSIT_ERR_UNSUPPORTED;
+    TraceScope t(GSIT_KERNEL_LINEAR, static_cast<cudaStream_t>(stream));
+    return from_cuda(launch_linear_tc_bf16(g, a, static_cast<cudaStream_t>(stream)));
+  }
   return run_linear(g, shape->dtype, a, static_cast<cudaStream_t>(stream));
 }
 

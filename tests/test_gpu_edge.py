@@ -183,6 +183,41 @@ def test_attention_on_packed_rows_equals_padded_layout(g, H, hd):
     assert g.last_device_status() == (0, 0)
 
 
+def test_projection_on_packed_rows_equals_padded_layout_and_leaves_other_rows_alone(g):
+    """gsit_im_qkv_proj on the packed row layout: the real rows get the bits of the padded layout; a call on a sub-range
+    of the samples writes their rows only (tiles at the edges of the range are shared with the neighbours)."""
+    rng = np.random.default_rng(77)
+    seg, B, d, H = (70, 200, 150), 5, 128, 8
+    L = sum(seg)
+    valid = np.array([[70, 200, 150], [33, 129, 65], [70, 0, 1], [0, 0, 0], [61, 77, 150]], dtype=np.int32)
+    vl = torch.from_numpy(valid).cuda()
+    x = to_dev(rng.standard_normal((B, L, d)).astype(np.float32), "bf16")
+    w = to_dev((rng.standard_normal((3 * d, d)) * d ** -0.5).astype(np.float32), "bf16")
+    bias = to_dev(rng.standard_normal(3 * d).astype(np.float32))
+    want = g.im_qkv_proj(x, w, bias, seg, H, vl).reshape(B, L, 3 * d)
+    cap = B * L + 128
+    plan = g.plan_rows(vl, seg)
+    plan_h = plan.cpu().numpy()
+    off = np.cumsum([0] + list(seg))
+    xp = torch.full((cap, d), float("nan"), dtype=torch.bfloat16, device="cuda")
+    for b in range(B):
+        for s_ in range(3):
+            n = int(valid[b, s_])
+            xp[plan_h[3 * b + s_]:plan_h[3 * b + s_] + n] = x[b, off[s_]:off[s_] + n]
+    for lo, hi in ((0, B), (1, 3), (4, 5)):
+        out = torch.full((cap, 3, H, d // H), 7.0, dtype=torch.bfloat16, device="cuda")
+        g.im_qkv_proj(xp, w, bias, seg, H, vl[lo:hi], out=out, row_start=plan[3 * lo:])
+        torch.cuda.synchronize()
+        flat = out.reshape(cap, 3 * d)
+        begin, end = int(plan_h[3 * lo]), int(plan_h[3 * hi])
+        for b in range(lo, hi):
+            for s_ in range(3):
+                n = int(valid[b, s_])
+                assert torch.equal(flat[plan_h[3 * b + s_]:plan_h[3 * b + s_] + n], want[b, off[s_]:off[s_] + n]), (lo, hi, b, s_)
+        assert bool((flat[:begin] == 7.0).all()) and bool((flat[end:] == 7.0).all()), (lo, hi)
+    assert g.last_device_status() == (0, 0)
+
+
 def test_bounded_wait_runs_out_and_is_reported(g):
     """A device-side wait that nothing will ever satisfy gives up after its poll limit: the kernel returns, the status
     word carries the timeout flag exactly once, and the next ordinary call is clean."""
