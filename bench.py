@@ -458,7 +458,27 @@ def run_gpu(args):
         sec = beg.elapsed_time(end) * 1e-3 / 10
         fl = 2.0 * wl5.batch * wl5.L * wl5.d_model * 3 * wl5.d_model
         scaled["qkv_proj"] = {"us": sec * 1e6, "tflops": fl / sec / 1e12, "frac_tensor_peak": fl / sec / 1e12 / pk["bf16_tflops"],
-                              "note": "all B*L rows multiplied (padded rows are zeroed in the epilogue)"}
+                              "note": "padded layout: all B*L rows multiplied (padded rows are zeroed in the epilogue)"}
+        # the same projection on the packed row layout: real rows only
+        cap5 = wl5.batch * wl5.L + 128
+        plan5 = g.plan_rows(vl5, wl5.seg_len)
+        xp5 = [torch.cat([x.reshape(-1, wl5.d_model), torch.zeros((128, wl5.d_model), device="cuda", dtype=torch.bfloat16)]) for x in xs5]
+        qp5 = [torch.empty((cap5, 3, wl5.heads, wl5.d_model // wl5.heads), device="cuda", dtype=torch.bfloat16) for _ in range(2)]
+        for i in range(2):
+            g.im_qkv_proj(xp5[i], w5, None, wl5.seg_len, wl5.heads, vl5, out=qp5[i], row_start=plan5)
+        torch.cuda.synchronize()
+        beg.record()
+        for _ in range(5):
+            for i in range(2):
+                g.im_qkv_proj(xp5[i], w5, None, wl5.seg_len, wl5.heads, vl5, out=qp5[i], row_start=plan5)
+        end.record()
+        torch.cuda.synchronize()
+        sec_p = beg.elapsed_time(end) * 1e-3 / 10
+        fl_real = 2.0 * tok5 * wl5.d_model * 3 * wl5.d_model
+        scaled["qkv_proj_packed"] = {"us": sec_p * 1e6, "tflops_real_rows": fl_real / sec_p / 1e12,
+                                     "padded_layout_tflops_real_rows": fl_real / sec / 1e12, "real_rows": tok5,
+                                     "note": "packed layout: real rows only, rows stored one by one instead of by TMA"}
+        del xp5, qp5
         del vl5, xs5, qs5
         torch.cuda.empty_cache()
 
